@@ -1,0 +1,274 @@
+#!/usr/bin/env python
+"""Benchmark of the 3D complex DFT hot path (one JSON line on stdout).
+
+A "step" is one whole 3D complex-to-complex transform of a seeded synthetic n^3 cube through the
+C-ABI library (`dft3d_execute`: three per-axis tensor-core GEMM passes).  Default workload: the
+1024^3 cube the headline metric is quoted on, input U(-1,1).  `value` is GFLOP/s in the 5*P*log2(P)
+convention (P = n^3 points), with the input already resident in HBM; `e2e` is the same metric
+through `dft3d_execute_host` with pinned HOST buffers (H2D and D2H copies inside the timed region).
+
+python bench.py [--gpus N] [--steps K] [--warmup W] [--mode kdft|fft] [--n 1024] [--impl reference]
+Under torchrun every rank transforms its own cube (independent problems, no collective): weak scaling.
+"""
+import argparse
+import json
+import math
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+SMI_QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--mode", choices=["kdft", "fft"], default=None)
+    ap.add_argument("--n", type=int, default=1024)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg")
+    ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing leg")
+    return ap.parse_args()
+
+
+def conv_flops(n):
+    P = float(n) ** 3
+    return 5.0 * P * math.log2(P)
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return json.load(f), "measured"
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}, "fallback"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons of one GPU while the timed region runs."""
+
+    def __init__(self, index):
+        self.index = index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.out = open(self.path, "w")
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + SMI_QUERY, "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=self.out, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.out.close()
+        clocks, maxc, power, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        with open(self.path) as f:
+            for line in f:
+                parts = [p.strip() for p in line.split(",")]
+                if len(parts) < 9:
+                    continue
+                try:
+                    clocks.append(float(parts[1]))
+                    maxc.append(float(parts[2]))
+                    power.append(float(parts[3]))
+                except ValueError:
+                    continue
+                for name, val in zip(names, parts[5:9]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+        os.unlink(self.path)
+        if not clocks:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        load = sorted(c for c, p in zip(clocks, power) if p >= 0.5 * max(power)) or sorted(clocks)
+        return {"sm_mhz": load[len(load) // 2], "sm_max_mhz": max(maxc), "power_w_max": max(power),
+                "samples": len(clocks), "reasons": sorted(reasons)}
+
+
+def oracle_sample(n, planes, seed):
+    """Times the oracle, as it stands, on `planes` n0-planes of the workload along the last axis and
+    extrapolates by the exact operation count (3 axes x n complex MACs per point) to a full transform."""
+    import numpy as np
+    from oracle import oracle
+    from paper_2002_03260_b200 import inputs
+    oracle.build()
+    x = inputs.cube((planes, n, n), "uniform", seed, device="cpu").numpy().astype(np.complex128)
+    t0 = time.perf_counter()
+    oracle.dft_axis(x, 2)
+    dt = time.perf_counter() - t0
+    full_seconds = dt * (n / planes) * 3.0
+    return {"value": conv_flops(n) / full_seconds * 1e-9, "unit": "GFLOP/s (5*P*log2P)", "cores": oracle.num_threads(),
+            "kind": "oracle",
+            "sample": "float64 direct summation of the last axis over %d of %d n0-planes (%.2f s), extrapolated by the "
+                      "exact operation count (3 axes x %d complex MACs per point) to %.0f s per transform"
+                      % (planes, n, dt, n, full_seconds),
+            "seconds_per_transform_extrapolated": full_seconds}
+
+
+def run_reference(args):
+    """--impl reference: the oracle on the host cores, each step a bounded sample of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    n = args.n
+    planes = max(1, min(n, int(2.0e9 / (float(n) ** 3))))  # about 2e9 complex MACs per step
+    times = []
+    res = None
+    for i in range(args.warmup + args.steps):
+        res = oracle_sample(n, planes, 1003)
+        if i >= args.warmup:
+            times.append(res["seconds_per_transform_extrapolated"])
+    sec = sum(times) / len(times)
+    value = conv_flops(n) / sec * 1e-9
+    line = {"impl": "reference", "metric": "3D C2C DFT GFLOP/s (5*P*log2P) at %d^3" % n, "value": value,
+            "unit": "GFLOP/s", "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f64", "data": "synthetic",
+            "config": {"workload": "%d^3 complex64 cube, U(-1,1), float64 direct-summation oracle" % n},
+            "cpu_baseline": {"value": value, "unit": "GFLOP/s", "cores": res["cores"], "kind": "oracle",
+                             "sample": res["sample"]},
+            "e2e": {"value": value, "unit": "GFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+    import torch
+    import torch.distributed as dist
+    import paper_2002_03260_b200 as dft
+    from paper_2002_03260_b200 import inputs
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the transform has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    n = args.n
+    mode = args.mode or "kdft"
+    mode_id = dft.DFT3D_KDFT if mode == "kdft" else dft.DFT3D_FFT
+    shape = (n, n, n)
+    x = inputs.cube(shape, "uniform", 1003 + rank, device="cuda")
+    y = torch.empty_like(x)
+    plan = dft.Plan(*shape, mode=mode_id, sign=dft.DFT3D_FORWARD)
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        plan.execute(x, y)
+    barrier()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    ev[0].record(stream)
+    for i in range(args.steps):
+        plan.execute(x, y)
+        ev[i + 1].record(stream)
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    plan.status()
+    ms_total = ev[0].elapsed_time(ev[-1])
+    t = torch.tensor([ms_total], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_step = float(t.item()) / args.steps
+    launches = plan.launches
+
+    # ---- end to end through the host-buffer entry point
+    e2e = None
+    if not args.no_e2e:
+        xh = x.cpu().pin_memory()
+        yh = torch.empty_like(xh).pin_memory()
+        plan.execute_host(xh, yh)   # warm-up, allocates the staging buffers
+        barrier()
+        e2e_steps = max(1, min(args.steps, 3))
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(e2e_steps):
+            plan.execute_host(xh, yh)
+        e1.record(stream)
+        barrier()
+        te = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device="cuda")
+        if world > 1:
+            dist.all_reduce(te, op=dist.ReduceOp.MAX)
+        ms_e2e = float(te.item()) / e2e_steps
+        nbytes = x.numel() * 8
+        e2e = {"value": world * conv_flops(n) / ms_e2e * 1e-6, "unit": "GFLOP/s", "ms_per_step": ms_e2e,
+               "h2d_bytes_per_step": nbytes, "d2h_bytes_per_step": nbytes, "steps": e2e_steps,
+               "call": "dft3d_execute_host (pinned host buffers)"}
+        del xh, yh
+
+    if rank == 0:
+        peaks, peak_kind = measured_peaks()
+        P = float(n) ** 3
+        if mode == "kdft":
+            # dominant (only) kernel: kdft_axis_kernel; algorithmic flops per point per axis = 8*n (4 real
+            # multiply-adds per complex MAC), issued three times for the TF32 split
+            algo_flops = 3 * 8.0 * n * P
+            issued_flops = 3.0 * algo_flops
+            tf32_peak = peaks["bf16_tflops_sustained"] * (1.1 / 2.25)
+            achieved = issued_flops / (ms_step * 1e-3) * 1e-12
+            roofline = {"bound": "tensor", "kernel": "kdft_axis_kernel", "achieved": achieved, "peak": tf32_peak,
+                        "unit": "TFLOP/s", "frac": achieved / tf32_peak, "traffic": None,
+                        "peak_source": "%s bf16 sustained x nominal TF32/bf16 ratio (1.1/2.25)" % peak_kind,
+                        "flops": "issued TF32 tensor flops = 3 split products x 8*n flops per point per axis",
+                        "useful_gemm_tflops": algo_flops / (ms_step * 1e-3) * 1e-12,
+                        "avg_launch_ms": ms_step / launches}
+        else:
+            algo_bytes = 3 * 16.0 * P
+            achieved = algo_bytes / (ms_step * 1e-3) * 1e-9
+            roofline = {"bound": "hbm", "kernel": "fft_axis_kernel", "achieved": achieved, "peak": peaks["hbm_gbs"],
+                        "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "traffic": None,
+                        "peak_source": "%s STREAM-style copy" % peak_kind, "avg_launch_ms": ms_step / launches}
+        cpu = None
+        if not args.no_cpu_baseline:
+            planes = max(1, min(n, int(3.0e10 / (float(n) ** 3))))
+            cpu = oracle_sample(n, planes, 1003)
+        line = {"metric": "3D C2C DFT GFLOP/s (5*P*log2P) at %d^3" % n,
+                "value": world * conv_flops(n) / ms_step * 1e-6, "unit": "GFLOP/s", "n_gpus": world,
+                "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": "tf32x3", "data": "synthetic",
+                "config": {"workload": "%s forward 3D complex64 DFT %d^3, re/im iid U(-1,1), seed 1003+rank" % (mode.upper(), n),
+                           "mode": mode, "n": n, "l2": "input and output (%.1f GiB each) are larger than L2" % (P * 8 / 2**30),
+                           "per_rank": "one independent cube per GPU"},
+                "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches * args.steps,
+                "clocks": clocks}
+        print(json.dumps(line))
+    plan.destroy()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,155 @@
+/*
+ * dft3d -- 3D complex-to-complex discrete Fourier transform on one NVIDIA B200,
+ * computed as dense matrix multiplications on the tensor cores.
+ *
+ * Two formulations of the same transform (both from "Large-Scale Discrete
+ * Fourier Transform on TPUs", arXiv 2002.03260):
+ *
+ *   KDFT (Section III-A, Eq. 11-13): every axis is multiplied by its N x N
+ *        Vandermonde / DFT matrix.  The matrix may be built from nonuniform
+ *        sample nodes (Eq. 3 with the sample points on the unit circle).
+ *   FFT  (Section III-B, Eq. 14-18): every axis of length N = N1*N2 becomes a
+ *        length-N1 DFT (matrix product), an elementwise phase adjustment
+ *        (twiddle), and a length-N2 DFT (matrix product); output in natural
+ *        order.  Uniform grids only.
+ *
+ * Data layout everywhere: row-major [n0][n1][n2], interleaved complex64
+ * (re, im as two float32), 8 bytes per point.
+ *
+ * All functions return a DFT3D_* status and never throw or abort.  A short
+ * description of the most recent failure on the calling thread is available
+ * from dft3d_last_error().
+ */
+#ifndef DFT3D_H_
+#define DFT3D_H_
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct dft3d_plan_s* dft3d_plan_t;
+
+enum { DFT3D_KDFT = 0, DFT3D_FFT = 1 };          /* mode */
+enum { DFT3D_FORWARD = -1, DFT3D_INVERSE = +1 }; /* sign of the exponent (Eq. 14 has the minus sign) */
+
+enum {
+  DFT3D_OK = 0,
+  DFT3D_ERR_INVALID_ARG = 1,    /* NULL where not allowed, n < 1, bad mode/sign, non-finite node, misaligned pointer */
+  DFT3D_ERR_UNSUPPORTED = 2,    /* size or option outside what the kernels handle (see dft3d_plan_create) */
+  DFT3D_ERR_ALLOC = 3,          /* host or device allocation failed */
+  DFT3D_ERR_CUDA = 4,           /* a CUDA runtime/driver call failed */
+  DFT3D_ERR_DEVICE_TIMEOUT = 5  /* a kernel gave up a bounded wait; the output of that execute is invalid */
+};
+
+/* option flags */
+enum {
+  DFT3D_NODES_ON_OUTPUT = 1u,   /* M[k,j] = exp(s*2*pi*i * node[k] * j): Eq. 1 read literally (arbitrary
+                                   evaluation points, integer powers).  Default is M[k,j] = exp(s*2*pi*i * k * node[j])
+                                   (nonuniform input samples, integer output frequencies). */
+  DFT3D_UNSCALED_INVERSE = 2u   /* sign=+1 without the 1/n_a factors */
+};
+
+typedef struct dft3d_options_s {
+  size_t struct_size;     /* sizeof(dft3d_options_t), for forward compatibility */
+  unsigned flags;         /* DFT3D_NODES_ON_OUTPUT | DFT3D_UNSCALED_INVERSE */
+  int fft_split[3][2];    /* FFT mode: {N1, N2} per axis with N1*N2 = n_a; {0,0} = default split */
+  size_t workspace_limit; /* KDFT mode: upper bound in bytes for the plan-owned workspace; 0 = default */
+} dft3d_options_t;
+
+/*
+ * Create a plan for an n0 x n1 x n2 transform (Eq. 11 / Eq. 12).
+ *
+ *   out      receives the handle; set to NULL on failure.
+ *   mode     DFT3D_KDFT or DFT3D_FFT.
+ *   sign     DFT3D_FORWARD: kernel exp(-2*pi*i*k*t), unscaled (Eq. 14).
+ *            DFT3D_INVERSE: conjugate kernel, each axis scaled by 1/n_a so that
+ *            inverse(forward(x)) = x on uniform grids (the paper describes the inverse
+ *            as solving Eq. 2; on a uniform grid that solve is this product).
+ *   nodesA   HOST pointer to n_a doubles, or NULL for the uniform grid t_j = j/n_a.
+ *            Any finite value is accepted and used modulo 1.  Copied during the call.
+ *            With nodes and sign=+1 the result is the conjugate-kernel product, not an
+ *            inverse of the nonuniform transform.  FFT mode takes no nodes.
+ *
+ * The DFT / Vandermonde matrices and twiddles are evaluated in float64 with exactly
+ * reduced phases and rounded once to the stored float32 pieces.  The plan owns its
+ * device tables and workspace (allocated on the current device during this call).
+ *
+ * Supported sizes: every n_a a multiple of 64, n_a <= 8192 (KDFT) ; FFT additionally needs
+ * N1 and N2 multiples of 16.  Other sizes return DFT3D_ERR_UNSUPPORTED.
+ */
+int dft3d_plan_create(dft3d_plan_t* out, long long n0, long long n1, long long n2, int mode, int sign,
+                      const double* nodes0, const double* nodes1, const double* nodes2);
+
+/* Same, with options (may be NULL). */
+int dft3d_plan_create_ex(dft3d_plan_t* out, long long n0, long long n1, long long n2, int mode, int sign,
+                         const double* nodes0, const double* nodes1, const double* nodes2,
+                         const dft3d_options_t* options);
+
+/*
+ * Run the transform (all three axes; Eq. 12 for KDFT, Eq. 17 per axis for FFT).
+ *
+ *   in, out      DEVICE pointers, 16-byte aligned, n0*n1*n2*8 bytes each, not overlapping.
+ *                `in` is only read.
+ *   cuda_stream  a cudaStream_t (NULL = default stream).
+ *
+ * Asynchronous: kernels are enqueued on the stream and the call returns without
+ * synchronising.  No allocation happens here.  One execute per plan may be in flight.
+ * After the stream has been synchronised, dft3d_plan_status() tells whether any kernel
+ * abandoned a bounded wait.
+ */
+int dft3d_execute(dft3d_plan_t plan, const void* in, void* out, void* cuda_stream);
+
+/*
+ * Convenience for callers whose data lives in HOST memory (pinned memory makes the copies
+ * faster): copies `host_in` to a plan-owned device buffer, runs dft3d_execute, copies the
+ * result to `host_out`, and synchronises the stream before returning.  The device buffers
+ * are allocated on first use and kept until the plan is destroyed.
+ */
+int dft3d_execute_host(dft3d_plan_t plan, const void* host_in, void* host_out, void* cuda_stream);
+
+/* Transform one axis only (0, 1 or 2) with the plan's matrix for that axis; same pointer rules as
+ * dft3d_execute.  KDFT: Eq. 5's left / right multiplication for that axis.  FFT: Eq. 17 along that axis. */
+int dft3d_execute_axis(dft3d_plan_t plan, int axis, const void* in, void* out, void* cuda_stream);
+
+/* DFT3D_OK, or DFT3D_ERR_DEVICE_TIMEOUT if a kernel of an earlier execute gave up a wait.
+ * Reads a plan-owned device word (a small synchronous copy); call it after synchronising. */
+int dft3d_plan_status(dft3d_plan_t plan);
+
+/* Bytes of device workspace the plan owns (0 for NULL). */
+size_t dft3d_plan_workspace_bytes(dft3d_plan_t plan);
+
+/* Number of kernels one dft3d_execute enqueues (0 for NULL). */
+int dft3d_plan_launches(dft3d_plan_t plan);
+
+/* Frees device and host memory of the plan.  NULL is accepted. */
+int dft3d_plan_destroy(dft3d_plan_t plan);
+
+const char* dft3d_status_string(int status);
+const char* dft3d_last_error(void);
+
+/*
+ * The table generator, exposed so that it can be checked on a machine without a GPU
+ * (HOST pointers only; no CUDA call is made).
+ *
+ * dft3d_generate_axis_matrix: the n x n complex matrix of one axis in float64,
+ *   M[k][j] interleaved (re, im), 2*n*n doubles.  (Eq. 3 / Eq. 13; Eq. 14 when nodes == NULL.)
+ * dft3d_generate_twiddle: T[k1][beta] = exp(sign*2*pi*i*k1*beta/(N1*N2)), N1*N2 complex doubles
+ *   (the phase adjustment of Eq. 17).
+ * dft3d_generate_real_table: the real 2n x 2n matrix W with W[2k+p][2j+q] =
+ *   (p==q ? Re M[k][j] : (p ? +Im : -Im) M[k][j]) that turns the complex product into a real
+ *   one on interleaved data, split into two float32 pieces hi + lo (hi has a 10-bit
+ *   mantissa, i.e. is exact in TF32; lo is the float32 rounding of the remainder rounded to
+ *   TF32).  Each piece is (2n)*(2n) floats, row-major.
+ */
+int dft3d_generate_axis_matrix(long long n, int sign, double scale, const double* nodes, int nodes_on_output,
+                               double* matrix);
+int dft3d_generate_twiddle(long long N1, long long N2, int sign, double* twiddle);
+int dft3d_generate_real_table(long long n, int sign, double scale, const double* nodes, int nodes_on_output,
+                              float* hi, float* lo);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DFT3D_H_ */

@@ -1,0 +1,456 @@
+// C-ABI of the dft3d library: plans, the float64 table generator entry points, and the launch
+// logic for the per-axis tensor-core kernels.  See include/dft3d.h for the contract of each call.
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include "../../include/dft3d.h"
+#include "generator.h"
+#include "kdft_kernel.cuh"
+#include "fft_kernel.cuh"
+
+namespace {
+
+thread_local char g_last_error[512] = "";
+
+int fail(int status, const char* fmt, ...) {
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(g_last_error, sizeof(g_last_error), fmt, ap);
+  va_end(ap);
+  return status;
+}
+
+#define DFT3D_CUDA(call)                                                                          \
+  do {                                                                                            \
+    cudaError_t e_ = (call);                                                                      \
+    if (e_ != cudaSuccess)                                                                        \
+      return fail(e_ == cudaErrorMemoryAllocation ? DFT3D_ERR_ALLOC : DFT3D_ERR_CUDA, "%s: %s", #call, \
+                  cudaGetErrorString(e_));                                                        \
+  } while (0)
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// The driver entry point is fetched through the runtime so that the library has no link-time
+// dependency on libcuda and can be loaded (for its host-only entry points) on a machine without a GPU.
+int get_encoder(EncodeTiledFn* fn) {
+  static EncodeTiledFn cached = nullptr;
+  if (!cached) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qr;
+    cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qr);
+    if (e != cudaSuccess || !p || qr != cudaDriverEntryPointSuccess)
+      return fail(DFT3D_ERR_CUDA, "cuTensorMapEncodeTiled is not available: %s", cudaGetErrorString(e));
+    cached = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  *fn = cached;
+  return DFT3D_OK;
+}
+
+// float32 tensor map with up to 3 dimensions; dims/box innermost first; strides in bytes for dims 1..rank-1
+int encode_f32(CUtensorMap* map, const void* base, int rank, const unsigned long long* dims,
+               const unsigned long long* strides_bytes, const unsigned* box, bool swizzle128) {
+  EncodeTiledFn enc;
+  int rc = get_encoder(&enc);
+  if (rc != DFT3D_OK) return rc;
+  cuuint64_t d[3], s[2];
+  cuuint32_t b[3], es[3];
+  for (int i = 0; i < rank; ++i) { d[i] = dims[i]; b[i] = box[i]; es[i] = 1; }
+  for (int i = 0; i + 1 < rank; ++i) s[i] = strides_bytes[i];
+  CUresult cr = enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, rank, const_cast<void*>(base), d, s, b, es,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (cr != CUDA_SUCCESS)
+    return fail(DFT3D_ERR_CUDA, "cuTensorMapEncodeTiled failed with %d (rank %d, dims %llu %llu %llu, box %u %u %u)",
+                int(cr), rank, dims[0], rank > 1 ? dims[1] : 0ull, rank > 2 ? dims[2] : 0ull, box[0],
+                rank > 1 ? box[1] : 0u, rank > 2 ? box[2] : 0u);
+  return DFT3D_OK;
+}
+
+struct KdftAxis {
+  long long n = 0;
+  float* d_w = nullptr;   // [2 pieces][2n][2n] floats
+  CUtensorMap map_w;
+  int bn = 0;
+};
+
+}  // namespace
+
+struct dft3d_plan_s {
+  long long n[3] = {0, 0, 0};
+  int mode = 0, sign = 0;
+  unsigned flags = 0;
+  int device = 0;
+  int sm_count = 0;
+  KdftAxis kax[3];
+  dft3d::FftAxis fax[3];
+  void* workspace = nullptr;
+  size_t workspace_bytes = 0;
+  long long group_planes = 0;   // n0-planes per workspace group (KDFT)
+  unsigned int* d_status = nullptr;
+  void* host_in_dev = nullptr;  // device staging for dft3d_execute_host
+  void* host_out_dev = nullptr;
+  bool attrs_set = false;
+};
+
+namespace {
+
+long long points(const dft3d_plan_s* p) { return p->n[0] * p->n[1] * p->n[2]; }
+
+int set_kernel_attributes() {
+  static bool done = false;
+  if (done) return DFT3D_OK;
+  DFT3D_CUDA(cudaFuncSetAttribute(dft3d::kdft_axis_kernel<dft3d::KDFT_CONTIG>,
+                                  cudaFuncAttributeMaxDynamicSharedMemorySize, int(dft3d::kKdftSmemBytes)));
+  DFT3D_CUDA(cudaFuncSetAttribute(dft3d::kdft_axis_kernel<dft3d::KDFT_STRIDED>,
+                                  cudaFuncAttributeMaxDynamicSharedMemorySize, int(dft3d::kKdftSmemBytes)));
+  int rc = dft3d::fft_set_kernel_attributes();
+  if (rc != 0) return fail(DFT3D_ERR_CUDA, "cudaFuncSetAttribute failed for the FFT kernels");
+  done = true;
+  return DFT3D_OK;
+}
+
+int build_kdft_axis(dft3d_plan_s* p, int a, const double* nodes) {
+  KdftAxis& ax = p->kax[a];
+  const long long n = p->n[a];
+  ax.n = n;
+  ax.bn = int(2 * n < 256 ? 2 * n : 256);
+  const bool scaled = (p->sign > 0) && !(p->flags & DFT3D_UNSCALED_INVERSE);
+  const double scale = scaled ? 1.0 / double(n) : 1.0;
+  std::vector<double> M;
+  std::vector<float> W;
+  try {
+    M.resize(size_t(2) * n * n);
+    W.resize(size_t(2) * 4 * n * n);
+  } catch (const std::bad_alloc&) {
+    return fail(DFT3D_ERR_ALLOC, "host allocation of the axis-%d table failed", a);
+  }
+  dft3d::gen::axis_matrix(n, p->sign, scale, nodes, (p->flags & DFT3D_NODES_ON_OUTPUT) != 0, M.data());
+  dft3d::gen::real_table_from_matrix(n, M.data(), W.data(), W.data() + size_t(4) * n * n);
+  DFT3D_CUDA(cudaMalloc(&ax.d_w, W.size() * sizeof(float)));
+  DFT3D_CUDA(cudaMemcpy(ax.d_w, W.data(), W.size() * sizeof(float), cudaMemcpyHostToDevice));
+  const unsigned long long dims[3] = {(unsigned long long)(2 * n), (unsigned long long)(2 * n), 2ull};
+  const unsigned long long strides[2] = {(unsigned long long)(2 * n * 4), (unsigned long long)(4 * n * n * 4)};
+  const unsigned box[3] = {unsigned(dft3d::kBlockK), unsigned(ax.bn), 2u};
+  return encode_f32(&ax.map_w, ax.d_w, 3, dims, strides, box, true);
+}
+
+// One KDFT axis pass over a [batches][J][C] complex view (STRIDED) or rows x J (CONTIG).
+int launch_kdft_strided(dft3d_plan_s* p, int a, const float* in, float* out, long long batches, long long C,
+                        cudaStream_t stream) {
+  const KdftAxis& ax = p->kax[a];
+  const long long J = ax.n;
+  dft3d::KdftParams kp;
+  memset(&kp, 0, sizeof(kp));
+  kp.k2 = int(2 * J);
+  kp.bn = ax.bn;
+  kp.n_tiles = int((2 * J + ax.bn - 1) / ax.bn);
+  kp.batches = batches;
+  kp.C = C;
+  kp.lpb = int(C < 128 ? C : 128);
+  kp.bpt = 128 / kp.lpb;
+  kp.c_tiles = (C + kp.lpb - 1) / kp.lpb;
+  kp.m_tiles = kp.c_tiles * ((batches + kp.bpt - 1) / kp.bpt);
+  kp.rows = 0;
+  kp.out = out;
+  kp.status = p->d_status;
+  CUtensorMap map_data;
+  const unsigned long long dims[3] = {(unsigned long long)(2 * C), (unsigned long long)J, (unsigned long long)batches};
+  const unsigned long long strides[2] = {(unsigned long long)(C * 8), (unsigned long long)(J * C * 8)};
+  const unsigned box[3] = {unsigned(2 * kp.lpb), unsigned(dft3d::kBlockK / 2), unsigned(kp.bpt)};
+  int rc = encode_f32(&map_data, in, 3, dims, strides, box, false);
+  if (rc != DFT3D_OK) return rc;
+  const long long total = kp.m_tiles * kp.n_tiles;
+  const int grid = int(total < p->sm_count ? total : p->sm_count);
+  dft3d::kdft_axis_kernel<dft3d::KDFT_STRIDED>
+      <<<grid, dft3d::kKdftThreads, dft3d::kKdftSmemBytes, stream>>>(map_data, ax.map_w, kp);
+  DFT3D_CUDA(cudaGetLastError());
+  return DFT3D_OK;
+}
+
+int launch_kdft_contig(dft3d_plan_s* p, int a, const float* in, float* out, long long rows, cudaStream_t stream) {
+  const KdftAxis& ax = p->kax[a];
+  const long long J = ax.n;
+  dft3d::KdftParams kp;
+  memset(&kp, 0, sizeof(kp));
+  kp.k2 = int(2 * J);
+  kp.bn = ax.bn;
+  kp.n_tiles = int((2 * J + ax.bn - 1) / ax.bn);
+  kp.rows = rows;
+  kp.m_tiles = (rows + dft3d::kTileM - 1) / dft3d::kTileM;
+  kp.lpb = 128;
+  kp.bpt = 1;
+  kp.c_tiles = 1;
+  kp.out = out;
+  kp.status = p->d_status;
+  CUtensorMap map_data;
+  const unsigned long long dims[2] = {(unsigned long long)(2 * J), (unsigned long long)rows};
+  const unsigned long long strides[1] = {(unsigned long long)(J * 8)};
+  const unsigned box[2] = {unsigned(dft3d::kBlockK), unsigned(dft3d::kTileM)};
+  int rc = encode_f32(&map_data, in, 2, dims, strides, box, true);
+  if (rc != DFT3D_OK) return rc;
+  const long long total = kp.m_tiles * kp.n_tiles;
+  const int grid = int(total < p->sm_count ? total : p->sm_count);
+  dft3d::kdft_axis_kernel<dft3d::KDFT_CONTIG>
+      <<<grid, dft3d::kKdftThreads, dft3d::kKdftSmemBytes, stream>>>(map_data, ax.map_w, kp);
+  DFT3D_CUDA(cudaGetLastError());
+  return DFT3D_OK;
+}
+
+int kdft_axis_pass(dft3d_plan_s* p, int axis, const float* in, float* out, long long planes, cudaStream_t stream) {
+  // `planes` n0-planes starting at in/out (axis 0 always takes the whole cube)
+  const long long n1 = p->n[1], n2 = p->n[2];
+  if (axis == 0) return launch_kdft_strided(p, 0, in, out, 1, n1 * n2, stream);
+  if (axis == 1) return launch_kdft_strided(p, 1, in, out, planes, n2, stream);
+  return launch_kdft_contig(p, 2, in, out, planes * n1, stream);
+}
+
+int check_io(const dft3d_plan_s* p, const void* in, const void* out) {
+  if (!p) return fail(DFT3D_ERR_INVALID_ARG, "plan is NULL");
+  if (!in || !out) return fail(DFT3D_ERR_INVALID_ARG, "in/out must not be NULL");
+  if ((reinterpret_cast<uintptr_t>(in) & 15) || (reinterpret_cast<uintptr_t>(out) & 15))
+    return fail(DFT3D_ERR_INVALID_ARG, "in/out must be 16-byte aligned");
+  const size_t bytes = size_t(points(p)) * 8;
+  const char* a = static_cast<const char*>(in);
+  const char* b = static_cast<const char*>(out);
+  if (a < b + bytes && b < a + bytes) return fail(DFT3D_ERR_INVALID_ARG, "in and out overlap");
+  return DFT3D_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* dft3d_status_string(int status) {
+  switch (status) {
+    case DFT3D_OK: return "ok";
+    case DFT3D_ERR_INVALID_ARG: return "invalid argument";
+    case DFT3D_ERR_UNSUPPORTED: return "unsupported size or option";
+    case DFT3D_ERR_ALLOC: return "allocation failed";
+    case DFT3D_ERR_CUDA: return "CUDA call failed";
+    case DFT3D_ERR_DEVICE_TIMEOUT: return "a kernel abandoned a bounded wait";
+    default: return "unknown status";
+  }
+}
+
+const char* dft3d_last_error(void) { return g_last_error; }
+
+int dft3d_generate_axis_matrix(long long n, int sign, double scale, const double* nodes, int nodes_on_output,
+                               double* matrix) {
+  if (n < 1 || !matrix || (sign != -1 && sign != 1)) return fail(DFT3D_ERR_INVALID_ARG, "bad argument");
+  if (nodes)
+    for (long long i = 0; i < n; ++i)
+      if (!std::isfinite(nodes[i])) return fail(DFT3D_ERR_INVALID_ARG, "node %lld is not finite", i);
+  dft3d::gen::axis_matrix(n, sign, scale, nodes, nodes_on_output != 0, matrix);
+  return DFT3D_OK;
+}
+
+int dft3d_generate_twiddle(long long N1, long long N2, int sign, double* twiddle) {
+  if (N1 < 1 || N2 < 1 || !twiddle || (sign != -1 && sign != 1)) return fail(DFT3D_ERR_INVALID_ARG, "bad argument");
+  dft3d::gen::twiddle(N1, N2, sign, twiddle);
+  return DFT3D_OK;
+}
+
+int dft3d_generate_real_table(long long n, int sign, double scale, const double* nodes, int nodes_on_output,
+                              float* hi, float* lo) {
+  if (n < 1 || !hi || !lo || (sign != -1 && sign != 1)) return fail(DFT3D_ERR_INVALID_ARG, "bad argument");
+  std::vector<double> M;
+  try {
+    M.resize(size_t(2) * n * n);
+  } catch (const std::bad_alloc&) {
+    return fail(DFT3D_ERR_ALLOC, "host allocation failed");
+  }
+  int rc = dft3d_generate_axis_matrix(n, sign, scale, nodes, nodes_on_output, M.data());
+  if (rc != DFT3D_OK) return rc;
+  dft3d::gen::real_table_from_matrix(n, M.data(), hi, lo);
+  return DFT3D_OK;
+}
+
+int dft3d_plan_create_ex(dft3d_plan_t* out, long long n0, long long n1, long long n2, int mode, int sign,
+                         const double* nodes0, const double* nodes1, const double* nodes2,
+                         const dft3d_options_t* options) {
+  if (!out) return fail(DFT3D_ERR_INVALID_ARG, "out is NULL");
+  *out = nullptr;
+  if (n0 < 1 || n1 < 1 || n2 < 1) return fail(DFT3D_ERR_INVALID_ARG, "sizes must be >= 1");
+  if (mode != DFT3D_KDFT && mode != DFT3D_FFT) return fail(DFT3D_ERR_INVALID_ARG, "mode must be DFT3D_KDFT or DFT3D_FFT");
+  if (sign != DFT3D_FORWARD && sign != DFT3D_INVERSE) return fail(DFT3D_ERR_INVALID_ARG, "sign must be -1 or +1");
+  const long long nn[3] = {n0, n1, n2};
+  const double* nodes[3] = {nodes0, nodes1, nodes2};
+  for (int a = 0; a < 3; ++a)
+    if (nodes[a])
+      for (long long i = 0; i < nn[a]; ++i)
+        if (!std::isfinite(nodes[a][i])) return fail(DFT3D_ERR_INVALID_ARG, "node %lld of axis %d is not finite", i, a);
+  dft3d_options_t opt;
+  memset(&opt, 0, sizeof(opt));
+  if (options) {
+    if (options->struct_size < sizeof(size_t) + sizeof(unsigned) || options->struct_size > sizeof(opt))
+      return fail(DFT3D_ERR_INVALID_ARG, "options->struct_size is not a known size");
+    memcpy(&opt, options, options->struct_size);
+  }
+  if (opt.flags & ~(DFT3D_NODES_ON_OUTPUT | DFT3D_UNSCALED_INVERSE)) return fail(DFT3D_ERR_INVALID_ARG, "unknown flag");
+  for (int a = 0; a < 3; ++a) {
+    if (nn[a] % 64 != 0) return fail(DFT3D_ERR_UNSUPPORTED, "n%d = %lld is not a multiple of 64", a, nn[a]);
+    if (nn[a] > 8192) return fail(DFT3D_ERR_UNSUPPORTED, "n%d = %lld exceeds 8192", a, nn[a]);
+  }
+  if (mode == DFT3D_FFT && (nodes0 || nodes1 || nodes2))
+    return fail(DFT3D_ERR_UNSUPPORTED, "the FFT formulation needs a uniform grid (no nodes)");
+
+  int ndev = 0;
+  if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev < 1) return fail(DFT3D_ERR_CUDA, "no CUDA device available");
+  dft3d_plan_s* p = new (std::nothrow) dft3d_plan_s();
+  if (!p) return fail(DFT3D_ERR_ALLOC, "host allocation of the plan failed");
+  int rc = DFT3D_OK;
+  do {
+    for (int a = 0; a < 3; ++a) p->n[a] = nn[a];
+    p->mode = mode;
+    p->sign = sign;
+    p->flags = opt.flags;
+    cudaDeviceProp prop;
+    if (cudaGetDevice(&p->device) != cudaSuccess || cudaGetDeviceProperties(&prop, p->device) != cudaSuccess) {
+      rc = fail(DFT3D_ERR_CUDA, "cannot query the current device");
+      break;
+    }
+    if (prop.major != 10) {
+      rc = fail(DFT3D_ERR_UNSUPPORTED, "device %s is sm_%d%d; this library is built for sm_100a only", prop.name,
+                prop.major, prop.minor);
+      break;
+    }
+    p->sm_count = prop.multiProcessorCount;
+    if ((rc = set_kernel_attributes()) != DFT3D_OK) break;
+    cudaError_t e = cudaMalloc(&p->d_status, sizeof(unsigned int));
+    if (e == cudaSuccess) e = cudaMemset(p->d_status, 0, sizeof(unsigned int));
+    if (e != cudaSuccess) { rc = fail(DFT3D_ERR_ALLOC, "cudaMalloc(status): %s", cudaGetErrorString(e)); break; }
+    if (mode == DFT3D_KDFT) {
+      for (int a = 0; a < 3 && rc == DFT3D_OK; ++a) rc = build_kdft_axis(p, a, nodes[a]);
+      if (rc != DFT3D_OK) break;
+      // workspace: whole cube when it fits the limit, else a group of n0-planes with at least ~8 waves of tiles
+      const size_t plane_bytes = size_t(n1) * n2 * 8;
+      size_t limit = opt.workspace_limit ? opt.workspace_limit : (size_t(16) << 30);
+      long long g = n0;
+      if (size_t(g) * plane_bytes > limit) {
+        g = (long long)(limit / plane_bytes);
+        if (g < 1) g = 1;
+        while (n0 % g) --g;   // groups of equal size
+      }
+      p->group_planes = g;
+      p->workspace_bytes = size_t(g) * plane_bytes;
+      e = cudaMalloc(&p->workspace, p->workspace_bytes);
+      if (e != cudaSuccess) { rc = fail(DFT3D_ERR_ALLOC, "cudaMalloc(workspace %zu bytes): %s", p->workspace_bytes, cudaGetErrorString(e)); break; }
+    } else {
+      for (int a = 0; a < 3 && rc == DFT3D_OK; ++a) {
+        rc = dft3d::fft_build_axis(&p->fax[a], nn[a], sign, (sign > 0) && !(opt.flags & DFT3D_UNSCALED_INVERSE),
+                                   opt.fft_split[a][0], opt.fft_split[a][1], g_last_error, sizeof(g_last_error));
+      }
+      if (rc != DFT3D_OK) break;
+    }
+  } while (0);
+  if (rc != DFT3D_OK) {
+    char keep[sizeof(g_last_error)];
+    memcpy(keep, g_last_error, sizeof(keep));
+    dft3d_plan_destroy(p);
+    memcpy(g_last_error, keep, sizeof(keep));
+    return rc;
+  }
+  *out = p;
+  return DFT3D_OK;
+}
+
+int dft3d_plan_create(dft3d_plan_t* out, long long n0, long long n1, long long n2, int mode, int sign,
+                      const double* nodes0, const double* nodes1, const double* nodes2) {
+  return dft3d_plan_create_ex(out, n0, n1, n2, mode, sign, nodes0, nodes1, nodes2, nullptr);
+}
+
+int dft3d_execute_axis(dft3d_plan_t p, int axis, const void* in, void* out, void* cuda_stream) {
+  int rc = check_io(p, in, out);
+  if (rc != DFT3D_OK) return rc;
+  if (axis < 0 || axis > 2) return fail(DFT3D_ERR_INVALID_ARG, "axis must be 0, 1 or 2");
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  if (p->mode == DFT3D_KDFT)
+    return kdft_axis_pass(p, axis, static_cast<const float*>(in), static_cast<float*>(out), p->n[0], stream);
+  rc = dft3d::fft_axis_pass(&p->fax[axis], axis, p->n, static_cast<const float*>(in), static_cast<float*>(out),
+                            p->d_status, p->sm_count, stream, g_last_error, sizeof(g_last_error));
+  return rc;
+}
+
+int dft3d_execute(dft3d_plan_t p, const void* in, void* out, void* cuda_stream) {
+  int rc = check_io(p, in, out);
+  if (rc != DFT3D_OK) return rc;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  const float* fin = static_cast<const float*>(in);
+  float* fout = static_cast<float*>(out);
+  if (p->mode == DFT3D_KDFT) {
+    // axis 0: in -> out; then per group of n0-planes: axis 1 out -> workspace, axis 2 workspace -> out
+    if ((rc = kdft_axis_pass(p, 0, fin, fout, p->n[0], stream)) != DFT3D_OK) return rc;
+    const long long g = p->group_planes;
+    const long long plane_floats = p->n[1] * p->n[2] * 2;
+    float* ws = static_cast<float*>(p->workspace);
+    for (long long a = 0; a < p->n[0]; a += g) {
+      float* slab = fout + a * plane_floats;
+      if ((rc = kdft_axis_pass(p, 1, slab, ws, g, stream)) != DFT3D_OK) return rc;
+      if ((rc = kdft_axis_pass(p, 2, ws, slab, g, stream)) != DFT3D_OK) return rc;
+    }
+    return DFT3D_OK;
+  }
+  // FFT: axis 2 in -> out, then axes 1 and 0 in place on out (a CTA reads its lines completely before it writes them)
+  if ((rc = dft3d::fft_axis_pass(&p->fax[2], 2, p->n, fin, fout, p->d_status, p->sm_count, stream, g_last_error,
+                                 sizeof(g_last_error))) != DFT3D_OK) return rc;
+  if ((rc = dft3d::fft_axis_pass(&p->fax[1], 1, p->n, fout, fout, p->d_status, p->sm_count, stream, g_last_error,
+                                 sizeof(g_last_error))) != DFT3D_OK) return rc;
+  return dft3d::fft_axis_pass(&p->fax[0], 0, p->n, fout, fout, p->d_status, p->sm_count, stream, g_last_error,
+                              sizeof(g_last_error));
+}
+
+int dft3d_execute_host(dft3d_plan_t p, const void* host_in, void* host_out, void* cuda_stream) {
+  if (!p) return fail(DFT3D_ERR_INVALID_ARG, "plan is NULL");
+  if (!host_in || !host_out) return fail(DFT3D_ERR_INVALID_ARG, "host_in/host_out must not be NULL");
+  const size_t bytes = size_t(points(p)) * 8;
+  if (!p->host_in_dev) DFT3D_CUDA(cudaMalloc(&p->host_in_dev, bytes));
+  if (!p->host_out_dev) DFT3D_CUDA(cudaMalloc(&p->host_out_dev, bytes));
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  DFT3D_CUDA(cudaMemcpyAsync(p->host_in_dev, host_in, bytes, cudaMemcpyHostToDevice, stream));
+  int rc = dft3d_execute(p, p->host_in_dev, p->host_out_dev, cuda_stream);
+  if (rc != DFT3D_OK) return rc;
+  DFT3D_CUDA(cudaMemcpyAsync(host_out, p->host_out_dev, bytes, cudaMemcpyDeviceToHost, stream));
+  DFT3D_CUDA(cudaStreamSynchronize(stream));
+  return dft3d_plan_status(p);
+}
+
+int dft3d_plan_status(dft3d_plan_t p) {
+  if (!p) return fail(DFT3D_ERR_INVALID_ARG, "plan is NULL");
+  unsigned int word = 0;
+  DFT3D_CUDA(cudaMemcpy(&word, p->d_status, sizeof(word), cudaMemcpyDeviceToHost));
+  if (word != 0) return fail(DFT3D_ERR_DEVICE_TIMEOUT, "a kernel abandoned a bounded wait (code 0x%x)", word);
+  return DFT3D_OK;
+}
+
+size_t dft3d_plan_workspace_bytes(dft3d_plan_t p) { return p ? p->workspace_bytes : 0; }
+
+int dft3d_plan_launches(dft3d_plan_t p) {
+  if (!p) return 0;
+  if (p->mode == DFT3D_KDFT) return int(1 + 2 * (p->n[0] / p->group_planes));
+  return 3;
+}
+
+int dft3d_plan_destroy(dft3d_plan_t p) {
+  if (!p) return DFT3D_OK;
+  for (int a = 0; a < 3; ++a) {
+    if (p->kax[a].d_w) cudaFree(p->kax[a].d_w);
+    dft3d::fft_free_axis(&p->fax[a]);
+  }
+  if (p->workspace) cudaFree(p->workspace);
+  if (p->d_status) cudaFree(p->d_status);
+  if (p->host_in_dev) cudaFree(p->host_in_dev);
+  if (p->host_out_dev) cudaFree(p->host_out_dev);
+  delete p;
+  return DFT3D_OK;
+}
+
+}  // extern "C"

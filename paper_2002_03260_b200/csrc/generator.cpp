@@ -1,0 +1,119 @@
+#include "generator.h"
+
+#include <cmath>
+
+namespace dft3d {
+namespace gen {
+
+namespace {
+
+constexpr double kHalfPi = 1.57079632679489661923132169163975144;
+
+// (cos, sin) of quadrant*pi/2 + frac_of_quadrant*pi/2 with 0 <= frac_of_quadrant < 1.
+// The angle handed to cos/sin never exceeds pi/4, and the quadrant is applied by exact swaps / sign flips.
+void quadrant_phasor(int quadrant, double frac_of_quadrant, double* c, double* s) {
+  double cc, ss;
+  if (frac_of_quadrant <= 0.5) {
+    const double th = frac_of_quadrant * kHalfPi;
+    cc = std::cos(th);
+    ss = std::sin(th);
+  } else {
+    const double th = (1.0 - frac_of_quadrant) * kHalfPi;
+    cc = std::sin(th);
+    ss = std::cos(th);
+  }
+  switch (quadrant & 3) {
+    case 0: *c = cc; *s = ss; break;
+    case 1: *c = -ss; *s = cc; break;
+    case 2: *c = -cc; *s = -ss; break;
+    default: *c = ss; *s = -cc; break;
+  }
+}
+
+// exp(sign*2*pi*i*a*t) for an integer-valued a and any finite t: a*t is reduced modulo 1 with the
+// rounding error of the product recovered by a fused multiply-add.
+void node_phasor(double a, double t, int sign, double* re, double* im) {
+  const double prod = a * t;
+  const double err = std::fma(a, t, -prod);
+  double f = prod - std::floor(prod);
+  f += err;
+  f -= std::floor(f);
+  const double f4 = 4.0 * f;
+  double qd = std::floor(f4);
+  if (qd >= 4.0) qd = 3.0;
+  double c, s;
+  quadrant_phasor(static_cast<int>(qd), f4 - qd, &c, &s);
+  *re = c;
+  *im = sign < 0 ? -s : s;
+}
+
+}  // namespace
+
+void root_of_unity(int64_t num, int64_t den, int sign, double* re, double* im) {
+  const __int128 four = static_cast<__int128>(4) * num;
+  const int quadrant = static_cast<int>(four / den);
+  const int64_t rem = static_cast<int64_t>(four % den);
+  double c, s;
+  if (rem == 0) {
+    quadrant_phasor(quadrant, 0.0, &c, &s);
+  } else {
+    quadrant_phasor(quadrant, static_cast<double>(rem) / static_cast<double>(den), &c, &s);
+  }
+  *re = c;
+  *im = sign < 0 ? -s : s;
+  if (*im == 0.0) *im = 0.0;  // no negative zero
+}
+
+void axis_matrix(int64_t n, int sign, double scale, const double* nodes, bool nodes_on_output, double* M) {
+  for (int64_t k = 0; k < n; ++k) {
+    for (int64_t j = 0; j < n; ++j) {
+      double re, im;
+      if (!nodes) {
+        const int64_t m = static_cast<int64_t>((static_cast<__int128>(k) * j) % n);
+        root_of_unity(m, n, sign, &re, &im);
+      } else if (!nodes_on_output) {
+        node_phasor(static_cast<double>(k), nodes[j], sign, &re, &im);
+      } else {
+        node_phasor(static_cast<double>(j), nodes[k], sign, &re, &im);
+      }
+      M[2 * (k * n + j)] = scale * re;
+      M[2 * (k * n + j) + 1] = scale * im;
+    }
+  }
+}
+
+void twiddle(int64_t N1, int64_t N2, int sign, double* T) {
+  const int64_t N = N1 * N2;
+  for (int64_t k1 = 0; k1 < N1; ++k1)
+    for (int64_t b = 0; b < N2; ++b) {
+      double re, im;
+      root_of_unity((k1 * b) % N, N, sign, &re, &im);
+      T[2 * (k1 * N2 + b)] = re;
+      T[2 * (k1 * N2 + b) + 1] = im;
+    }
+}
+
+float round_to_tf32(double v) {
+  if (v == 0.0 || !std::isfinite(v)) return static_cast<float>(v);
+  if (std::fabs(v) < 1e-30) return 0.0f;  // far below anything a DFT table holds; avoids float subnormals
+  int e;
+  const double m = std::frexp(v, &e);             // v = m * 2^e, 0.5 <= |m| < 1
+  const double r = std::nearbyint(std::ldexp(m, 11));  // 11 significant bits, ties to even
+  return static_cast<float>(std::ldexp(r, e - 11));
+}
+
+void real_table_from_matrix(int64_t n, const double* M, float* hi, float* lo) {
+  const int64_t ld = 2 * n;
+  for (int64_t k = 0; k < n; ++k)
+    for (int64_t j = 0; j < n; ++j) {
+      const double re = M[2 * (k * n + j)], im = M[2 * (k * n + j) + 1];
+      const int64_t r0 = (2 * k) * ld + 2 * j, r1 = (2 * k + 1) * ld + 2 * j;
+      split_tf32(re, &hi[r0], &lo[r0]);
+      split_tf32(-im, &hi[r0 + 1], &lo[r0 + 1]);
+      split_tf32(im, &hi[r1], &lo[r1]);
+      split_tf32(re, &hi[r1 + 1], &lo[r1 + 1]);
+    }
+}
+
+}  // namespace gen
+}  // namespace dft3d

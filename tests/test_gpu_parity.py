@@ -1,0 +1,176 @@
+"""Parity of the CUDA path (through the C-ABI) with the float64 oracle on the same seeded inputs.
+
+Tolerance: relative L2 error <= 1e-5 against the float64 oracle (the bar the task states).  The
+split-precision arithmetic should land near 1e-7..1e-6; a tighter sanity bound of 3e-6 is asserted too,
+because an error of ~2.6e-4 would mean a split product is missing and >1e-3 an indexing bug.
+"""
+import numpy as np
+import pytest
+
+torch = pytest.importorskip("torch")
+
+pytestmark = pytest.mark.gpu
+
+TOL = 1e-5
+SANITY = 3e-6
+
+
+@pytest.fixture(scope="module")
+def lib():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    import paper_2002_03260_b200 as d
+    return d
+
+
+def _inputs():
+    from paper_2002_03260_b200 import inputs
+    return inputs
+
+
+def _finish(plan):
+    torch.cuda.synchronize()
+    plan.status()
+
+
+# ------------------------------------------------------------------ single axes (each kernel variant alone)
+
+@pytest.mark.parametrize("shape", [(64, 64, 64), (64, 128, 192), (128, 64, 256), (192, 64, 64)])
+@pytest.mark.parametrize("axis", [0, 1, 2])
+def test_kdft_single_axis(lib, oracle, shape, axis):
+    x = _inputs().cube(shape, "normal", 7 + axis, device="cuda")
+    plan = lib.Plan(*shape, mode=lib.DFT3D_KDFT)
+    y = plan.execute_axis(axis, x)
+    _finish(plan)
+    ref = oracle.dft_axis(x.cpu().numpy().astype(np.complex128), axis)
+    err = oracle.rel_l2(y.cpu().numpy(), ref)
+    assert err < SANITY, (shape, axis, err)
+    plan.destroy()
+
+
+# ------------------------------------------------------------------ config 1: 64^3 KDFT forward, U(-1,1)
+
+def test_config1_kdft_64(lib, oracle):
+    shape = (64, 64, 64)
+    x = _inputs().cube(shape, "uniform", 1001, device="cuda")
+    plan = lib.Plan(*shape, mode=lib.DFT3D_KDFT, sign=lib.DFT3D_FORWARD)
+    y = plan(x)
+    _finish(plan)
+    ref = oracle.dft3d(x.cpu().numpy())
+    err = oracle.rel_l2(y.cpu().numpy(), ref)
+    assert err < TOL and err < SANITY, err
+    # the input is never written
+    assert torch.equal(x, _inputs().cube(shape, "uniform", 1001, device="cuda"))
+    plan.destroy()
+
+
+@pytest.mark.parametrize("shape", [(64, 128, 256), (256, 64, 128), (128, 192, 64)])
+def test_kdft_noncubic(lib, oracle, shape):
+    x = _inputs().cube(shape, "uniform", 31, device="cuda")
+    plan = lib.Plan(*shape)
+    y = plan(x)
+    _finish(plan)
+    err = oracle.rel_l2(y.cpu().numpy(), oracle.dft3d(x.cpu().numpy()))
+    assert err < SANITY, (shape, err)
+    plan.destroy()
+
+
+def test_kdft_workspace_groups(lib, oracle):
+    """A small workspace limit forces the plane-group schedule (several launches per axis)."""
+    shape = (64, 64, 128)
+    x = _inputs().cube(shape, "normal", 32, device="cuda")
+    plan = lib.Plan(*shape, workspace_limit=16 * 64 * 128 * 8)
+    assert plan.workspace_bytes == 16 * 64 * 128 * 8 and plan.launches == 1 + 2 * 4
+    y = plan(x)
+    _finish(plan)
+    err = oracle.rel_l2(y.cpu().numpy(), oracle.dft3d(x.cpu().numpy()))
+    assert err < SANITY, err
+    plan.destroy()
+
+
+def test_kdft_inverse_and_roundtrip(lib, oracle):
+    shape = (128, 64, 64)
+    x = _inputs().cube(shape, "normal", 33, device="cuda")
+    fwd, inv = lib.Plan(*shape, sign=lib.DFT3D_FORWARD), lib.Plan(*shape, sign=lib.DFT3D_INVERSE)
+    X = fwd(x)
+    back = inv(X)
+    _finish(inv)
+    fwd.status()
+    assert oracle.rel_l2(back.cpu().numpy(), x.cpu().numpy()) < SANITY
+    ref = oracle.dft3d(X.cpu().numpy(), sign=+1, scaled_inverse=True)
+    assert oracle.rel_l2(back.cpu().numpy(), ref) < SANITY
+    raw = lib.Plan(*shape, sign=lib.DFT3D_INVERSE, flags=lib.DFT3D_UNSCALED_INVERSE)
+    y = raw(X)
+    _finish(raw)
+    assert oracle.rel_l2(y.cpu().numpy(), oracle.dft3d(X.cpu().numpy(), sign=+1)) < SANITY
+    for p in (fwd, inv, raw):
+        p.destroy()
+
+
+# ------------------------------------------------------------------ config 4: nonuniform KDFT 256^3
+
+def test_config4_nonuniform_256(lib, oracle):
+    shape = (256, 256, 256)
+    inp = _inputs()
+    x = inp.cube(shape, "normal", 1004, device="cuda")
+    nodes = inp.sorted_nodes(shape, 2004)
+    plan = lib.Plan(*shape, nodes=nodes)
+    y = plan(x)
+    _finish(plan)
+    ref = oracle.dft3d(x.cpu().numpy(), nodes=nodes)
+    err = oracle.rel_l2(y.cpu().numpy(), ref)
+    assert err < TOL and err < SANITY, err
+    plan.destroy()
+
+
+def test_nonuniform_nodes_on_output_and_mixed(lib, oracle):
+    shape = (64, 128, 64)
+    inp = _inputs()
+    x = inp.cube(shape, "normal", 41, device="cuda")
+    nodes = inp.sorted_nodes(shape, 42)
+    plan = lib.Plan(*shape, nodes=nodes, flags=lib.DFT3D_NODES_ON_OUTPUT)
+    y = plan(x)
+    _finish(plan)
+    ref = oracle.dft3d(x.cpu().numpy(), nodes=nodes, nodes_on_output=True)
+    assert oracle.rel_l2(y.cpu().numpy(), ref) < SANITY
+    plan.destroy()
+    mixed = (None, nodes[1], None)
+    plan = lib.Plan(*shape, nodes=mixed)
+    y = plan(x)
+    _finish(plan)
+    assert oracle.rel_l2(y.cpu().numpy(), oracle.dft3d(x.cpu().numpy(), nodes=mixed)) < SANITY
+    plan.destroy()
+
+
+# ------------------------------------------------------------------ config 2: 512^3 forward + inverse
+
+@pytest.mark.slow
+def test_config2_kdft_512_forward_inverse(lib, oracle):
+    shape = (512, 512, 512)
+    x = _inputs().cube(shape, "normal", 1002, device="cuda")
+    fwd, inv = lib.Plan(*shape, sign=lib.DFT3D_FORWARD), lib.Plan(*shape, sign=lib.DFT3D_INVERSE)
+    X = fwd(x)
+    _finish(fwd)
+    xh = x.cpu().numpy()
+    ref = oracle.dft3d(xh)            # full float64 oracle: 2e11 complex MACs
+    err = oracle.rel_l2(X.cpu().numpy(), ref)
+    del ref
+    assert err < TOL and err < SANITY, err
+    back = inv(X)
+    _finish(inv)
+    assert oracle.rel_l2(back.cpu().numpy(), xh) < TOL
+    fwd.destroy()
+    inv.destroy()
+
+
+# ------------------------------------------------------------------ host-buffer entry point
+
+def test_execute_host(lib, oracle):
+    shape = (64, 64, 128)
+    x = _inputs().cube(shape, "uniform", 51, device="cpu").pin_memory()
+    out = torch.empty_like(x).pin_memory()
+    plan = lib.Plan(*shape)
+    plan.execute_host(x, out)
+    err = oracle.rel_l2(out.numpy(), oracle.dft3d(x.numpy()))
+    assert err < SANITY, err
+    plan.destroy()
