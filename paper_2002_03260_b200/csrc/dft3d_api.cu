@@ -3,6 +3,7 @@
 #include <cmath>
 #include <cstdarg>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <vector>
@@ -95,7 +96,9 @@ struct dft3d_plan_s {
   void* workspace = nullptr;
   size_t workspace_bytes = 0;
   long long group_planes = 0;   // n0-planes per workspace group (KDFT)
+  int chunk_kb = 4;             // 32-real stages per tensor-core accumulation chain (KDFT)
   unsigned int* d_status = nullptr;
+  long long* d_profile = nullptr;   // wait-cycle counters, only allocated in DFT3D_PROFILE_WAITS builds
   void* host_in_dev = nullptr;  // device staging for dft3d_execute_host
   void* host_out_dev = nullptr;
   bool attrs_set = false;
@@ -153,6 +156,7 @@ int launch_kdft_strided(dft3d_plan_s* p, int a, const float* in, float* out, lon
   kp.k2 = int(2 * J);
   kp.bn = ax.bn;
   kp.n_tiles = int((2 * J + ax.bn - 1) / ax.bn);
+  kp.chunk_kb = p->chunk_kb;
   kp.batches = batches;
   kp.C = C;
   kp.lpb = int(C < 128 ? C : 128);
@@ -162,6 +166,7 @@ int launch_kdft_strided(dft3d_plan_s* p, int a, const float* in, float* out, lon
   kp.rows = 0;
   kp.out = out;
   kp.status = p->d_status;
+  kp.profile = p->d_profile;
   CUtensorMap map_data;
   const unsigned long long dims[3] = {(unsigned long long)(2 * C), (unsigned long long)J, (unsigned long long)batches};
   const unsigned long long strides[2] = {(unsigned long long)(C * 8), (unsigned long long)(J * C * 8)};
@@ -184,6 +189,7 @@ int launch_kdft_contig(dft3d_plan_s* p, int a, const float* in, float* out, long
   kp.k2 = int(2 * J);
   kp.bn = ax.bn;
   kp.n_tiles = int((2 * J + ax.bn - 1) / ax.bn);
+  kp.chunk_kb = p->chunk_kb;
   kp.rows = rows;
   kp.m_tiles = (rows + dft3d::kTileM - 1) / dft3d::kTileM;
   kp.lpb = 128;
@@ -191,6 +197,7 @@ int launch_kdft_contig(dft3d_plan_s* p, int a, const float* in, float* out, long
   kp.c_tiles = 1;
   kp.out = out;
   kp.status = p->d_status;
+  kp.profile = p->d_profile;
   CUtensorMap map_data;
   const unsigned long long dims[2] = {(unsigned long long)(2 * J), (unsigned long long)rows};
   const unsigned long long strides[1] = {(unsigned long long)(J * 8)};
@@ -242,6 +249,13 @@ const char* dft3d_status_string(int status) {
 }
 
 const char* dft3d_last_error(void) { return g_last_error; }
+
+#ifdef DFT3D_PROFILE_WAITS
+// diagnostic builds only: copies the MMA issuer's cycle counters [grid][4] = {total, wait acc, wait W, wait data}
+int dft3d_debug_read_profile(dft3d_plan_t p, long long* host, int ctas) {
+  return cudaMemcpy(host, p->d_profile, sizeof(long long) * 4 * ctas, cudaMemcpyDeviceToHost) == cudaSuccess ? 0 : 4;
+}
+#endif
 
 int dft3d_generate_axis_matrix(long long n, int sign, double scale, const double* nodes, int nodes_on_output,
                                double* matrix) {
@@ -324,10 +338,18 @@ int dft3d_plan_create_ex(dft3d_plan_t* out, long long n0, long long n1, long lon
       break;
     }
     p->sm_count = prop.multiProcessorCount;
+    if (const char* env = getenv("DFT3D_CHUNK_KB")) {   // tuning knob: stages per accumulation chain
+      const int v = atoi(env);
+      if (v >= 1) p->chunk_kb = v;
+    }
     if ((rc = set_kernel_attributes()) != DFT3D_OK) break;
     cudaError_t e = cudaMalloc(&p->d_status, sizeof(unsigned int));
     if (e == cudaSuccess) e = cudaMemset(p->d_status, 0, sizeof(unsigned int));
     if (e != cudaSuccess) { rc = fail(DFT3D_ERR_ALLOC, "cudaMalloc(status): %s", cudaGetErrorString(e)); break; }
+#ifdef DFT3D_PROFILE_WAITS
+    e = cudaMalloc(&p->d_profile, sizeof(long long) * 4 * 1024);
+    if (e != cudaSuccess) { rc = fail(DFT3D_ERR_ALLOC, "cudaMalloc(profile)"); break; }
+#endif
     if (mode == DFT3D_KDFT) {
       for (int a = 0; a < 3 && rc == DFT3D_OK; ++a) rc = build_kdft_axis(p, a, nodes[a]);
       if (rc != DFT3D_OK) break;
@@ -447,6 +469,7 @@ int dft3d_plan_destroy(dft3d_plan_t p) {
   }
   if (p->workspace) cudaFree(p->workspace);
   if (p->d_status) cudaFree(p->d_status);
+  if (p->d_profile) cudaFree(p->d_profile);
   if (p->host_in_dev) cudaFree(p->host_in_dev);
   if (p->host_out_dev) cudaFree(p->host_out_dev);
   delete p;

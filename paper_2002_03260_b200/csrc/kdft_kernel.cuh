@@ -22,16 +22,23 @@
 //
 // Pipeline per CTA (persistent over tiles, one CTA per SM):
 //   warp 0      TMA producer: W tile (both pieces, K-major, 128B swizzle) and the raw data tile
-//   warps 2-5   split: shared memory -> registers -> (x_hi, x_lo) -> tensor memory (A operand)
+//   warps 4-7   split: shared memory -> registers -> (x_hi, x_lo) -> tensor memory (A operand)
 //   warp 1      one thread issues tcgen05.mma kind::tf32, A from tensor memory, B from shared memory,
 //               fp32 accumulator 128 x 256 in tensor memory
-//   warps 6-9   epilogue: tcgen05.ld -> global stores
+//   warps 8-15  epilogue: tcgen05.ld every chunk -> fp32 running sum in registers -> global stores
 // All waits are bounded; a wait that gives up sets the status word and the CTA unwinds.
 #pragma once
 #include <cstdint>
 #include <cuda.h>
 #include <cuda_runtime.h>
 #include "ptx_sm100.cuh"
+
+// registers per thread of each warp group after the split of the register file (sum x 128 = 65536)
+#ifndef DFT3D_REGS_WG0
+#define DFT3D_REGS_WG0 40
+#define DFT3D_REGS_SPLIT 120
+#define DFT3D_REGS_EPI 176
+#endif
 
 namespace dft3d {
 
@@ -47,13 +54,15 @@ constexpr int kAccCols = 256;       // accumulator columns in tensor memory
 constexpr int kTmemCols = 512;
 constexpr int kBytesStageB = 2 * kMaxTileN * kBlockK * 4;   // hi + lo
 constexpr int kBytesStageA = kTileM * kBlockK * 4;
-constexpr int kKdftThreads = 320;
+constexpr int kKdftThreads = 512;      // 4 warp groups: {producer, MMA, 2 idle}, split, epilogue x 2
+constexpr int kEpilogueWarps = 8;
 constexpr size_t kKdftSmemBytes = size_t(kStagesB) * kBytesStageB + size_t(kStagesA) * kBytesStageA + 1024 + 512;
 
 struct KdftParams {
   int k2;              // 2*N: real contraction length = real output length per line
   int bn;              // output reals per tile: min(256, 2N)
   int n_tiles;         // ceil(2N / bn)
+  int chunk_kb;        // pipeline stages (of 32 reals) per tensor-core accumulation chain
   long long m_tiles;   // tiles along the lines
   // CONTIG
   long long rows;      // number of lines
@@ -65,6 +74,7 @@ struct KdftParams {
   long long c_tiles;   // ceil(C / lpb)
   float* out;
   unsigned int* status;  // device word, set non-zero when a wait gives up
+  long long* profile;    // optional [grid][4] cycle counters of the MMA issuer (builds with DFT3D_PROFILE_WAITS)
 };
 
 struct KdftShared {
@@ -133,7 +143,7 @@ kdft_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_cons
     for (int i = 0; i < kStagesA; ++i) { ptx::mbar_init(&sh.a_full[i], 1); ptx::mbar_init(&sh.a_empty[i], 4); }
     for (int i = 0; i < kStagesT; ++i) { ptx::mbar_init(&sh.t_full[i], 4); ptx::mbar_init(&sh.t_empty[i], 1); }
     ptx::mbar_init(&sh.acc_full, 1);
-    ptx::mbar_init(&sh.acc_empty, 4);
+    ptx::mbar_init(&sh.acc_empty, kEpilogueWarps);
     sh.abort_flag = 0;
     ptx::fence_mbar_init();
   }
@@ -154,79 +164,113 @@ kdft_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_cons
   const int num_kb = p.k2 / kBlockK;
   const uint32_t bytes_b = 2u * uint32_t(p.bn) * kBlockK * 4u;
 
-  if (warp == 0) {
-    // ------------------------------------------------------------ TMA producer
-    if (lane == 0) {
-      uint32_t ib = 0, ia = 0;   // running stage counters
-      for (long long t = blockIdx.x; t < total_tiles; t += gridDim.x) {
-        const long long mt = t / p.n_tiles;
-        const int nt = int(t % p.n_tiles);
-        int ax = 0, ay = 0, az = 0;
-        if (MODE == KDFT_CONTIG) {
-          ay = int(mt * kTileM);
-        } else {
-          const long long ct = mt % p.c_tiles;
-          const long long bt = mt / p.c_tiles;
-          ax = int(ct * p.lpb * 2);
-          az = int(bt * p.bpt);
-        }
-        for (int kb = 0; kb < num_kb; ++kb) {
-          {
-            const uint32_t s = ib % kStagesB, ph = (ib / kStagesB) & 1;
-            DFT3D_WAIT(&sh.b_empty[s], ph ^ 1, 0x101);
-            ptx::mbar_arrive_expect_tx(&sh.b_full[s], bytes_b);
-            ptx::tma_load_3d(smem_b + size_t(s) * kBytesStageB, &map_w, &sh.b_full[s], kb * kBlockK, nt * p.bn, 0);
-            ++ib;
+  if (warp < 4) {
+    // warp group 0: producer and MMA issuer need few registers; hand the rest to the epilogue
+    ptx::setmaxnreg_dec<DFT3D_REGS_WG0>();
+    if (warp == 0) {
+      // ------------------------------------------------------------ TMA producer
+      if (lane == 0) {
+        uint32_t ib = 0, ia = 0;   // running stage counters
+        for (long long t = blockIdx.x; t < total_tiles; t += gridDim.x) {
+          const long long mt = t / p.n_tiles;
+          const int nt = int(t % p.n_tiles);
+          int ax = 0, ay = 0, az = 0;
+          if (MODE == KDFT_CONTIG) {
+            ay = int(mt * kTileM);
+          } else {
+            const long long ct = mt % p.c_tiles;
+            const long long bt = mt / p.c_tiles;
+            ax = int(ct * p.lpb * 2);
+            az = int(bt * p.bpt);
           }
-          {
-            const uint32_t s = ia % kStagesA, ph = (ia / kStagesA) & 1;
-            DFT3D_WAIT(&sh.a_empty[s], ph ^ 1, 0x102);
-            ptx::mbar_arrive_expect_tx(&sh.a_full[s], kBytesStageA);
-            if (MODE == KDFT_CONTIG)
-              ptx::tma_load_2d(smem_a + size_t(s) * kBytesStageA, &map_data, &sh.a_full[s], kb * kBlockK, ay);
-            else
-              ptx::tma_load_3d(smem_a + size_t(s) * kBytesStageA, &map_data, &sh.a_full[s], ax, kb * (kBlockK / 2), az);
-            ++ia;
+          for (int kb = 0; kb < num_kb; ++kb) {
+            {
+              const uint32_t s = ib % kStagesB, ph = (ib / kStagesB) & 1;
+              DFT3D_WAIT(&sh.b_empty[s], ph ^ 1, 0x101);
+              ptx::mbar_arrive_expect_tx(&sh.b_full[s], bytes_b);
+              ptx::tma_load_3d(smem_b + size_t(s) * kBytesStageB, &map_w, &sh.b_full[s], kb * kBlockK, nt * p.bn, 0);
+              ++ib;
+            }
+            {
+              const uint32_t s = ia % kStagesA, ph = (ia / kStagesA) & 1;
+              DFT3D_WAIT(&sh.a_empty[s], ph ^ 1, 0x102);
+              ptx::mbar_arrive_expect_tx(&sh.a_full[s], kBytesStageA);
+              if (MODE == KDFT_CONTIG)
+                ptx::tma_load_2d(smem_a + size_t(s) * kBytesStageA, &map_data, &sh.a_full[s], kb * kBlockK, ay);
+              else
+                ptx::tma_load_3d(smem_a + size_t(s) * kBytesStageA, &map_data, &sh.a_full[s], ax, kb * (kBlockK / 2), az);
+              ++ia;
+            }
           }
         }
       }
-    }
-  } else if (warp == 1) {
-    // ------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
-      const uint32_t idesc = ptx::make_idesc_tf32(kTileM, p.bn);
-      uint32_t ib = 0, it = 0, tile_count = 0;
-      for (long long t = blockIdx.x; t < total_tiles; t += gridDim.x, ++tile_count) {
-        DFT3D_WAIT(&sh.acc_empty, (tile_count & 1) ^ 1, 0x201);
-        ptx::tc_fence_after();
-        for (int kb = 0; kb < num_kb; ++kb) {
-          const uint32_t sb = ib % kStagesB, phb = (ib / kStagesB) & 1;
-          const uint32_t st = it % kStagesT, pht = (it / kStagesT) & 1;
-          DFT3D_WAIT(&sh.b_full[sb], phb, 0x202);
-          DFT3D_WAIT(&sh.t_full[st], pht, 0x203);
-          ptx::tc_fence_after();
-          const uint32_t b_hi = ptx::smem_u32(smem_b + size_t(sb) * kBytesStageB);
-          const uint32_t b_lo = b_hi + uint32_t(p.bn) * kBlockK * 4u;
-          const uint32_t a_hi = tmem + kAccCols + st * 64;
-          const uint32_t a_lo = a_hi + 32;
+    } else if (warp == 1) {
+      // ------------------------------------------------------------ MMA issuer
+      if (lane == 0) {
+        const uint32_t idesc = ptx::make_idesc_tf32(kTileM, p.bn);
+        uint32_t ib = 0, it = 0, chunk_count = 0;
+#ifdef DFT3D_PROFILE_WAITS
+        long long w_acc = 0, w_b = 0, w_t = 0, t_begin = clock64(), tq;
+#define PW_BEGIN tq = clock64();
+#define PW_END(v) v += clock64() - tq;
+#else
+#define PW_BEGIN
+#define PW_END(v)
+#endif
+        for (long long t = blockIdx.x; t < total_tiles; t += gridDim.x) {
+          for (int kb = 0; kb < num_kb; ++kb) {
+            const bool chunk_first = (kb % p.chunk_kb) == 0;
+            if (chunk_first) {
+              // the tensor-core accumulator restarts from zero every chunk (see the epilogue)
+              PW_BEGIN
+              DFT3D_WAIT(&sh.acc_empty, (chunk_count & 1) ^ 1, 0x201);
+              PW_END(w_acc)
+              ptx::tc_fence_after();
+            }
+            const uint32_t sb = ib % kStagesB, phb = (ib / kStagesB) & 1;
+            const uint32_t st = it % kStagesT, pht = (it / kStagesT) & 1;
+            PW_BEGIN
+            DFT3D_WAIT(&sh.b_full[sb], phb, 0x202);
+            PW_END(w_b)
+            PW_BEGIN
+            DFT3D_WAIT(&sh.t_full[st], pht, 0x203);
+            PW_END(w_t)
+            ptx::tc_fence_after();
+            const uint32_t b_hi = ptx::smem_u32(smem_b + size_t(sb) * kBytesStageB);
+            const uint32_t b_lo = b_hi + uint32_t(p.bn) * kBlockK * 4u;
+            const uint32_t a_hi = tmem + kAccCols + st * 64;
+            const uint32_t a_lo = a_hi + 32;
 #pragma unroll
-          for (int k = 0; k < kBlockK / 8; ++k) {
-            const uint64_t dhi = ptx::make_kmajor_sw128_desc(b_hi + k * 32);
-            const uint64_t dlo = ptx::make_kmajor_sw128_desc(b_lo + k * 32);
-            ptx::mma_tf32_ts(tmem, a_hi + k * 8, dhi, idesc, (kb | k) != 0);
-            ptx::mma_tf32_ts(tmem, a_lo + k * 8, dhi, idesc, 1);
-            ptx::mma_tf32_ts(tmem, a_hi + k * 8, dlo, idesc, 1);
+            for (int k = 0; k < kBlockK / 8; ++k) {
+              const uint64_t dhi = ptx::make_kmajor_sw128_desc(b_hi + k * 32);
+              const uint64_t dlo = ptx::make_kmajor_sw128_desc(b_lo + k * 32);
+              ptx::mma_tf32_ts(tmem, a_hi + k * 8, dhi, idesc, (k != 0 || !chunk_first) ? 1u : 0u);
+              ptx::mma_tf32_ts(tmem, a_lo + k * 8, dhi, idesc, 1);
+              ptx::mma_tf32_ts(tmem, a_hi + k * 8, dlo, idesc, 1);
+            }
+            ptx::tc_commit(&sh.b_empty[sb]);
+            ptx::tc_commit(&sh.t_empty[st]);
+            ++ib;
+            ++it;
+            if ((kb + 1) % p.chunk_kb == 0 || kb + 1 == num_kb) {
+              ptx::tc_commit(&sh.acc_full);
+              ++chunk_count;
+            }
           }
-          ptx::tc_commit(&sh.b_empty[sb]);
-          ptx::tc_commit(&sh.t_empty[st]);
-          ++ib;
-          ++it;
         }
-        ptx::tc_commit(&sh.acc_full);
+#ifdef DFT3D_PROFILE_WAITS
+        if (p.profile) {
+          p.profile[blockIdx.x * 4 + 0] = clock64() - t_begin;
+          p.profile[blockIdx.x * 4 + 1] = w_acc;
+          p.profile[blockIdx.x * 4 + 2] = w_b;
+          p.profile[blockIdx.x * 4 + 3] = w_t;
+        }
+#endif
       }
     }
-  } else if (warp < 6) {
+  } else if (warp < 8) {
     // ------------------------------------------------------------ split: smem -> (hi, lo) -> tensor memory
+    ptx::setmaxnreg_dec<DFT3D_REGS_SPLIT>();
     const int q = warp & 3;                 // lane quarter this warp may touch in tensor memory
     const int m = q * 32 + lane;            // lane of the tile
     const uint32_t lane_addr = tmem + (uint32_t(q * 32) << 16);
@@ -255,6 +299,8 @@ kdft_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_cons
             x[2 * j] = v.x; x[2 * j + 1] = v.y;
           }
         }
+        // the stage is refilled by TMA (async proxy): order this thread's reads before that write
+        ptx::fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0) ptx::mbar_arrive(&sh.a_empty[sa]);
         uint32_t lo[32];
@@ -278,56 +324,64 @@ kdft_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_cons
       }
     }
   } else {
-    // ------------------------------------------------------------ epilogue
+    // ------------------------------------------------------------ epilogue (8 warps)
+    // The tensor core adds into its fp32 accumulator with truncation, a bias that grows with the
+    // number of MMAs chained on one accumulator.  So the chain is cut every `chunk_kb` stages: the
+    // partial sum is pulled into registers and summed there in round-to-nearest fp32, and the tensor
+    // core restarts from zero.
+    ptx::setmaxnreg_inc<DFT3D_REGS_EPI>();
     const int q = warp & 3;
+    const int half = (warp - 8) >> 2;        // which 128 columns of the 256-wide accumulator
     const int m = q * 32 + lane;
-    const uint32_t lane_addr = tmem + (uint32_t(q * 32) << 16);
-    uint32_t tile_count = 0;
-    for (long long t = blockIdx.x; t < total_tiles; t += gridDim.x, ++tile_count) {
+    const uint32_t lane_addr = tmem + (uint32_t(q * 32) << 16) + half * 128;
+    const bool cols_active = half * 128 < p.bn;
+    const int chunks_per_tile = (num_kb + p.chunk_kb - 1) / p.chunk_kb;
+    uint32_t chunk_count = 0;
+    for (long long t = blockIdx.x; t < total_tiles; t += gridDim.x) {
       const long long mt = t / p.n_tiles;
       const int nt = int(t % p.n_tiles);
-      const int col0 = nt * p.bn;
-      // where this lane's line goes
-      bool lane_ok;
-      float* line_ptr;        // CONTIG: start of the output row; STRIDED: &out[batch][0][c]
-      long long k_stride = 0; // STRIDED: floats between consecutive k
-      if (MODE == KDFT_CONTIG) {
-        const long long row = mt * kTileM + m;
-        lane_ok = row < p.rows;
-        line_ptr = p.out + row * (long long)p.k2;
-      } else {
-        const long long ct = mt % p.c_tiles;
-        const long long bt = mt / p.c_tiles;
-        const long long batch = bt * p.bpt + m / p.lpb;
-        const long long c = ct * p.lpb + (m % p.lpb);
-        lane_ok = (batch < p.batches) && (c < p.C);
-        const long long J = p.k2 / 2;
-        line_ptr = p.out + 2 * ((batch * J) * p.C + c);
-        k_stride = 2 * p.C;
-      }
-      DFT3D_WAIT_WARP(&sh.acc_full, tile_count & 1, 0x401);
-      ptx::tc_fence_after();
-      const int chunks = p.bn / 32;
-      for (int ch = 0; ch < chunks; ++ch) {
-        uint32_t v[32];
-        ptx::tmem_ld_32x32(lane_addr + ch * 32, v);
-        ptx::tc_wait_ld();
-        if (ch == chunks - 1) {
-          ptx::tc_fence_before();
-          __syncwarp();
-          if (lane == 0) ptx::mbar_arrive(&sh.acc_empty);
+      float acc[128];
+#pragma unroll
+      for (int i = 0; i < 128; ++i) acc[i] = 0.0f;
+      for (int c = 0; c < chunks_per_tile; ++c, ++chunk_count) {
+        DFT3D_WAIT_WARP(&sh.acc_full, chunk_count & 1, 0x401);
+        ptx::tc_fence_after();
+        if (cols_active) {
+#pragma unroll
+          for (int g = 0; g < 4; ++g) {
+            uint32_t v[32];
+            ptx::tmem_ld_32x32(lane_addr + g * 32, v);
+            ptx::tc_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) acc[g * 32 + i] += __uint_as_float(v[i]);
+          }
         }
-        const int c0 = col0 + ch * 32;
-        if (lane_ok && c0 < p.k2) {
-          if (MODE == KDFT_CONTIG) {
-            uint4* dst = reinterpret_cast<uint4*>(line_ptr + c0);
+        ptx::tc_fence_before();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(&sh.acc_empty);
+      }
+      // ---- store this lane's 128 reals
+      const int c0 = nt * p.bn + half * 128;   // first real output column held by this thread
+      if (cols_active && c0 < p.k2) {
+        if (MODE == KDFT_CONTIG) {
+          const long long row = mt * kTileM + m;
+          if (row < p.rows) {
+            float4* dst = reinterpret_cast<float4*>(p.out + row * (long long)p.k2 + c0);
 #pragma unroll
-            for (int i = 0; i < 8; ++i) dst[i] = make_uint4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
-          } else {
-            float* dst = line_ptr + (long long)(c0 / 2) * k_stride;
+            for (int i = 0; i < 32; ++i) dst[i] = make_float4(acc[4 * i], acc[4 * i + 1], acc[4 * i + 2], acc[4 * i + 3]);
+          }
+        } else {
+          const long long ct = mt % p.c_tiles;
+          const long long bt = mt / p.c_tiles;
+          const long long batch = bt * p.bpt + m / p.lpb;
+          const long long cc = ct * p.lpb + (m % p.lpb);
+          if (batch < p.batches && cc < p.C) {
+            const long long J = p.k2 / 2;
+            const long long k_stride = 2 * p.C;
+            float* dst = p.out + 2 * ((batch * J + c0 / 2) * p.C + cc);
 #pragma unroll
-            for (int i = 0; i < 16; ++i)
-              *reinterpret_cast<uint2*>(dst + i * k_stride) = make_uint2(v[2 * i], v[2 * i + 1]);
+            for (int i = 0; i < 64; ++i)
+              *reinterpret_cast<float2*>(dst + i * k_stride) = make_float2(acc[2 * i], acc[2 * i + 1]);
           }
         }
       }

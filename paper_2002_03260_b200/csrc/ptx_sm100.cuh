@@ -28,6 +28,20 @@ __device__ __forceinline__ bool elect_one() {
   return pred != 0;
 }
 
+// register reallocation between warp groups (all four warps of the group execute it)
+template <int N>
+__device__ __forceinline__ void setmaxnreg_inc() {
+#ifndef DFT3D_NO_SETMAXNREG
+  asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N));
+#endif
+}
+template <int N>
+__device__ __forceinline__ void setmaxnreg_dec() {
+#ifndef DFT3D_NO_SETMAXNREG
+  asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N));
+#endif
+}
+
 // ---------------------------------------------------------------- mbarrier
 
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {

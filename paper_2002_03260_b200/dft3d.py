@@ -10,7 +10,8 @@ import os
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-_LIB_PATH = os.path.join(_HERE, "libdft3d.so")
+# DFT3D_LIBRARY overrides the path of the shared library (for trying differently built variants)
+_LIB_PATH = os.environ.get("DFT3D_LIBRARY") or os.path.join(_HERE, "libdft3d.so")
 
 DFT3D_KDFT, DFT3D_FFT = 0, 1
 DFT3D_FORWARD, DFT3D_INVERSE = -1, +1

@@ -1,8 +1,10 @@
 """Parity of the CUDA path (through the C-ABI) with the float64 oracle on the same seeded inputs.
 
 Tolerance: relative L2 error <= 1e-5 against the float64 oracle (the bar the task states).  The
-split-precision arithmetic should land near 1e-7..1e-6; a tighter sanity bound of 3e-6 is asserted too,
-because an error of ~2.6e-4 would mean a split product is missing and >1e-3 an indexing bug.
+3xTF32 arithmetic with accumulation chains of 48 MMAs lands near 1e-6 per axis (the tensor core adds
+into its fp32 accumulator with truncation, a bias that adds up over the axes), so tighter sanity
+bounds are asserted as well: 2e-6 for one axis, 5e-6 for a 3D transform.  An error of ~2.6e-4 would
+mean a split product is missing, >1e-3 an indexing bug.
 """
 import numpy as np
 import pytest
@@ -12,7 +14,8 @@ torch = pytest.importorskip("torch")
 pytestmark = pytest.mark.gpu
 
 TOL = 1e-5
-SANITY = 3e-6
+SANITY = 5e-6       # one 3D transform (three axis passes)
+SANITY_AXIS = 2e-6  # one axis pass
 
 
 @pytest.fixture(scope="module")
@@ -44,7 +47,7 @@ def test_kdft_single_axis(lib, oracle, shape, axis):
     _finish(plan)
     ref = oracle.dft_axis(x.cpu().numpy().astype(np.complex128), axis)
     err = oracle.rel_l2(y.cpu().numpy(), ref)
-    assert err < SANITY, (shape, axis, err)
+    assert err < SANITY_AXIS, (shape, axis, err)
     plan.destroy()
 
 
@@ -96,7 +99,7 @@ def test_kdft_inverse_and_roundtrip(lib, oracle):
     back = inv(X)
     _finish(inv)
     fwd.status()
-    assert oracle.rel_l2(back.cpu().numpy(), x.cpu().numpy()) < SANITY
+    assert oracle.rel_l2(back.cpu().numpy(), x.cpu().numpy()) < TOL   # two transforms in a row
     ref = oracle.dft3d(X.cpu().numpy(), sign=+1, scaled_inverse=True)
     assert oracle.rel_l2(back.cpu().numpy(), ref) < SANITY
     raw = lib.Plan(*shape, sign=lib.DFT3D_INVERSE, flags=lib.DFT3D_UNSCALED_INVERSE)
