@@ -83,6 +83,14 @@ struct KdftAxis {
   int bn = 0;
 };
 
+struct FftAxis {
+  long long n = 0;
+  int R = 0;               // n = R*R
+  float* d_w = nullptr;    // stacked [W_hi; W_lo] of F_R as 2R/32 panels of [4R rows][32 floats]
+  float2* d_tw = nullptr;  // T[k1][beta], R*R complex64
+  CUtensorMap map_w;
+};
+
 }  // namespace
 
 struct dft3d_plan_s {
@@ -92,7 +100,7 @@ struct dft3d_plan_s {
   int device = 0;
   int sm_count = 0;
   KdftAxis kax[3];
-  dft3d::FftAxis fax[3];
+  FftAxis fax[3];
   void* workspace = nullptr;
   size_t workspace_bytes = 0;
   long long group_planes = 0;   // n0-planes per workspace group (KDFT)
@@ -115,8 +123,14 @@ int set_kernel_attributes() {
                                   cudaFuncAttributeMaxDynamicSharedMemorySize, int(dft3d::kKdftSmemBytes)));
   DFT3D_CUDA(cudaFuncSetAttribute(dft3d::kdft_axis_kernel<dft3d::KDFT_STRIDED>,
                                   cudaFuncAttributeMaxDynamicSharedMemorySize, int(dft3d::kKdftSmemBytes)));
-  int rc = dft3d::fft_set_kernel_attributes();
-  if (rc != 0) return fail(DFT3D_ERR_CUDA, "cudaFuncSetAttribute failed for the FFT kernels");
+  DFT3D_CUDA(cudaFuncSetAttribute(dft3d::fft_axis_kernel<dft3d::FFT_CONTIG, 32>,
+                                  cudaFuncAttributeMaxDynamicSharedMemorySize, int(dft3d::fft_smem_bytes(32))));
+  DFT3D_CUDA(cudaFuncSetAttribute(dft3d::fft_axis_kernel<dft3d::FFT_STRIDED, 32>,
+                                  cudaFuncAttributeMaxDynamicSharedMemorySize, int(dft3d::fft_smem_bytes(32))));
+  DFT3D_CUDA(cudaFuncSetAttribute(dft3d::fft_axis_kernel<dft3d::FFT_CONTIG, 16>,
+                                  cudaFuncAttributeMaxDynamicSharedMemorySize, int(dft3d::fft_smem_bytes(16))));
+  DFT3D_CUDA(cudaFuncSetAttribute(dft3d::fft_axis_kernel<dft3d::FFT_STRIDED, 16>,
+                                  cudaFuncAttributeMaxDynamicSharedMemorySize, int(dft3d::fft_smem_bytes(16))));
   done = true;
   return DFT3D_OK;
 }
@@ -218,6 +232,95 @@ int kdft_axis_pass(dft3d_plan_s* p, int axis, const float* in, float* out, long 
   if (axis == 0) return launch_kdft_strided(p, 0, in, out, 1, n1 * n2, stream);
   if (axis == 1) return launch_kdft_strided(p, 1, in, out, planes, n2, stream);
   return launch_kdft_contig(p, 2, in, out, planes * n1, stream);
+}
+
+// FFT formulation, one axis: n = R*R with R = 16 or 32 (Eq. 17 with P = R).  Tables: the real form of F_R
+// split in TF32 pieces and stacked [hi; lo], in the panel layout the kernel's TMA loads expect, and the
+// twiddle factors rounded once to complex64.  The 1/n of a scaled inverse is 1/R in each stage's matrix.
+int build_fft_axis(dft3d_plan_s* p, int a, const int split[2]) {
+  FftAxis& ax = p->fax[a];
+  const long long n = p->n[a];
+  int R = 0;
+  if (n == 256) R = 16;
+  if (n == 1024) R = 32;
+  if (!R) return fail(DFT3D_ERR_UNSUPPORTED, "FFT mode supports axis lengths 256 (16*16) and 1024 (32*32); n%d = %lld", a, n);
+  if ((split[0] || split[1]) && (split[0] != R || split[1] != R))
+    return fail(DFT3D_ERR_UNSUPPORTED, "FFT split %dx%d for n%d = %lld is not supported (only %dx%d)", split[0], split[1], a, n, R, R);
+  ax.n = n;
+  ax.R = R;
+  const bool scaled = (p->sign > 0) && !(p->flags & DFT3D_UNSCALED_INVERSE);
+  const int K = 2 * R, NB = 4 * R, panels = K / 32;
+  std::vector<double> M(size_t(2) * R * R), T(size_t(2) * R * R);
+  std::vector<float> hi(size_t(K) * K), lo(size_t(K) * K), W(size_t(panels) * NB * 32), tw(size_t(2) * R * R);
+  dft3d::gen::axis_matrix(R, p->sign, scaled ? 1.0 / R : 1.0, nullptr, false, M.data());
+  dft3d::gen::real_table_from_matrix(R, M.data(), hi.data(), lo.data());
+  for (int pn = 0; pn < panels; ++pn)
+    for (int r = 0; r < NB; ++r)
+      for (int c = 0; c < 32; ++c) {
+        const std::vector<float>& piece = (r < K) ? hi : lo;
+        W[(size_t(pn) * NB + r) * 32 + c] = piece[size_t(r % K) * K + pn * 32 + c];
+      }
+  dft3d::gen::twiddle(R, R, p->sign, T.data());
+  for (size_t i = 0; i < T.size(); ++i) tw[i] = float(T[i]);
+  DFT3D_CUDA(cudaMalloc(&ax.d_w, W.size() * sizeof(float)));
+  DFT3D_CUDA(cudaMemcpy(ax.d_w, W.data(), W.size() * sizeof(float), cudaMemcpyHostToDevice));
+  DFT3D_CUDA(cudaMalloc(&ax.d_tw, tw.size() * sizeof(float)));
+  DFT3D_CUDA(cudaMemcpy(ax.d_tw, tw.data(), tw.size() * sizeof(float), cudaMemcpyHostToDevice));
+  const unsigned long long dims[2] = {32ull, (unsigned long long)(panels * NB)};
+  const unsigned long long strides[1] = {128ull};
+  const unsigned box[2] = {32u, unsigned(NB)};
+  return encode_f32(&ax.map_w, ax.d_w, 2, dims, strides, box, true);
+}
+
+int fft_axis_pass(dft3d_plan_s* p, int axis, const float* in, float* out, cudaStream_t stream) {
+  const FftAxis& ax = p->fax[axis];
+  const int R = ax.R, N = int(ax.n), Lg = 128 / R;
+  dft3d::FftParams fp;
+  memset(&fp, 0, sizeof(fp));
+  fp.N = N;
+  fp.twiddle = ax.d_tw;
+  fp.out = out;
+  fp.status = p->d_status;
+  CUtensorMap map_data;
+  int rc;
+  if (axis == 2) {
+    const long long rows = p->n[0] * p->n[1];
+    fp.rows = rows;
+    fp.mtiles_per_stage = 1;
+    fp.stage_bytes = Lg * N * 8;
+    fp.num_stages = rows / Lg;
+    const unsigned long long dims[3] = {256ull, (unsigned long long)(N / 128), (unsigned long long)rows};
+    const unsigned long long strides[2] = {1024ull, (unsigned long long)N * 8ull};
+    const unsigned box[3] = {256u, unsigned(N / 128), unsigned(Lg)};
+    rc = encode_f32(&map_data, in, 3, dims, strides, box, false);
+  } else {
+    const long long batches = (axis == 0) ? 1 : p->n[0];
+    const long long C = (axis == 0) ? p->n[1] * p->n[2] : p->n[2];
+    fp.C = C;
+    fp.c_tiles = C / dft3d::kFftStridedCols;
+    fp.mtiles_per_stage = dft3d::kFftStridedCols / Lg;
+    fp.stage_bytes = N * 128;
+    fp.num_stages = batches * fp.c_tiles;
+    const unsigned long long dims[3] = {(unsigned long long)(2 * C), (unsigned long long)N, (unsigned long long)batches};
+    const unsigned long long strides[2] = {(unsigned long long)(C * 8), (unsigned long long)N * C * 8ull};
+    const unsigned box[3] = {32u, 256u, 1u};
+    rc = encode_f32(&map_data, in, 3, dims, strides, box, true);
+  }
+  if (rc != DFT3D_OK) return rc;
+  fp.raw_stages = dft3d::kFftRawBytes / fp.stage_bytes;
+  if (fp.raw_stages > 4) fp.raw_stages = 4;
+  const int grid = int(fp.num_stages < p->sm_count ? fp.num_stages : p->sm_count);
+  const size_t smem = dft3d::fft_smem_bytes(R);
+  if (axis == 2 && R == 32)
+    dft3d::fft_axis_kernel<dft3d::FFT_CONTIG, 32><<<grid, dft3d::kFftThreads, smem, stream>>>(map_data, ax.map_w, fp);
+  else if (axis == 2)
+    dft3d::fft_axis_kernel<dft3d::FFT_CONTIG, 16><<<grid, dft3d::kFftThreads, smem, stream>>>(map_data, ax.map_w, fp);
+  else if (R == 32)
+    dft3d::fft_axis_kernel<dft3d::FFT_STRIDED, 32><<<grid, dft3d::kFftThreads, smem, stream>>>(map_data, ax.map_w, fp);
+  else
+    dft3d::fft_axis_kernel<dft3d::FFT_STRIDED, 16><<<grid, dft3d::kFftThreads, smem, stream>>>(map_data, ax.map_w, fp);
+  DFT3D_CUDA(cudaGetLastError());
+  return DFT3D_OK;
 }
 
 int check_io(const dft3d_plan_s* p, const void* in, const void* out) {
@@ -367,10 +470,7 @@ int dft3d_plan_create_ex(dft3d_plan_t* out, long long n0, long long n1, long lon
       e = cudaMalloc(&p->workspace, p->workspace_bytes);
       if (e != cudaSuccess) { rc = fail(DFT3D_ERR_ALLOC, "cudaMalloc(workspace %zu bytes): %s", p->workspace_bytes, cudaGetErrorString(e)); break; }
     } else {
-      for (int a = 0; a < 3 && rc == DFT3D_OK; ++a) {
-        rc = dft3d::fft_build_axis(&p->fax[a], nn[a], sign, (sign > 0) && !(opt.flags & DFT3D_UNSCALED_INVERSE),
-                                   opt.fft_split[a][0], opt.fft_split[a][1], g_last_error, sizeof(g_last_error));
-      }
+      for (int a = 0; a < 3 && rc == DFT3D_OK; ++a) rc = build_fft_axis(p, a, opt.fft_split[a]);
       if (rc != DFT3D_OK) break;
     }
   } while (0);
@@ -397,9 +497,7 @@ int dft3d_execute_axis(dft3d_plan_t p, int axis, const void* in, void* out, void
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   if (p->mode == DFT3D_KDFT)
     return kdft_axis_pass(p, axis, static_cast<const float*>(in), static_cast<float*>(out), p->n[0], stream);
-  rc = dft3d::fft_axis_pass(&p->fax[axis], axis, p->n, static_cast<const float*>(in), static_cast<float*>(out),
-                            p->d_status, p->sm_count, stream, g_last_error, sizeof(g_last_error));
-  return rc;
+  return fft_axis_pass(p, axis, static_cast<const float*>(in), static_cast<float*>(out), stream);
 }
 
 int dft3d_execute(dft3d_plan_t p, const void* in, void* out, void* cuda_stream) {
@@ -421,13 +519,11 @@ int dft3d_execute(dft3d_plan_t p, const void* in, void* out, void* cuda_stream) 
     }
     return DFT3D_OK;
   }
-  // FFT: axis 2 in -> out, then axes 1 and 0 in place on out (a CTA reads its lines completely before it writes them)
-  if ((rc = dft3d::fft_axis_pass(&p->fax[2], 2, p->n, fin, fout, p->d_status, p->sm_count, stream, g_last_error,
-                                 sizeof(g_last_error))) != DFT3D_OK) return rc;
-  if ((rc = dft3d::fft_axis_pass(&p->fax[1], 1, p->n, fout, fout, p->d_status, p->sm_count, stream, g_last_error,
-                                 sizeof(g_last_error))) != DFT3D_OK) return rc;
-  return dft3d::fft_axis_pass(&p->fax[0], 0, p->n, fout, fout, p->d_status, p->sm_count, stream, g_last_error,
-                              sizeof(g_last_error));
+  // FFT: axis 2 in -> out, then axes 1 and 0 in place on out (a CTA loads a group of lines completely into
+  // shared memory before it stores any of their results, and groups are disjoint)
+  if ((rc = fft_axis_pass(p, 2, fin, fout, stream)) != DFT3D_OK) return rc;
+  if ((rc = fft_axis_pass(p, 1, fout, fout, stream)) != DFT3D_OK) return rc;
+  return fft_axis_pass(p, 0, fout, fout, stream);
 }
 
 int dft3d_execute_host(dft3d_plan_t p, const void* host_in, void* host_out, void* cuda_stream) {
@@ -465,7 +561,8 @@ int dft3d_plan_destroy(dft3d_plan_t p) {
   if (!p) return DFT3D_OK;
   for (int a = 0; a < 3; ++a) {
     if (p->kax[a].d_w) cudaFree(p->kax[a].d_w);
-    dft3d::fft_free_axis(&p->fax[a]);
+    if (p->fax[a].d_w) cudaFree(p->fax[a].d_w);
+    if (p->fax[a].d_tw) cudaFree(p->fax[a].d_tw);
   }
   if (p->workspace) cudaFree(p->workspace);
   if (p->d_status) cudaFree(p->d_status);

@@ -1,28 +1,371 @@
-// FFT formulation (paper Section III-B, Eq. 14-18): placeholder interface; the fused kernel follows.
+// One axis of the FFT formulation (paper Section III-B, Eq. 14-18) as ONE fused kernel: with the line
+// index split as n = R*l + beta and the output index as k = k1 + R*k2 (N = R*R),
+//
+//   stage 1   B[k1][beta] = sum_l  F_R[k1][l] * x[R*l + beta]          (the "local transform" of Eq. 18, as a GEMM)
+//   twiddle   C[k1][beta] = B[k1][beta] * exp(s*2*pi*i*k1*beta/N)      (the phase adjustment, outer factor of Eq. 17)
+//   stage 2   X[k1 + R*k2] = sum_beta F_R[k2][beta] * C[k1][beta]      (second GEMM; stored in natural order)
+//
+// The intermediate never leaves the SM: stage 1 accumulates in tensor memory, the twiddle is applied
+// in the registers of the warps that drain that accumulator, and the result is written to shared memory
+// directly in the operand layout stage 2's MMA reads.  HBM traffic is one read and one write of the data.
+//
+// Both stages use the same complex-as-real mapping as the KDFT kernel (interleaved re/im, real 2R x 2R
+// matrix W).  fp32 accuracy from TF32: the data is split x = hi + lo (two MMAs per K step) and the two
+// table pieces are stacked along N, B = [W_hi ; W_lo] (4R rows), so that the accumulator's column halves
+// hold x*W_hi and x*W_lo; the halves are added when the accumulator is drained.  A chain is at most 16 MMAs
+// long, so the truncation bias of the tensor-core accumulator stays far below fp32 rounding.
+//
+// Tile geometry.  An "M-tile" is 128 accumulator lanes.
+//   stage 1 lanes = (line g, beta)  : 128/R lines of the tile, all beta
+//   stage 2 lanes = (line g, k1)    : the same lines, all k1
+//   CONTIG  (last axis): a shared-memory stage holds 128/R whole lines (one M-tile), loaded as contiguous rows.
+//   STRIDED (axes 0, 1): a stage holds all N rows of 16 neighbouring lines (128-byte rows, 128B swizzle), i.e.
+//                        R/8 M-tiles; loads and stores touch 128-byte / 32-byte contiguous pieces.
+//
+// Warp roles (512 threads): warp 0 TMA producer, warp 1 MMA issuer, warps 4-7 split (smem -> hi/lo -> tensor
+// memory), warps 8-11 drain stage 1 (+twiddle, write stage-2 operand), warps 12-15 drain stage 2 (+store).
 #pragma once
-#include <cstdio>
+#include <cstdint>
+#include <cuda.h>
 #include <cuda_runtime.h>
+#include "ptx_sm100.cuh"
+#include "kdft_kernel.cuh"   // bounded_wait
 
 namespace dft3d {
 
-struct FftAxis {
-  long long n = 0;
-  int N1 = 0, N2 = 0;
+enum : int { FFT_CONTIG = 0, FFT_STRIDED = 1 };
+
+constexpr int kFftThreads = 512;
+constexpr int kFftRawBytes = 128 * 1024;       // ring of raw-data stages
+constexpr int kFftStridedCols = 16;            // lines per STRIDED stage (128-byte rows)
+constexpr int kFftTmemD1 = 0, kFftTmemD2 = 128, kFftTmemA1 = 256;   // tensor-memory column map (A1: two buffers of 128)
+
+struct FftParams {
+  int N;                 // R*R
+  int raw_stages;        // stages in the raw ring
+  int stage_bytes;       // bytes of one raw stage
+  int mtiles_per_stage;  // CONTIG 1, STRIDED 16/(128/R)
+  long long num_stages;  // work items (stages) in the whole pass
+  // CONTIG
+  long long rows;        // number of lines
+  // STRIDED: view [batches][N][C] complex
+  long long C;
+  long long c_tiles;     // C / 16
+  const float2* twiddle; // [R][R] complex64, T[k1][beta]
+  float* out;
+  unsigned int* status;
 };
 
-inline int fft_set_kernel_attributes() { return 0; }
+struct FftShared {
+  uint64_t raw_full[4], raw_empty[4];
+  uint64_t a1_full[2], a1_empty[2];
+  uint64_t d1_full, d1_empty;
+  uint64_t a2_full, a2_empty;
+  uint64_t d2_full, d2_empty;
+  uint64_t w_full;
+  uint32_t tmem_base;
+  volatile int abort_flag;
+};
 
-inline int fft_build_axis(FftAxis*, long long, int, bool, int, int, char* err, size_t errlen) {
-  snprintf(err, errlen, "the FFT formulation is not built yet");
-  return 2;  // DFT3D_ERR_UNSUPPORTED
+// shared memory: [W: 4R rows x 2R floats, as 2R/32 panels of 4R x 128 B] [A2: hi panels, lo panels] [raw ring] [barriers]
+__host__ __device__ constexpr int fft_w_bytes(int R) { return (2 * R / 32) * 4 * R * 128; }
+__host__ __device__ constexpr int fft_a2_piece_bytes(int R) { return (2 * R / 32) * 128 * 128; }
+__host__ __device__ constexpr size_t fft_smem_bytes(int R) {
+  return size_t(fft_w_bytes(R)) + 2 * size_t(fft_a2_piece_bytes(R)) + kFftRawBytes + 1024 + 512;
 }
 
-inline int fft_axis_pass(const FftAxis*, int, const long long*, const float*, float*, unsigned int*, int, cudaStream_t,
-                         char* err, size_t errlen) {
-  snprintf(err, errlen, "the FFT formulation is not built yet");
-  return 2;
+#define FFT_WAIT(bar, parity, code)                                 \
+  if (!bounded_wait((bar), (parity), &sh.abort_flag)) {             \
+    sh.abort_flag = 1;                                              \
+    atomicCAS(p.status, 0u, (unsigned)(code));                      \
+    goto role_done;                                                 \
+  }
+#define FFT_WAIT_WARP(bar, parity, code)                                                \
+  if (!__all_sync(0xffffffffu, bounded_wait((bar), (parity), &sh.abort_flag) ? 1 : 0)) { \
+    sh.abort_flag = 1;                                                                  \
+    atomicCAS(p.status, 0u, (unsigned)(code));                                          \
+    goto role_done;                                                                     \
+  }
+
+template <int MODE, int R>
+__global__ void __launch_bounds__(kFftThreads, 1)
+fft_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_constant__ CUtensorMap map_w,
+                const FftParams p) {
+  extern __shared__ uint8_t smem_raw_[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw_) + 1023) & ~uintptr_t(1023));
+  constexpr int K = 2 * R;             // reals per contraction
+  constexpr int NB = 4 * R;            // MMA N: stacked [W_hi; W_lo]
+  constexpr int panels = K / 32;
+  uint8_t* smem_w = smem;
+  uint8_t* smem_a2 = smem_w + fft_w_bytes(R);
+  constexpr int a2_piece = fft_a2_piece_bytes(R);
+  uint8_t* smem_rawring = smem_a2 + 2 * a2_piece;
+  FftShared& sh = *reinterpret_cast<FftShared*>(smem_rawring + kFftRawBytes);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  constexpr int Lg = 128 / R;          // lines per M-tile
+
+  if (tid == 0) {
+    for (int i = 0; i < 4; ++i) { ptx::mbar_init(&sh.raw_full[i], 1); ptx::mbar_init(&sh.raw_empty[i], 4 * p.mtiles_per_stage); }
+    for (int i = 0; i < 2; ++i) { ptx::mbar_init(&sh.a1_full[i], 4); ptx::mbar_init(&sh.a1_empty[i], 1); }
+    ptx::mbar_init(&sh.d1_full, 1); ptx::mbar_init(&sh.d1_empty, 4);
+    ptx::mbar_init(&sh.a2_full, 4); ptx::mbar_init(&sh.a2_empty, 1);
+    ptx::mbar_init(&sh.d2_full, 1); ptx::mbar_init(&sh.d2_empty, 4);
+    ptx::mbar_init(&sh.w_full, 1);
+    sh.abort_flag = 0;
+    ptx::fence_mbar_init();
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc(&sh.tmem_base, 512);
+    ptx::tmem_relinquish();
+  }
+  if (warp == 0 && lane == 0) {
+    ptx::prefetch_tensormap(&map_data);
+    ptx::prefetch_tensormap(&map_w);
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem = sh.tmem_base;
+
+  // this CTA's share of the stages, and the M-tiles in them
+  long long my_stages = 0;
+  if ((long long)blockIdx.x < p.num_stages) my_stages = (p.num_stages - 1 - blockIdx.x) / gridDim.x + 1;
+  const long long my_mtiles = my_stages * p.mtiles_per_stage;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      ptx::mbar_arrive_expect_tx(&sh.w_full, uint32_t(fft_w_bytes(R)));
+      for (int pn = 0; pn < panels; ++pn)
+        ptx::tma_load_2d(smem_w + pn * NB * 128, &map_w, &sh.w_full, 0, pn * NB);
+      long long i = 0;
+      for (long long sidx = blockIdx.x; sidx < p.num_stages; sidx += gridDim.x, ++i) {
+        const uint32_t s = uint32_t(i % p.raw_stages), ph = uint32_t(i / p.raw_stages) & 1;
+        FFT_WAIT(&sh.raw_empty[s], ph ^ 1, 0x501);
+        ptx::mbar_arrive_expect_tx(&sh.raw_full[s], uint32_t(p.stage_bytes));
+        uint8_t* dst = smem_rawring + size_t(s) * p.stage_bytes;
+        if (MODE == FFT_CONTIG) {
+          ptx::tma_load_3d(dst, &map_data, &sh.raw_full[s], 0, 0, int(sidx * Lg));
+        } else {
+          const long long ct = sidx % p.c_tiles, bt = sidx / p.c_tiles;
+          for (int r0 = 0; r0 < p.N; r0 += 256)
+            ptx::tma_load_3d(dst + size_t(r0) * 128, &map_data, &sh.raw_full[s], int(ct * 32), r0, int(bt));
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer (stage 1 of M-tile t, then stage 2 of t-1)
+    if (lane == 0) {
+      const uint32_t idesc = ptx::make_idesc_tf32(128, NB);
+      const uint32_t w_addr = ptx::smem_u32(smem_w);
+      const uint32_t a2_addr = ptx::smem_u32(smem_a2);
+      FFT_WAIT(&sh.w_full, 0, 0x601);
+      for (long long t = 0; t <= my_mtiles; ++t) {
+        if (t < my_mtiles) {
+          const uint32_t b = uint32_t(t & 1), phb = uint32_t(t >> 1) & 1;
+          FFT_WAIT(&sh.a1_full[b], phb, 0x602);
+          FFT_WAIT(&sh.d1_empty, (uint32_t(t) & 1) ^ 1, 0x603);
+          ptx::tc_fence_after();
+          const uint32_t a_hi = tmem + kFftTmemA1 + b * 128, a_lo = a_hi + K;
+#pragma unroll
+          for (int k8 = 0; k8 < K / 8; ++k8) {
+            const uint64_t wd = ptx::make_kmajor_sw128_desc(w_addr + (k8 >> 2) * NB * 128 + (k8 & 3) * 32);
+            ptx::mma_tf32_ts(tmem + kFftTmemD1, a_hi + k8 * 8, wd, idesc, k8 != 0);
+            ptx::mma_tf32_ts(tmem + kFftTmemD1, a_lo + k8 * 8, wd, idesc, 1);
+          }
+          ptx::tc_commit(&sh.a1_empty[b]);
+          ptx::tc_commit(&sh.d1_full);
+        }
+        if (t >= 1) {
+          const uint32_t u = uint32_t(t - 1);
+          FFT_WAIT(&sh.a2_full, u & 1, 0x604);
+          FFT_WAIT(&sh.d2_empty, (u & 1) ^ 1, 0x605);
+          ptx::tc_fence_after();
+#pragma unroll
+          for (int k8 = 0; k8 < K / 8; ++k8) {
+            const uint32_t off = (k8 >> 2) * 128 * 128 + (k8 & 3) * 32;
+            const uint64_t wd = ptx::make_kmajor_sw128_desc(w_addr + (k8 >> 2) * NB * 128 + (k8 & 3) * 32);
+            ptx::mma_tf32_ss(tmem + kFftTmemD2, ptx::make_kmajor_sw128_desc(a2_addr + off), wd, idesc, k8 != 0);
+            ptx::mma_tf32_ss(tmem + kFftTmemD2, ptx::make_kmajor_sw128_desc(a2_addr + a2_piece + off), wd, idesc, 1);
+          }
+          ptx::tc_commit(&sh.a2_empty);
+          ptx::tc_commit(&sh.d2_full);
+        }
+      }
+    }
+  } else if (warp >= 4 && warp < 8) {
+    // ------------------------------------------------------------ split: raw lines -> (hi, lo) -> tensor memory A1
+    const int q = warp & 3;
+    const int m = q * 32 + lane;
+    const int g = m / R, beta = m % R;            // stage-1 lane = (line g, beta), beta fastest
+    const uint32_t lane_addr = tmem + (uint32_t(q * 32) << 16);
+    long long t = 0;
+    for (long long i = 0; i < my_stages; ++i) {
+      const uint32_t s = uint32_t(i % p.raw_stages), phs = uint32_t(i / p.raw_stages) & 1;
+      FFT_WAIT_WARP(&sh.raw_full[s], phs, 0x701);
+      const uint8_t* stage = smem_rawring + size_t(s) * p.stage_bytes;
+      for (int mt = 0; mt < p.mtiles_per_stage; ++mt, ++t) {
+        // element l of this lane's sub-sequence sits at base + l*stride (bytes)
+        uint32_t base, stride;
+        if (MODE == FFT_CONTIG) {
+          base = uint32_t(g * p.N + beta) * 8u;
+          stride = uint32_t(R) * 8u;
+        } else {
+          const int c = mt * Lg + g;                // column within the 16-wide stage
+          base = uint32_t(beta) * 128u + (uint32_t((c >> 1) ^ (beta & 7)) << 4) + uint32_t(c & 1) * 8u;
+          stride = uint32_t(R) * 128u;
+        }
+        const uint32_t b = uint32_t(t & 1), phb = uint32_t(t >> 1) & 1;
+        FFT_WAIT_WARP(&sh.a1_empty[b], phb ^ 1, 0x702);
+        ptx::tc_fence_after();
+        const uint32_t a_hi = lane_addr + kFftTmemA1 + b * 128, a_lo = a_hi + K;
+#pragma unroll
+        for (int l0 = 0; l0 < R; l0 += 16) {      // 16 complex = 32 reals per tensor-memory store
+          uint32_t x[32], lo[32];
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            const uint2 v = *reinterpret_cast<const uint2*>(stage + base + uint32_t(l0 + j) * stride);
+            x[2 * j] = v.x; x[2 * j + 1] = v.y;
+          }
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            const float r = __uint_as_float(x[j]) - __uint_as_float(x[j] & 0xffffe000u);
+            lo[j] = (__float_as_uint(r) + 0x1000u) & 0xffffe000u;
+          }
+          ptx::tmem_st_32x32(a_hi + l0 * 2, x);
+          ptx::tmem_st_32x32(a_lo + l0 * 2, lo);
+        }
+        ptx::tc_wait_st();
+        ptx::tc_fence_before();
+        // the raw stage is refilled by TMA (async proxy): order this thread's reads before that write
+        ptx::fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) {
+          ptx::mbar_arrive(&sh.a1_full[b]);
+          ptx::mbar_arrive(&sh.raw_empty[s]);
+        }
+      }
+    }
+  } else if (warp >= 8 && warp < 12) {
+    // ------------------------------------------------------------ drain stage 1: sum halves, twiddle, split, write A2
+    const int q = warp & 3;
+    const int m = q * 32 + lane;
+    const int g = m / R, beta = m % R;
+    const uint32_t lane_addr = tmem + (uint32_t(q * 32) << 16) + kFftTmemD1;
+    // A2 row of (g, k1): CONTIG g*R + k1 ; STRIDED k1*Lg + g (so that stage-2 stores of one k2 touch neighbouring lines)
+    const int row_mul_k1 = (MODE == FFT_CONTIG) ? 1 : Lg;
+    const int row_base = (MODE == FFT_CONTIG) ? g * R : g;
+    // K column (beta, q) -> panel beta/16, 16-byte chunk (beta%16)/2, half beta%2
+    const uint32_t a2_col = uint32_t(beta >> 4) * (128u * 128u) + uint32_t(beta & 1) * 8u;
+    const uint32_t a2_chunk = uint32_t(beta & 15) >> 1;
+    const float2* tw = p.twiddle + beta;
+    for (long long t = 0; t < my_mtiles; ++t) {
+      FFT_WAIT_WARP(&sh.d1_full, uint32_t(t) & 1, 0x801);
+      ptx::tc_fence_after();
+      float cre[R], cim[R];                         // C[k1] for this lane's beta
+#pragma unroll
+      for (int ch = 0; ch < K / 32; ++ch) {         // 32 reals = 16 values of k1 per chunk
+        uint32_t v0[32], v1[32];
+        ptx::tmem_ld_32x32(lane_addr + ch * 32, v0);
+        ptx::tmem_ld_32x32(lane_addr + K + ch * 32, v1);
+        ptx::tc_wait_ld();
+        if (ch == K / 32 - 1) {
+          ptx::tc_fence_before();
+          __syncwarp();
+          if (lane == 0) ptx::mbar_arrive(&sh.d1_empty);
+        }
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          const float br = __uint_as_float(v0[2 * j]) + __uint_as_float(v1[2 * j]);
+          const float bi = __uint_as_float(v0[2 * j + 1]) + __uint_as_float(v1[2 * j + 1]);
+          const float2 w = __ldg(tw + (ch * 16 + j) * R);
+          cre[ch * 16 + j] = br * w.x - bi * w.y;
+          cim[ch * 16 + j] = br * w.y + bi * w.x;
+        }
+      }
+      // stage 2 of the previous M-tile must be done reading A2
+      FFT_WAIT_WARP(&sh.a2_empty, (uint32_t(t) & 1) ^ 1, 0x802);
+#pragma unroll
+      for (int k1 = 0; k1 < R; ++k1) {
+        {
+          const int row = row_base + k1 * row_mul_k1;
+          const uint32_t off = a2_col + uint32_t(row) * 128u + ((a2_chunk ^ uint32_t(row & 7)) << 4);
+          const uint32_t hr = __float_as_uint(cre[k1]), hi_ = __float_as_uint(cim[k1]);
+          const float lr = cre[k1] - __uint_as_float(hr & 0xffffe000u);
+          const float li = cim[k1] - __uint_as_float(hi_ & 0xffffe000u);
+          *reinterpret_cast<uint2*>(smem_a2 + off) = make_uint2(hr, hi_);
+          *reinterpret_cast<uint2*>(smem_a2 + a2_piece + off) =
+              make_uint2((__float_as_uint(lr) + 0x1000u) & 0xffffe000u, (__float_as_uint(li) + 0x1000u) & 0xffffe000u);
+        }
+      }
+      ptx::fence_proxy_async_smem();                // generic writes -> visible to the MMA's shared-memory reads
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(&sh.a2_full);
+    }
+  } else if (warp >= 12) {
+    // ------------------------------------------------------------ drain stage 2: sum halves, store in natural order
+    const int q = warp & 3;
+    const int m = q * 32 + lane;
+    const int g = (MODE == FFT_CONTIG) ? m / R : m % Lg;
+    const int k1 = (MODE == FFT_CONTIG) ? m % R : m / Lg;
+    const uint32_t lane_addr = tmem + (uint32_t(q * 32) << 16) + kFftTmemD2;
+    long long t = 0;
+    long long i = 0;
+    for (long long sidx = blockIdx.x; sidx < p.num_stages; sidx += gridDim.x, ++i) {
+      for (int mt = 0; mt < p.mtiles_per_stage; ++mt, ++t) {
+        float2* dst;              // &out[line][k1], element k2 at dst + k2*k2_stride
+        long long k2_stride;
+        bool ok;
+        if (MODE == FFT_CONTIG) {
+          const long long line = sidx * Lg + g;
+          ok = line < p.rows;
+          dst = reinterpret_cast<float2*>(p.out) + line * p.N + k1;
+          k2_stride = R;
+        } else {
+          const long long ct = sidx % p.c_tiles, bt = sidx / p.c_tiles;
+          const long long col = ct * kFftStridedCols + mt * Lg + g;
+          ok = col < p.C;
+          dst = reinterpret_cast<float2*>(p.out) + (bt * p.N + k1) * p.C + col;
+          k2_stride = (long long)R * p.C;
+        }
+        FFT_WAIT_WARP(&sh.d2_full, uint32_t(t) & 1, 0x901);
+        ptx::tc_fence_after();
+#pragma unroll
+        for (int ch = 0; ch < K / 32; ++ch) {
+          uint32_t v0[32], v1[32];
+          ptx::tmem_ld_32x32(lane_addr + ch * 32, v0);
+          ptx::tmem_ld_32x32(lane_addr + K + ch * 32, v1);
+          ptx::tc_wait_ld();
+          if (ch == K / 32 - 1) {
+            ptx::tc_fence_before();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(&sh.d2_empty);
+          }
+          if (ok) {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              const float yr = __uint_as_float(v0[2 * j]) + __uint_as_float(v1[2 * j]);
+              const float yi = __uint_as_float(v0[2 * j + 1]) + __uint_as_float(v1[2 * j + 1]);
+              dst[(long long)(ch * 16 + j) * k2_stride] = make_float2(yr, yi);
+            }
+          }
+        }
+      }
+    }
+  }
+
+role_done:
+  if (warp == 0 && lane == 0 && sh.abort_flag) {
+    const long long t0 = clock64();
+    while (clock64() - t0 < 2000000LL) { }
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (warp == 1) ptx::tmem_dealloc(tmem, 512);
 }
 
-inline void fft_free_axis(FftAxis*) {}
+#undef FFT_WAIT
+#undef FFT_WAIT_WARP
 
 }  // namespace dft3d
