@@ -1,13 +1,15 @@
 #!/usr/bin/env python
 """Benchmark of the 3D complex DFT hot path (one JSON line on stdout).
 
-A "step" is one whole 3D complex-to-complex transform of a seeded synthetic n^3 cube through the
-C-ABI library (`dft3d_execute`: three per-axis tensor-core GEMM passes).  Default workload: the
-1024^3 cube the headline metric is quoted on, input U(-1,1).  `value` is GFLOP/s in the 5*P*log2(P)
-convention (P = n^3 points), with the input already resident in HBM; `e2e` is the same metric
-through `dft3d_execute_host` with pinned HOST buffers (H2D and D2H copies inside the timed region).
+A "step" is one whole 3D complex-to-complex transform of a seeded synthetic cube through the C-ABI
+library (`dft3d_execute`: three per-axis tensor-core passes).  Default workload: the 1024^3 cube the
+headline metric is quoted on, input U(-1,1), in the FFT formulation (GEMM - twiddle - GEMM per axis);
+the KDFT formulation (dense N x N matrix per axis) of the same cube is timed in the same run and
+reported under "kdft".  `value` is GFLOP/s in the 5*P*log2(P) convention (P points), with the input
+already resident in HBM; `e2e` is the same metric through `dft3d_execute_host` with pinned HOST
+buffers (H2D and D2H copies inside the timed region).
 
-python bench.py [--gpus N] [--steps K] [--warmup W] [--mode kdft|fft] [--n 1024] [--impl reference]
+python bench.py [--gpus N] [--steps K] [--warmup W] [--mode fft|kdft] [--n 1024 | --shape a,b,c] [--impl reference]
 Under torchrun every rank transforms its own cube (independent problems, no collective): weak scaling.
 """
 import argparse
@@ -34,6 +36,8 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--mode", choices=["kdft", "fft"], default=None)
     ap.add_argument("--n", type=int, default=1024)
+    ap.add_argument("--shape", type=str, default=None, help="n0,n1,n2 instead of a cube (profiling on smaller cases)")
+    ap.add_argument("--no-kdft", action="store_true", help="FFT mode only: skip the KDFT timing of the same cube")
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing leg")
@@ -41,7 +45,8 @@ def parse_args():
 
 
 def conv_flops(n):
-    P = float(n) ** 3
+    """5*P*log2(P); n is the cube edge or a shape tuple."""
+    P = float(n) ** 3 if not isinstance(n, tuple) else float(n[0]) * n[1] * n[2]
     return 5.0 * P * math.log2(P)
 
 
@@ -171,12 +176,10 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
 
     n = args.n
-    mode = args.mode or "kdft"
-    mode_id = dft.DFT3D_KDFT if mode == "kdft" else dft.DFT3D_FFT
-    shape = (n, n, n)
+    mode = args.mode or "fft"
+    shape = (n, n, n) if not args.shape else tuple(int(v) for v in args.shape.split(","))
     x = inputs.cube(shape, "uniform", 1003 + rank, device="cuda")
     y = torch.empty_like(x)
-    plan = dft.Plan(*shape, mode=mode_id, sign=dft.DFT3D_FORWARD)
     stream = torch.cuda.current_stream()
 
     def barrier():
@@ -184,26 +187,36 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
-    for _ in range(args.warmup):
-        plan.execute(x, y)
-    barrier()
-    sampler = ClockSampler(local_rank)
-    if rank == 0:
-        sampler.start()
-    ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
-    ev[0].record(stream)
-    for i in range(args.steps):
-        plan.execute(x, y)
-        ev[i + 1].record(stream)
-    barrier()
-    clocks = sampler.stop() if rank == 0 else None
-    plan.status()
-    ms_total = ev[0].elapsed_time(ev[-1])
-    t = torch.tensor([ms_total], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_step = float(t.item()) / args.steps
+    def time_mode(mode_name, steps, warmup, sample_clocks):
+        """W warm-up steps, then K timed steps between barriers; CUDA events on the launching stream; max over ranks."""
+        plan_ = dft.Plan(*shape, mode=dft.DFT3D_KDFT if mode_name == "kdft" else dft.DFT3D_FFT, sign=dft.DFT3D_FORWARD)
+        for _ in range(warmup):
+            plan_.execute(x, y)
+        barrier()
+        sampler = ClockSampler(local_rank)
+        if sample_clocks and rank == 0:
+            sampler.start()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(steps):
+            plan_.execute(x, y)
+        e1.record(stream)
+        barrier()
+        clk = sampler.stop() if (sample_clocks and rank == 0) else None
+        plan_.status()
+        t = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device="cuda")
+        if world > 1:
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return plan_, float(t.item()) / steps, clk
+
+    plan, ms_step, clocks = time_mode(mode, args.steps, args.warmup, True)
     launches = plan.launches
+    kdft_info = None
+    if mode == "fft" and not args.no_kdft:
+        ksteps = max(1, min(args.steps, 3))
+        kplan, kms, kclk = time_mode("kdft", ksteps, 3, True)
+        kdft_info = {"ms_per_step": kms, "steps": ksteps, "warmup": 3, "launches_per_step": kplan.launches, "clocks": kclk}
+        kplan.destroy()
 
     # ---- end to end through the host-buffer entry point
     e2e = None
@@ -224,46 +237,58 @@ def main():
             dist.all_reduce(te, op=dist.ReduceOp.MAX)
         ms_e2e = float(te.item()) / e2e_steps
         nbytes = x.numel() * 8
-        e2e = {"value": world * conv_flops(n) / ms_e2e * 1e-6, "unit": "GFLOP/s", "ms_per_step": ms_e2e,
+        e2e = {"value": world * conv_flops(shape) / ms_e2e * 1e-6, "unit": "GFLOP/s", "ms_per_step": ms_e2e,
                "h2d_bytes_per_step": nbytes, "d2h_bytes_per_step": nbytes, "steps": e2e_steps,
                "call": "dft3d_execute_host (pinned host buffers)"}
         del xh, yh
 
     if rank == 0:
         peaks, peak_kind = measured_peaks()
-        P = float(n) ** 3
-        if mode == "kdft":
-            # dominant (only) kernel: kdft_axis_kernel; algorithmic flops per point per axis = 8*n (4 real
-            # multiply-adds per complex MAC), issued three times for the TF32 split
-            algo_flops = 3 * 8.0 * n * P
-            issued_flops = 3.0 * algo_flops
+        P = float(shape[0]) * shape[1] * shape[2]
+        nsum = float(sum(shape))
+
+        def kdft_roofline(ms, nlaunch):
+            # only kernel: kdft_axis_kernel.  Algorithmic flops per point per axis = 8*n_a (4 real multiply-adds per
+            # complex MAC); the tensor cores issue them three times (TF32 split: hi*hi, lo*hi, hi*lo).
+            algo_flops = 8.0 * nsum * P
+            issued = 3.0 * algo_flops
             tf32_peak = peaks["bf16_tflops_sustained"] * (1.1 / 2.25)
-            achieved = issued_flops / (ms_step * 1e-3) * 1e-12
-            roofline = {"bound": "tensor", "kernel": "kdft_axis_kernel", "achieved": achieved, "peak": tf32_peak,
-                        "unit": "TFLOP/s", "frac": achieved / tf32_peak, "traffic": None,
-                        "peak_source": "%s bf16 sustained x nominal TF32/bf16 ratio (1.1/2.25)" % peak_kind,
-                        "flops": "issued TF32 tensor flops = 3 split products x 8*n flops per point per axis",
-                        "useful_gemm_tflops": algo_flops / (ms_step * 1e-3) * 1e-12,
-                        "avg_launch_ms": ms_step / launches}
+            ach = issued / (ms * 1e-3) * 1e-12
+            return {"bound": "tensor", "kernel": "kdft_axis_kernel", "achieved": ach, "peak": tf32_peak, "unit": "TFLOP/s",
+                    "frac": ach / tf32_peak, "traffic": None,
+                    "peak_source": "%s bf16 sustained x nominal TF32/bf16 ratio (1.1/2.25)" % peak_kind,
+                    "flops": "issued TF32 tensor flops = 3 split products x 8*n_a flops per point per axis",
+                    "useful_gemm_tflops": algo_flops / (ms * 1e-3) * 1e-12, "avg_launch_ms": ms / nlaunch}
+
+        if mode == "kdft":
+            roofline = kdft_roofline(ms_step, launches)
         else:
+            # only kernel: fft_axis_kernel, one launch per axis; algorithmic traffic 16 B per point per axis
             algo_bytes = 3 * 16.0 * P
             achieved = algo_bytes / (ms_step * 1e-3) * 1e-9
             roofline = {"bound": "hbm", "kernel": "fft_axis_kernel", "achieved": achieved, "peak": peaks["hbm_gbs"],
                         "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "traffic": None,
-                        "peak_source": "%s STREAM-style copy" % peak_kind, "avg_launch_ms": ms_step / launches}
+                        "peak_source": "%s STREAM-style copy" % peak_kind, "avg_launch_ms": ms_step / launches,
+                        "bytes": "8 B read + 8 B written per point per axis pass"}
+        if kdft_info is not None:
+            kdft_info["value"] = world * conv_flops(shape) / kdft_info["ms_per_step"] * 1e-6
+            kdft_info["unit"] = "GFLOP/s"
+            kdft_info["roofline"] = kdft_roofline(kdft_info["ms_per_step"], kdft_info["launches_per_step"])
         cpu = None
         if not args.no_cpu_baseline:
             planes = max(1, min(n, int(3.0e10 / (float(n) ** 3))))
-            cpu = oracle_sample(n, planes, 1003)
-        line = {"metric": "3D C2C DFT GFLOP/s (5*P*log2P) at %d^3" % n,
-                "value": world * conv_flops(n) / ms_step * 1e-6, "unit": "GFLOP/s", "n_gpus": world,
+            cpu = oracle_sample(n, planes, 1003) if not args.shape else None
+        wl = "%d^3" % n if not args.shape else "x".join(str(v) for v in shape)
+        line = {"metric": "3D C2C DFT GFLOP/s (5*P*log2P) at %s" % wl,
+                "value": world * conv_flops(shape) / ms_step * 1e-6, "unit": "GFLOP/s", "n_gpus": world,
                 "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": "tf32x3", "data": "synthetic",
-                "config": {"workload": "%s forward 3D complex64 DFT %d^3, re/im iid U(-1,1), seed 1003+rank" % (mode.upper(), n),
-                           "mode": mode, "n": n, "l2": "input and output (%.1f GiB each) are larger than L2" % (P * 8 / 2**30),
+                "config": {"workload": "%s forward 3D complex64 DFT %s, re/im iid U(-1,1), seed 1003+rank" % (mode.upper(), wl),
+                           "mode": mode, "shape": list(shape),
+                           "l2": "input and output (%.2f GiB each) are larger than L2" % (P * 8 / 2**30),
                            "per_rank": "one independent cube per GPU"},
                 "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches * args.steps,
-                "clocks": clocks}
+                "clocks": clocks, "kdft": kdft_info}
         print(json.dumps(line))
     plan.destroy()
     if world > 1:
