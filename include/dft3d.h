@@ -149,6 +149,33 @@ int dft3d_generate_twiddle(long long N1, long long N2, int sign, double* twiddle
 int dft3d_generate_real_table(long long n, int sign, double scale, const double* nodes, int nodes_on_output,
                               float* hi, float* lo);
 
+/*
+ * The KDFT forward/inverse transform without any allocation (the paper has no counterpart to this call; it
+ * exists for callers that cannot call cudaMalloc: code inside a section where the allocator is off limits,
+ * plugins whose host owns all device memory, processes that have given every free byte to their own arena).
+ *
+ *   n0, n1, n2   sizes, each a multiple of 64, with n0*n1*n2 <= 2,097,152 points (the static scratch holds
+ *                16 MiB); larger sizes return DFT3D_ERR_UNSUPPORTED and say so in error_message.
+ *   w0, w1, w2   DEVICE pointers, 16-byte aligned: the per-axis real tables, [hi piece][lo piece], each piece
+ *                (2*n_a)*(2*n_a) floats, exactly as dft3d_generate_real_table writes them (hi first, lo right
+ *                after it).  Sign, inverse scaling and nonuniform nodes are whatever the caller generated.
+ *   in, out      DEVICE pointers as for dft3d_execute (16-byte aligned, n0*n1*n2*8 bytes, not overlapping).
+ *   cuda_stream  the stream the three axis kernels run on.
+ *   error_message / error_message_size   optional HOST buffer that receives a description of a failure.
+ *
+ * The scratch cube between the axis passes is a file-scope device array inside the library: every GPU that
+ * loads the library holds it until the process exits, every call on that GPU shares it, and it keeps the
+ * previous call's contents (the call clears the one word that must start at zero).  Calls that overlap on the
+ * same GPU, from any stream or thread, therefore race; run them one after the other.
+ * The first call on a device resolves the array's address and sets kernel attributes; make that first call
+ * before any stream capture.  The call enqueues its kernels, then waits for the stream and returns
+ * DFT3D_ERR_DEVICE_TIMEOUT if a kernel abandoned a wait.  It calls no cudaMalloc, cudaFree or other
+ * allocating routine.
+ */
+int dft3d_kdft_execute_static(long long n0, long long n1, long long n2, const float* w0, const float* w1,
+                              const float* w2, const void* in, void* out, void* cuda_stream,
+                              char* error_message, size_t error_message_size);
+
 #ifdef __cplusplus
 }
 #endif

@@ -21,7 +21,7 @@ EXPORTS = [
     "dft3d_plan_create", "dft3d_plan_create_ex", "dft3d_execute", "dft3d_execute_host", "dft3d_execute_axis",
     "dft3d_plan_status", "dft3d_plan_workspace_bytes", "dft3d_plan_launches", "dft3d_plan_destroy",
     "dft3d_status_string", "dft3d_last_error", "dft3d_generate_axis_matrix", "dft3d_generate_twiddle",
-    "dft3d_generate_real_table",
+    "dft3d_generate_real_table", "dft3d_kdft_execute_static",
 ]
 
 
@@ -63,6 +63,7 @@ def _load():
     lib.dft3d_generate_axis_matrix.argtypes = [ll, ci, cd, vp, ci, vp]
     lib.dft3d_generate_twiddle.argtypes = [ll, ll, ci, vp]
     lib.dft3d_generate_real_table.argtypes = [ll, ci, cd, vp, ci, vp, vp]
+    lib.dft3d_kdft_execute_static.argtypes = [ll, ll, ll, vp, vp, vp, vp, vp, vp, ctypes.c_char_p, ctypes.c_size_t]
     return lib
 
 
@@ -107,6 +108,23 @@ def generate_real_table(n, sign=-1, scale=1.0, nodes=None, nodes_on_output=False
     _check(_lib.dft3d_generate_real_table(n, sign, float(scale), ptr, int(nodes_on_output),
                                           hi.ctypes.data, lo.ctypes.data))
     return hi, lo
+
+
+def kdft_execute_static(x, out, tables, stream=None):
+    """dft3d_kdft_execute_static: KDFT of `x` into `out` without any allocation by the library.
+
+    For callers that cannot allocate device memory where the transform is needed.  `tables` are three
+    float32 CUDA tensors of shape [2, 2*n_a, 2*n_a] (the hi and lo pieces of dft3d_generate_real_table for
+    each axis), owned by the caller.  Limited to n0*n1*n2 <= 2**21 points; calls on one GPU must not overlap.
+    """
+    n0, n1, n2 = x.shape
+    msg = ctypes.create_string_buffer(384)
+    status = _lib.dft3d_kdft_execute_static(n0, n1, n2, tables[0].data_ptr(), tables[1].data_ptr(),
+                                            tables[2].data_ptr(), x.data_ptr(), out.data_ptr(),
+                                            _stream_ptr(stream), msg, len(msg))
+    if status != 0:
+        raise Dft3dError(status, "%s: %s" % (_lib.dft3d_status_string(status).decode(), msg.value.decode()))
+    return out
 
 
 def _stream_ptr(stream):
