@@ -32,7 +32,7 @@ SMI_QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.acti
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--mode", choices=["kdft", "fft"], default=None)
     ap.add_argument("--n", type=int, default=1024)
@@ -73,7 +73,7 @@ class ClockSampler:
             self.out = open(self.path, "w")
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + SMI_QUERY, "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=self.out, stderr=subprocess.DEVNULL)
+                 "-lms", "50"], stdout=self.out, stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
 
@@ -164,7 +164,7 @@ def main():
     import torch
     import torch.distributed as dist
     import paper_2002_03260_b200 as dft
-    from paper_2002_03260_b200 import inputs
+    from paper_2002_03260_b200 import inputs, replicas
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -178,7 +178,7 @@ def main():
     n = args.n
     mode = args.mode or "fft"
     shape = (n, n, n) if not args.shape else tuple(int(v) for v in args.shape.split(","))
-    x = inputs.cube(shape, "uniform", 1003 + rank, device="cuda")
+    x = inputs.cube(shape, "uniform", replicas.rank_seed(1003, rank), device="cuda")
     y = torch.empty_like(x)
     stream = torch.cuda.current_stream()
 
@@ -204,10 +204,7 @@ def main():
         barrier()
         clk = sampler.stop() if (sample_clocks and rank == 0) else None
         plan_.status()
-        t = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device="cuda")
-        if world > 1:
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return plan_, float(t.item()) / steps, clk
+        return plan_, replicas.max_over_ranks(e0.elapsed_time(e1), "cuda") / steps, clk
 
     plan, ms_step, clocks = time_mode(mode, args.steps, args.warmup, True)
     launches = plan.launches
@@ -232,10 +229,7 @@ def main():
             plan.execute_host(xh, yh)
         e1.record(stream)
         barrier()
-        te = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device="cuda")
-        if world > 1:
-            dist.all_reduce(te, op=dist.ReduceOp.MAX)
-        ms_e2e = float(te.item()) / e2e_steps
+        ms_e2e = replicas.max_over_ranks(e0.elapsed_time(e1), "cuda") / e2e_steps
         nbytes = x.numel() * 8
         e2e = {"value": world * conv_flops(shape) / ms_e2e * 1e-6, "unit": "GFLOP/s", "ms_per_step": ms_e2e,
                "h2d_bytes_per_step": nbytes, "d2h_bytes_per_step": nbytes, "steps": e2e_steps,

@@ -58,7 +58,7 @@ int get_encoder(EncodeTiledFn* fn) {
 
 // float32 tensor map with up to 3 dimensions; dims/box innermost first; strides in bytes for dims 1..rank-1
 int encode_f32(CUtensorMap* map, const void* base, int rank, const unsigned long long* dims,
-               const unsigned long long* strides_bytes, const unsigned* box, bool swizzle128) {
+               const unsigned long long* strides_bytes, const unsigned* box, int swizzle_bytes) {
   EncodeTiledFn enc;
   int rc = get_encoder(&enc);
   if (rc != DFT3D_OK) return rc;
@@ -67,7 +67,9 @@ int encode_f32(CUtensorMap* map, const void* base, int rank, const unsigned long
   for (int i = 0; i < rank; ++i) { d[i] = dims[i]; b[i] = box[i]; es[i] = 1; }
   for (int i = 0; i + 1 < rank; ++i) s[i] = strides_bytes[i];
   CUresult cr = enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, rank, const_cast<void*>(base), d, s, b, es,
-                    CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE,
+                    swizzle_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
+                                         : (swizzle_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_NONE),
                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (cr != CUDA_SUCCESS)
     return fail(DFT3D_ERR_CUDA, "cuTensorMapEncodeTiled failed with %d (rank %d, dims %llu %llu %llu, box %u %u %u)",
@@ -157,7 +159,7 @@ int build_kdft_axis(dft3d_plan_s* p, int a, const double* nodes) {
   const unsigned long long dims[3] = {(unsigned long long)(2 * n), (unsigned long long)(2 * n), 2ull};
   const unsigned long long strides[2] = {(unsigned long long)(2 * n * 4), (unsigned long long)(4 * n * n * 4)};
   const unsigned box[3] = {unsigned(dft3d::kBlockK), unsigned(ax.bn), 2u};
-  return encode_f32(&ax.map_w, ax.d_w, 3, dims, strides, box, true);
+  return encode_f32(&ax.map_w, ax.d_w, 3, dims, strides, box, 128);
 }
 
 // One KDFT axis pass over a [batches][J][C] complex view (STRIDED) or rows x J (CONTIG).
@@ -185,7 +187,7 @@ int launch_kdft_strided(dft3d_plan_s* p, int a, const float* in, float* out, lon
   const unsigned long long dims[3] = {(unsigned long long)(2 * C), (unsigned long long)J, (unsigned long long)batches};
   const unsigned long long strides[2] = {(unsigned long long)(C * 8), (unsigned long long)(J * C * 8)};
   const unsigned box[3] = {unsigned(2 * kp.lpb), unsigned(dft3d::kBlockK / 2), unsigned(kp.bpt)};
-  int rc = encode_f32(&map_data, in, 3, dims, strides, box, false);
+  int rc = encode_f32(&map_data, in, 3, dims, strides, box, 0);
   if (rc != DFT3D_OK) return rc;
   const long long total = kp.m_tiles * kp.n_tiles;
   const int grid = int(total < p->sm_count ? total : p->sm_count);
@@ -216,7 +218,7 @@ int launch_kdft_contig(dft3d_plan_s* p, int a, const float* in, float* out, long
   const unsigned long long dims[2] = {(unsigned long long)(2 * J), (unsigned long long)rows};
   const unsigned long long strides[1] = {(unsigned long long)(J * 8)};
   const unsigned box[2] = {unsigned(dft3d::kBlockK), unsigned(dft3d::kTileM)};
-  int rc = encode_f32(&map_data, in, 2, dims, strides, box, true);
+  int rc = encode_f32(&map_data, in, 2, dims, strides, box, 128);
   if (rc != DFT3D_OK) return rc;
   const long long total = kp.m_tiles * kp.n_tiles;
   const int grid = int(total < p->sm_count ? total : p->sm_count);
@@ -269,7 +271,7 @@ int build_fft_axis(dft3d_plan_s* p, int a, const int split[2]) {
   const unsigned long long dims[2] = {32ull, (unsigned long long)(panels * NB)};
   const unsigned long long strides[1] = {128ull};
   const unsigned box[2] = {32u, unsigned(NB)};
-  return encode_f32(&ax.map_w, ax.d_w, 2, dims, strides, box, true);
+  return encode_f32(&ax.map_w, ax.d_w, 2, dims, strides, box, 128);
 }
 
 int fft_axis_pass(dft3d_plan_s* p, int axis, const float* in, float* out, cudaStream_t stream) {
@@ -292,19 +294,19 @@ int fft_axis_pass(dft3d_plan_s* p, int axis, const float* in, float* out, cudaSt
     const unsigned long long dims[3] = {256ull, (unsigned long long)(N / 128), (unsigned long long)rows};
     const unsigned long long strides[2] = {1024ull, (unsigned long long)N * 8ull};
     const unsigned box[3] = {256u, unsigned(N / 128), unsigned(Lg)};
-    rc = encode_f32(&map_data, in, 3, dims, strides, box, false);
+    rc = encode_f32(&map_data, in, 3, dims, strides, box, 0);
   } else {
     const long long batches = (axis == 0) ? 1 : p->n[0];
     const long long C = (axis == 0) ? p->n[1] * p->n[2] : p->n[2];
     fp.C = C;
     fp.c_tiles = C / dft3d::kFftStridedCols;
     fp.mtiles_per_stage = dft3d::kFftStridedCols / Lg;
-    fp.stage_bytes = N * 128;
+    fp.stage_bytes = N * dft3d::kFftStridedCols * 8;
     fp.num_stages = batches * fp.c_tiles;
     const unsigned long long dims[3] = {(unsigned long long)(2 * C), (unsigned long long)N, (unsigned long long)batches};
     const unsigned long long strides[2] = {(unsigned long long)(C * 8), (unsigned long long)N * C * 8ull};
-    const unsigned box[3] = {32u, 256u, 1u};
-    rc = encode_f32(&map_data, in, 3, dims, strides, box, true);
+    const unsigned box[3] = {unsigned(2 * dft3d::kFftStridedCols), 256u, 1u};
+    rc = encode_f32(&map_data, in, 3, dims, strides, box, dft3d::kFftStridedCols * 8);
   }
   if (rc != DFT3D_OK) return rc;
   fp.raw_stages = dft3d::kFftRawBytes / fp.stage_bytes;

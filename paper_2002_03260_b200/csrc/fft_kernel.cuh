@@ -37,7 +37,11 @@ enum : int { FFT_CONTIG = 0, FFT_STRIDED = 1 };
 
 constexpr int kFftThreads = 512;
 constexpr int kFftRawBytes = 128 * 1024;       // ring of raw-data stages
-constexpr int kFftStridedCols = 16;            // lines per STRIDED stage (128-byte rows)
+#ifndef DFT3D_FFT_COLS
+#define DFT3D_FFT_COLS 8
+#endif
+constexpr int kFftStridedCols = DFT3D_FFT_COLS;   // lines per STRIDED stage: 16 (128-byte rows, 128B swizzle) or 8 (64-byte rows, 64B swizzle)
+constexpr int kFftRowBytes = kFftStridedCols * 8;
 constexpr int kFftTmemD1 = 0, kFftTmemD2 = 128, kFftTmemA1 = 256;   // tensor-memory column map (A1: two buffers of 128)
 
 struct FftParams {
@@ -150,7 +154,7 @@ fft_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_const
         } else {
           const long long ct = sidx % p.c_tiles, bt = sidx / p.c_tiles;
           for (int r0 = 0; r0 < p.N; r0 += 256)
-            ptx::tma_load_3d(dst + size_t(r0) * 128, &map_data, &sh.raw_full[s], int(ct * 32), r0, int(bt));
+            ptx::tma_load_3d(dst + size_t(r0) * kFftRowBytes, &map_data, &sh.raw_full[s], int(ct * 2 * kFftStridedCols), r0, int(bt));
         }
       }
     }
@@ -213,8 +217,9 @@ fft_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_const
           stride = uint32_t(R) * 8u;
         } else {
           const int c = mt * Lg + g;                // column within the 16-wide stage
-          base = uint32_t(beta) * 128u + (uint32_t((c >> 1) ^ (beta & 7)) << 4) + uint32_t(c & 1) * 8u;
-          stride = uint32_t(R) * 128u;
+          const uint32_t swz = (kFftStridedCols == 16) ? uint32_t(beta & 7) : uint32_t((beta >> 1) & 3);   // TMA swizzle of row beta
+          base = uint32_t(beta) * kFftRowBytes + ((uint32_t(c >> 1) ^ swz) << 4) + uint32_t(c & 1) * 8u;
+          stride = uint32_t(R) * kFftRowBytes;
         }
         const uint32_t b = uint32_t(t & 1), phb = uint32_t(t >> 1) & 1;
         FFT_WAIT_WARP(&sh.a1_empty[b], phb ^ 1, 0x702);
