@@ -87,9 +87,11 @@ struct KdftAxis {
 
 struct FftAxis {
   long long n = 0;
-  int R = 0;               // n = R*R
+  int R = 0, RX = 1;       // n = RX*R*R, RX = 1 or 2
+  int cols = 16;           // lines per STRIDED stage
   float* d_w = nullptr;    // stacked [W_hi; W_lo] of F_R as 2R/32 panels of [4R rows][32 floats]
   float2* d_tw = nullptr;  // T[k1][beta], R*R complex64
+  float2* d_tw2 = nullptr; // RX == 2: exp(s*2*pi*i*m/n), m < R*R
   CUtensorMap map_w;
 };
 
@@ -125,14 +127,18 @@ int set_kernel_attributes() {
                                   cudaFuncAttributeMaxDynamicSharedMemorySize, int(dft3d::kKdftSmemBytes)));
   DFT3D_CUDA(cudaFuncSetAttribute(dft3d::kdft_axis_kernel<dft3d::KDFT_STRIDED>,
                                   cudaFuncAttributeMaxDynamicSharedMemorySize, int(dft3d::kKdftSmemBytes)));
-  DFT3D_CUDA(cudaFuncSetAttribute(dft3d::fft_axis_kernel<dft3d::FFT_CONTIG, 32>,
-                                  cudaFuncAttributeMaxDynamicSharedMemorySize, int(dft3d::fft_smem_bytes(32))));
-  DFT3D_CUDA(cudaFuncSetAttribute(dft3d::fft_axis_kernel<dft3d::FFT_STRIDED, 32>,
-                                  cudaFuncAttributeMaxDynamicSharedMemorySize, int(dft3d::fft_smem_bytes(32))));
-  DFT3D_CUDA(cudaFuncSetAttribute(dft3d::fft_axis_kernel<dft3d::FFT_CONTIG, 16>,
-                                  cudaFuncAttributeMaxDynamicSharedMemorySize, int(dft3d::fft_smem_bytes(16))));
-  DFT3D_CUDA(cudaFuncSetAttribute(dft3d::fft_axis_kernel<dft3d::FFT_STRIDED, 16>,
-                                  cudaFuncAttributeMaxDynamicSharedMemorySize, int(dft3d::fft_smem_bytes(16))));
+#define DFT3D_FFT_ATTR(MODE, R, RX, COLS)                                                                     \
+  DFT3D_CUDA(cudaFuncSetAttribute(dft3d::fft_axis_kernel<MODE, R, RX, COLS>,                                   \
+                                  cudaFuncAttributeMaxDynamicSharedMemorySize, int(dft3d::fft_smem_bytes(R))))
+  DFT3D_FFT_ATTR(dft3d::FFT_CONTIG, 32, 1, 16);
+  DFT3D_FFT_ATTR(dft3d::FFT_CONTIG, 16, 1, 16);
+  DFT3D_FFT_ATTR(dft3d::FFT_CONTIG, 32, 2, 16);
+  DFT3D_FFT_ATTR(dft3d::FFT_CONTIG, 16, 2, 16);
+  DFT3D_FFT_ATTR(dft3d::FFT_STRIDED, 32, 1, 16);
+  DFT3D_FFT_ATTR(dft3d::FFT_STRIDED, 16, 1, 16);
+  DFT3D_FFT_ATTR(dft3d::FFT_STRIDED, 32, 2, 8);
+  DFT3D_FFT_ATTR(dft3d::FFT_STRIDED, 16, 2, 16);
+#undef DFT3D_FFT_ATTR
   done = true;
   return DFT3D_OK;
 }
@@ -236,20 +242,27 @@ int kdft_axis_pass(dft3d_plan_s* p, int axis, const float* in, float* out, long 
   return launch_kdft_contig(p, 2, in, out, planes * n1, stream);
 }
 
-// FFT formulation, one axis: n = R*R with R = 16 or 32 (Eq. 17 with P = R).  Tables: the real form of F_R
-// split in TF32 pieces and stacked [hi; lo], in the panel layout the kernel's TMA loads expect, and the
-// twiddle factors rounded once to complex64.  The 1/n of a scaled inverse is 1/R in each stage's matrix.
+// FFT formulation, one axis: n = RX*R*R with R = 16 or 32 and RX = 1 or 2 (Eq. 17 with P = R, preceded for
+// RX = 2 by one more application with P = n/2, a radix-2 butterfly).  Tables: the real form of F_R split in TF32
+// pieces and stacked [hi; lo], in the panel layout the kernel's TMA loads expect, and the twiddle factors rounded
+// once to complex64.  The 1/n of a scaled inverse is 1/R in each stage's matrix and 1/RX in the twiddles.
 int build_fft_axis(dft3d_plan_s* p, int a, const int split[2]) {
   FftAxis& ax = p->fax[a];
   const long long n = p->n[a];
-  int R = 0;
-  if (n == 256) R = 16;
-  if (n == 1024) R = 32;
-  if (!R) return fail(DFT3D_ERR_UNSUPPORTED, "FFT mode supports axis lengths 256 (16*16) and 1024 (32*32); n%d = %lld", a, n);
-  if ((split[0] || split[1]) && (split[0] != R || split[1] != R))
-    return fail(DFT3D_ERR_UNSUPPORTED, "FFT split %dx%d for n%d = %lld is not supported (only %dx%d)", split[0], split[1], a, n, R, R);
+  int R = 0, RX = 1;
+  if (n == 256) { R = 16; }
+  if (n == 512) { R = 16; RX = 2; }
+  if (n == 1024) { R = 32; }
+  if (n == 2048) { R = 32; RX = 2; }
+  if (!R)
+    return fail(DFT3D_ERR_UNSUPPORTED, "FFT mode supports axis lengths 256, 512, 1024 and 2048; n%d = %lld", a, n);
+  if ((split[0] || split[1]) && (split[0] != RX * R || split[1] != R))
+    return fail(DFT3D_ERR_UNSUPPORTED, "FFT split %dx%d for n%d = %lld is not supported (only %dx%d)", split[0],
+                split[1], a, n, RX * R, R);
   ax.n = n;
   ax.R = R;
+  ax.RX = RX;
+  ax.cols = (R == 32 && RX == 2) ? 8 : 16;
   const bool scaled = (p->sign > 0) && !(p->flags & DFT3D_UNSCALED_INVERSE);
   const int K = 2 * R, NB = 4 * R, panels = K / 32;
   std::vector<double> M(size_t(2) * R * R), T(size_t(2) * R * R);
@@ -263,11 +276,24 @@ int build_fft_axis(dft3d_plan_s* p, int a, const int split[2]) {
         W[(size_t(pn) * NB + r) * 32 + c] = piece[size_t(r % K) * K + pn * 32 + c];
       }
   dft3d::gen::twiddle(R, R, p->sign, T.data());
-  for (size_t i = 0; i < T.size(); ++i) tw[i] = float(T[i]);
+  const double tscale = scaled ? 1.0 / RX : 1.0;
+  for (size_t i = 0; i < T.size(); ++i) tw[i] = float(T[i] * tscale);
   DFT3D_CUDA(cudaMalloc(&ax.d_w, W.size() * sizeof(float)));
   DFT3D_CUDA(cudaMemcpy(ax.d_w, W.data(), W.size() * sizeof(float), cudaMemcpyHostToDevice));
   DFT3D_CUDA(cudaMalloc(&ax.d_tw, tw.size() * sizeof(float)));
   DFT3D_CUDA(cudaMemcpy(ax.d_tw, tw.data(), tw.size() * sizeof(float), cudaMemcpyHostToDevice));
+  if (RX == 2) {
+    // exp(s*2*pi*i*m/n) for m < R*R: the first column block of the (R*R) x 2 twiddle array
+    std::vector<float> tw2(size_t(2) * R * R);
+    for (long long m = 0; m < (long long)R * R; ++m) {
+      double re, im;
+      dft3d::gen::root_of_unity(m, n, p->sign, &re, &im);
+      tw2[2 * m] = float(re);
+      tw2[2 * m + 1] = float(im);
+    }
+    DFT3D_CUDA(cudaMalloc(&ax.d_tw2, tw2.size() * sizeof(float)));
+    DFT3D_CUDA(cudaMemcpy(ax.d_tw2, tw2.data(), tw2.size() * sizeof(float), cudaMemcpyHostToDevice));
+  }
   const unsigned long long dims[2] = {32ull, (unsigned long long)(panels * NB)};
   const unsigned long long strides[1] = {128ull};
   const unsigned box[2] = {32u, unsigned(NB)};
@@ -276,11 +302,12 @@ int build_fft_axis(dft3d_plan_s* p, int a, const int split[2]) {
 
 int fft_axis_pass(dft3d_plan_s* p, int axis, const float* in, float* out, cudaStream_t stream) {
   const FftAxis& ax = p->fax[axis];
-  const int R = ax.R, N = int(ax.n), Lg = 128 / R;
+  const int R = ax.R, RX = ax.RX, N = int(ax.n), Lg = 128 / (R * RX);
   dft3d::FftParams fp;
   memset(&fp, 0, sizeof(fp));
   fp.N = N;
   fp.twiddle = ax.d_tw;
+  fp.twiddle2 = ax.d_tw2;
   fp.out = out;
   fp.status = p->d_status;
   CUtensorMap map_data;
@@ -299,28 +326,34 @@ int fft_axis_pass(dft3d_plan_s* p, int axis, const float* in, float* out, cudaSt
     const long long batches = (axis == 0) ? 1 : p->n[0];
     const long long C = (axis == 0) ? p->n[1] * p->n[2] : p->n[2];
     fp.C = C;
-    fp.c_tiles = C / dft3d::kFftStridedCols;
-    fp.mtiles_per_stage = dft3d::kFftStridedCols / Lg;
-    fp.stage_bytes = N * dft3d::kFftStridedCols * 8;
+    fp.c_tiles = C / ax.cols;
+    fp.mtiles_per_stage = ax.cols / Lg;
+    fp.stage_bytes = N * ax.cols * 8;
     fp.num_stages = batches * fp.c_tiles;
     const unsigned long long dims[3] = {(unsigned long long)(2 * C), (unsigned long long)N, (unsigned long long)batches};
     const unsigned long long strides[2] = {(unsigned long long)(C * 8), (unsigned long long)N * C * 8ull};
-    const unsigned box[3] = {unsigned(2 * dft3d::kFftStridedCols), 256u, 1u};
-    rc = encode_f32(&map_data, in, 3, dims, strides, box, dft3d::kFftStridedCols * 8);
+    const unsigned box[3] = {unsigned(2 * ax.cols), 256u, 1u};
+    rc = encode_f32(&map_data, in, 3, dims, strides, box, ax.cols * 8);
   }
   if (rc != DFT3D_OK) return rc;
   fp.raw_stages = dft3d::kFftRawBytes / fp.stage_bytes;
   if (fp.raw_stages > 4) fp.raw_stages = 4;
   const int grid = int(fp.num_stages < p->sm_count ? fp.num_stages : p->sm_count);
   const size_t smem = dft3d::fft_smem_bytes(R);
-  if (axis == 2 && R == 32)
-    dft3d::fft_axis_kernel<dft3d::FFT_CONTIG, 32><<<grid, dft3d::kFftThreads, smem, stream>>>(map_data, ax.map_w, fp);
-  else if (axis == 2)
-    dft3d::fft_axis_kernel<dft3d::FFT_CONTIG, 16><<<grid, dft3d::kFftThreads, smem, stream>>>(map_data, ax.map_w, fp);
-  else if (R == 32)
-    dft3d::fft_axis_kernel<dft3d::FFT_STRIDED, 32><<<grid, dft3d::kFftThreads, smem, stream>>>(map_data, ax.map_w, fp);
-  else
-    dft3d::fft_axis_kernel<dft3d::FFT_STRIDED, 16><<<grid, dft3d::kFftThreads, smem, stream>>>(map_data, ax.map_w, fp);
+#define DFT3D_FFT_LAUNCH(MODE, R_, RX_, COLS_)                                                              \
+  dft3d::fft_axis_kernel<MODE, R_, RX_, COLS_><<<grid, dft3d::kFftThreads, smem, stream>>>(map_data, ax.map_w, fp)
+  if (axis == 2) {
+    if (R == 32 && RX == 1) DFT3D_FFT_LAUNCH(dft3d::FFT_CONTIG, 32, 1, 16);
+    else if (R == 16 && RX == 1) DFT3D_FFT_LAUNCH(dft3d::FFT_CONTIG, 16, 1, 16);
+    else if (R == 32) DFT3D_FFT_LAUNCH(dft3d::FFT_CONTIG, 32, 2, 16);
+    else DFT3D_FFT_LAUNCH(dft3d::FFT_CONTIG, 16, 2, 16);
+  } else {
+    if (R == 32 && RX == 1) DFT3D_FFT_LAUNCH(dft3d::FFT_STRIDED, 32, 1, 16);
+    else if (R == 16 && RX == 1) DFT3D_FFT_LAUNCH(dft3d::FFT_STRIDED, 16, 1, 16);
+    else if (R == 32) DFT3D_FFT_LAUNCH(dft3d::FFT_STRIDED, 32, 2, 8);
+    else DFT3D_FFT_LAUNCH(dft3d::FFT_STRIDED, 16, 2, 16);
+  }
+#undef DFT3D_FFT_LAUNCH
   DFT3D_CUDA(cudaGetLastError());
   return DFT3D_OK;
 }
@@ -565,6 +598,7 @@ int dft3d_plan_destroy(dft3d_plan_t p) {
     if (p->kax[a].d_w) cudaFree(p->kax[a].d_w);
     if (p->fax[a].d_w) cudaFree(p->fax[a].d_w);
     if (p->fax[a].d_tw) cudaFree(p->fax[a].d_tw);
+    if (p->fax[a].d_tw2) cudaFree(p->fax[a].d_tw2);
   }
   if (p->workspace) cudaFree(p->workspace);
   if (p->d_status) cudaFree(p->d_status);

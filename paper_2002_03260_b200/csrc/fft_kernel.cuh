@@ -22,6 +22,11 @@
 //   STRIDED (axes 0, 1): a stage holds all N rows of 16 neighbouring lines (128-byte rows, 128B swizzle), i.e.
 //                        R/8 M-tiles; loads and stores touch 128-byte / 32-byte contiguous pieces.
 //
+// Lengths N = 2*R*R (512, 2048) take one more application of Eq. 17 with P = N/2: the split warps first form
+//   a[m] = x[m] + x[m + N/2],   b[m] = (x[m] - x[m + N/2]) * exp(s*2*pi*i*m/N),   m < R*R
+// (a radix-2 butterfly on the CUDA cores), treat a and b as two lines of length R*R, and the final store
+// interleaves them: X[2k] from a, X[2k+1] from b.
+//
 // Warp roles (512 threads): warp 0 TMA producer, warp 1 MMA issuer, warps 4-7 split (smem -> hi/lo -> tensor
 // memory), warps 8-11 drain stage 1 (+twiddle, write stage-2 operand), warps 12-15 drain stage 2 (+store).
 #pragma once
@@ -37,15 +42,11 @@ enum : int { FFT_CONTIG = 0, FFT_STRIDED = 1 };
 
 constexpr int kFftThreads = 512;
 constexpr int kFftRawBytes = 128 * 1024;       // ring of raw-data stages
-#ifndef DFT3D_FFT_COLS
-#define DFT3D_FFT_COLS 8
-#endif
-constexpr int kFftStridedCols = DFT3D_FFT_COLS;   // lines per STRIDED stage: 16 (128-byte rows, 128B swizzle) or 8 (64-byte rows, 64B swizzle)
-constexpr int kFftRowBytes = kFftStridedCols * 8;
+// STRIDED stages hold COLS neighbouring lines: 16 (128-byte rows, 128B swizzle) or 8 (64-byte rows, 64B swizzle)
 constexpr int kFftTmemD1 = 0, kFftTmemD2 = 128, kFftTmemA1 = 256;   // tensor-memory column map (A1: two buffers of 128)
 
 struct FftParams {
-  int N;                 // R*R
+  int N;                 // RX*R*R
   int raw_stages;        // stages in the raw ring
   int stage_bytes;       // bytes of one raw stage
   int mtiles_per_stage;  // CONTIG 1, STRIDED 16/(128/R)
@@ -54,8 +55,9 @@ struct FftParams {
   long long rows;        // number of lines
   // STRIDED: view [batches][N][C] complex
   long long C;
-  long long c_tiles;     // C / 16
-  const float2* twiddle; // [R][R] complex64, T[k1][beta]
+  long long c_tiles;     // C / COLS
+  const float2* twiddle; // [R][R] complex64, T[k1][beta] (times 1/RX for a scaled inverse)
+  const float2* twiddle2;// RX == 2: [R*R] complex64, exp(s*2*pi*i*m/N)
   float* out;
   unsigned int* status;
 };
@@ -91,7 +93,7 @@ __host__ __device__ constexpr size_t fft_smem_bytes(int R) {
     goto role_done;                                                                     \
   }
 
-template <int MODE, int R>
+template <int MODE, int R, int RX, int COLS>
 __global__ void __launch_bounds__(kFftThreads, 1)
 fft_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_constant__ CUtensorMap map_w,
                 const FftParams p) {
@@ -107,7 +109,10 @@ fft_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_const
   FftShared& sh = *reinterpret_cast<FftShared*>(smem_rawring + kFftRawBytes);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  constexpr int Lg = 128 / R;          // lines per M-tile
+  constexpr int SL = 128 / R;          // lines of length R*R per M-tile (sub-lines when RX == 2)
+  constexpr int Lg = SL / RX;          // lines of the cube per M-tile
+  constexpr int NL = R * R;            // length of a (sub-)line
+  constexpr int kRowBytes = COLS * 8;  // STRIDED: bytes of one row of a raw stage
 
   if (tid == 0) {
     for (int i = 0; i < 4; ++i) { ptx::mbar_init(&sh.raw_full[i], 1); ptx::mbar_init(&sh.raw_empty[i], 4 * p.mtiles_per_stage); }
@@ -154,7 +159,7 @@ fft_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_const
         } else {
           const long long ct = sidx % p.c_tiles, bt = sidx / p.c_tiles;
           for (int r0 = 0; r0 < p.N; r0 += 256)
-            ptx::tma_load_3d(dst + size_t(r0) * kFftRowBytes, &map_data, &sh.raw_full[s], int(ct * 2 * kFftStridedCols), r0, int(bt));
+            ptx::tma_load_3d(dst + size_t(r0) * kRowBytes, &map_data, &sh.raw_full[s], int(ct * 2 * COLS), r0, int(bt));
         }
       }
     }
@@ -202,7 +207,8 @@ fft_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_const
     // ------------------------------------------------------------ split: raw lines -> (hi, lo) -> tensor memory A1
     const int q = warp & 3;
     const int m = q * 32 + lane;
-    const int g = m / R, beta = m % R;            // stage-1 lane = (line g, beta), beta fastest
+    const int sl = m / R, beta = m % R;           // stage-1 lane = (sub-line sl, beta), beta fastest
+    const int g = sl / RX, bsel = sl % RX;        // line of the cube within the M-tile; which butterfly output
     const uint32_t lane_addr = tmem + (uint32_t(q * 32) << 16);
     long long t = 0;
     for (long long i = 0; i < my_stages; ++i) {
@@ -210,16 +216,18 @@ fft_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_const
       FFT_WAIT_WARP(&sh.raw_full[s], phs, 0x701);
       const uint8_t* stage = smem_rawring + size_t(s) * p.stage_bytes;
       for (int mt = 0; mt < p.mtiles_per_stage; ++mt, ++t) {
-        // element l of this lane's sub-sequence sits at base + l*stride (bytes)
-        uint32_t base, stride;
+        // element m = R*l + beta of this lane's line sits at base + l*stride; its butterfly partner `half` further
+        uint32_t base, stride, half;
         if (MODE == FFT_CONTIG) {
           base = uint32_t(g * p.N + beta) * 8u;
           stride = uint32_t(R) * 8u;
+          half = uint32_t(NL) * 8u;
         } else {
-          const int c = mt * Lg + g;                // column within the 16-wide stage
-          const uint32_t swz = (kFftStridedCols == 16) ? uint32_t(beta & 7) : uint32_t((beta >> 1) & 3);   // TMA swizzle of row beta
-          base = uint32_t(beta) * kFftRowBytes + ((uint32_t(c >> 1) ^ swz) << 4) + uint32_t(c & 1) * 8u;
-          stride = uint32_t(R) * kFftRowBytes;
+          const int c = mt * Lg + g;                // column within the stage
+          const uint32_t swz = (COLS == 16) ? uint32_t(beta & 7) : uint32_t((beta >> 1) & 3);   // TMA swizzle of the row
+          base = uint32_t(beta) * kRowBytes + ((uint32_t(c >> 1) ^ swz) << 4) + uint32_t(c & 1) * 8u;
+          stride = uint32_t(R) * kRowBytes;
+          half = uint32_t(NL) * kRowBytes;
         }
         const uint32_t b = uint32_t(t & 1), phb = uint32_t(t >> 1) & 1;
         FFT_WAIT_WARP(&sh.a1_empty[b], phb ^ 1, 0x702);
@@ -231,7 +239,20 @@ fft_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_const
 #pragma unroll
           for (int j = 0; j < 16; ++j) {
             const uint2 v = *reinterpret_cast<const uint2*>(stage + base + uint32_t(l0 + j) * stride);
-            x[2 * j] = v.x; x[2 * j + 1] = v.y;
+            if (RX == 1) {
+              x[2 * j] = v.x; x[2 * j + 1] = v.y;
+            } else {
+              const uint2 w = *reinterpret_cast<const uint2*>(stage + base + half + uint32_t(l0 + j) * stride);
+              const float ur = __uint_as_float(v.x), ui = __uint_as_float(v.y);
+              const float vr = __uint_as_float(w.x), vi = __uint_as_float(w.y);
+              if (bsel == 0) {
+                x[2 * j] = __float_as_uint(ur + vr); x[2 * j + 1] = __float_as_uint(ui + vi);
+              } else {
+                const float2 tw = __ldg(p.twiddle2 + (l0 + j) * R + beta);
+                const float dr = ur - vr, di = ui - vi;
+                x[2 * j] = __float_as_uint(dr * tw.x - di * tw.y); x[2 * j + 1] = __float_as_uint(dr * tw.y + di * tw.x);
+              }
+            }
           }
 #pragma unroll
           for (int j = 0; j < 32; ++j) {
@@ -256,11 +277,11 @@ fft_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_const
     // ------------------------------------------------------------ drain stage 1: sum halves, twiddle, split, write A2
     const int q = warp & 3;
     const int m = q * 32 + lane;
-    const int g = m / R, beta = m % R;
+    const int sl = m / R, beta = m % R;
     const uint32_t lane_addr = tmem + (uint32_t(q * 32) << 16) + kFftTmemD1;
-    // A2 row of (g, k1): CONTIG g*R + k1 ; STRIDED k1*Lg + g (so that stage-2 stores of one k2 touch neighbouring lines)
-    const int row_mul_k1 = (MODE == FFT_CONTIG) ? 1 : Lg;
-    const int row_base = (MODE == FFT_CONTIG) ? g * R : g;
+    // A2 row of (sl, k1): CONTIG sl*R + k1 ; STRIDED k1*SL + sl (so that stage-2 stores of one k2 touch neighbouring lines)
+    const int row_mul_k1 = (MODE == FFT_CONTIG) ? 1 : SL;
+    const int row_base = (MODE == FFT_CONTIG) ? sl * R : sl;
     // K column (beta, q) -> panel beta/16, 16-byte chunk (beta%16)/2, half beta%2
     const uint32_t a2_col = uint32_t(beta >> 4) * (128u * 128u) + uint32_t(beta & 1) * 8u;
     const uint32_t a2_chunk = uint32_t(beta & 15) >> 1;
@@ -312,27 +333,27 @@ fft_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_const
     // ------------------------------------------------------------ drain stage 2: sum halves, store in natural order
     const int q = warp & 3;
     const int m = q * 32 + lane;
-    const int g = (MODE == FFT_CONTIG) ? m / R : m % Lg;
-    const int k1 = (MODE == FFT_CONTIG) ? m % R : m / Lg;
+    const int sl = (MODE == FFT_CONTIG) ? m / R : m % SL;
+    const int k1 = (MODE == FFT_CONTIG) ? m % R : m / SL;
+    const int g = sl / RX, bsel = sl % RX;
     const uint32_t lane_addr = tmem + (uint32_t(q * 32) << 16) + kFftTmemD2;
     long long t = 0;
-    long long i = 0;
-    for (long long sidx = blockIdx.x; sidx < p.num_stages; sidx += gridDim.x, ++i) {
+    for (long long sidx = blockIdx.x; sidx < p.num_stages; sidx += gridDim.x) {
       for (int mt = 0; mt < p.mtiles_per_stage; ++mt, ++t) {
-        float2* dst;              // &out[line][k1], element k2 at dst + k2*k2_stride
+        float2* dst;              // &out[line][RX*k1 + bsel]; output k = RX*(k1 + R*k2) + bsel is k2*k2_stride further
         long long k2_stride;
         bool ok;
         if (MODE == FFT_CONTIG) {
           const long long line = sidx * Lg + g;
           ok = line < p.rows;
-          dst = reinterpret_cast<float2*>(p.out) + line * p.N + k1;
-          k2_stride = R;
+          dst = reinterpret_cast<float2*>(p.out) + line * p.N + (RX * k1 + bsel);
+          k2_stride = RX * R;
         } else {
           const long long ct = sidx % p.c_tiles, bt = sidx / p.c_tiles;
-          const long long col = ct * kFftStridedCols + mt * Lg + g;
+          const long long col = ct * COLS + mt * Lg + g;
           ok = col < p.C;
-          dst = reinterpret_cast<float2*>(p.out) + (bt * p.N + k1) * p.C + col;
-          k2_stride = (long long)R * p.C;
+          dst = reinterpret_cast<float2*>(p.out) + (bt * p.N + (RX * k1 + bsel)) * p.C + col;
+          k2_stride = (long long)(RX * R) * p.C;
         }
         FFT_WAIT_WARP(&sh.d2_full, uint32_t(t) & 1, 0x901);
         ptx::tc_fence_after();

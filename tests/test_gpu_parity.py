@@ -231,8 +231,45 @@ def test_fft_mixed_axis_lengths(lib, oracle):
         lib.Plan(*shape, mode=lib.DFT3D_FFT, fft_split=((32, 8), None, None))
     assert e.value.status == 2
     with pytest.raises(lib.Dft3dError) as e:
-        lib.Plan(512, 256, 256, mode=lib.DFT3D_FFT)
+        lib.Plan(768, 256, 256, mode=lib.DFT3D_FFT)
     assert e.value.status == 2
+
+
+@pytest.mark.parametrize("shape,axis", [((256, 256, 512), 2), ((256, 512, 256), 1), ((512, 256, 256), 0),
+                                        ((256, 256, 2048), 2), ((256, 2048, 256), 1), ((2048, 256, 256), 0)])
+def test_fft_radix2_lengths_single_axis(lib, oracle, shape, axis):
+    """N = 2*R*R (512 = 2*16*16, 2048 = 2*32*32): butterfly + two GEMM stages.  The oracle transforms a slab of
+    8 lines-worth along an untransformed axis (lines are independent), which keeps the 2048 cases short."""
+    x = _inputs().cube(shape, "normal", 64 + axis, device="cuda")
+    plan = lib.Plan(*shape, mode=lib.DFT3D_FFT)
+    y = plan.execute_axis(axis, x)
+    _finish(plan)
+    plan.destroy()
+    sl = (slice(None), slice(0, 8), slice(None)) if axis == 0 else (slice(0, 8), slice(None), slice(None))
+    ref = oracle.dft_axis(x[sl].cpu().numpy().astype(np.complex128), axis)
+    err = oracle.rel_l2(y[sl].cpu().numpy(), ref)
+    assert err < SANITY_AXIS, (shape, axis, err)
+    # the rest of the output against the (oracle-checked) KDFT kernel of the same axis
+    kdft = lib.Plan(*shape, mode=lib.DFT3D_KDFT)
+    z = kdft.execute_axis(axis, x)
+    _finish(kdft)
+    kdft.destroy()
+    assert _rel_l2_gpu(y, z) < TOL
+
+
+def test_fft_512_cube_forward_inverse(lib, oracle):
+    shape = (512, 256, 512)
+    x = _inputs().cube(shape, "uniform", 65, device="cuda")
+    fwd = lib.Plan(*shape, mode=lib.DFT3D_FFT)
+    inv = lib.Plan(*shape, mode=lib.DFT3D_FFT, sign=lib.DFT3D_INVERSE)
+    y = fwd(x)
+    back = inv(y)
+    _finish(inv)
+    fwd.status()
+    assert oracle.rel_l2(y.cpu().numpy(), oracle.dft3d(x.cpu().numpy())) < SANITY
+    assert oracle.rel_l2(back.cpu().numpy(), x.cpu().numpy()) < SANITY
+    fwd.destroy()
+    inv.destroy()
 
 
 # ------------------------------------------------------------------ config 3: 1024^3, FFT (32*32) against KDFT and the oracle
