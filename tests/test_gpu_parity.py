@@ -329,3 +329,80 @@ def test_config3_fft_1024_vs_kdft_and_oracle_subset(lib, oracle):
         assert abs(want - ref[pos]) < 1e-9 * rms, (k, want, ref[pos])
         got = complex(y[k].item())
         assert abs(got - want) < 5e-5 * rms, (k, got, want, abs(got - want) / rms)
+
+
+# ------------------------------------------------------------------ config 5: 2048^3 (64 GiB in, 64 GiB out), both formulations
+
+@pytest.mark.slow
+def test_config5_2048_exponentials_both_modes(lib, oracle):
+    """Largest single-GPU instance.  Input: 16 unit exponentials (distinct integer frequencies, seeded phases)
+    plus N(0, sigma = 1e-3) noise, so the spectrum is 16 peaks of magnitude P over a floor of about sigma*sqrt(2P).
+    Only two 64 GiB tensors fit, so FFT and KDFT run one after the other into the same output and are compared
+    on sampled planes; each is compared with the float64 oracle on a product grid of coefficients that contains
+    all peaks.  Gate: the norm-wise relative L2 error of the whole output, estimated from the subset by strata.
+    A coefficient's error level depends on how many of its three indices coincide with a peak's index on that axis
+    (it then lies on a line or plane that carried a peak through one or two of the axis passes), and the product
+    grid over-represents those; so the samples are grouped by that count c = 0..3, each group's mean |d|^2 is scaled
+    to the group's true population N_c, and rel^2 = sum_c N_c * mean_c |d|^2 / (P * sum|x|^2) <= 1e-10 (the
+    denominator is the output energy by Parseval).  Also: every peak within 1e-5 relative, Parseval to 1e-5.
+    """
+    free, total = torch.cuda.mem_get_info()
+    if total < 170 * 2 ** 30:
+        pytest.skip("needs a 180 GB device")
+    n = 2048
+    shape = (n, n, n)
+    P = float(n) ** 3
+    inp = _inputs()
+    x, freqs, phases = inp.exponentials(shape, 16, 2005, 1e-3, 1005, device="cuda")
+    ex = sum(float((torch.view_as_real(x[i]).double() ** 2).sum()) for i in range(n))
+    S = [inp.stratified_indices(n, 16, 5005 + a, forced=freqs[:, a]) for a in range(3)]
+    sub = oracle.Subset(shape, S[0], S[1], S[2])
+    for a in range(0, n, 32):
+        sub.feed(x[a:a + 32].cpu().numpy())
+    ref = sub.result()
+    pos = [{int(v): i for i, v in enumerate(S[a])} for a in range(3)]
+    peak_pos = [tuple(pos[a][int(f[a])] for a in range(3)) for f in freqs]
+    # closed form of the peaks: P * exp(i phi) up to the noise term (a few sigma*sqrt(2P) = 130)
+    for e, pp in enumerate(peak_pos):
+        assert abs(ref[pp] - P * np.exp(1j * phases[e])) < 2000.0
+    # strata: number of axes on which the sample's index is some peak's index; exact population of each stratum
+    F = [np.unique(freqs[:, a]) for a in range(3)]
+    on = [np.isin(S[a], F[a]) for a in range(3)]
+    count = on[0][:, None, None].astype(int) + on[1][None, :, None] + on[2][None, None, :]
+    u = [len(f) for f in F]
+    pop = [float((n - u[0]) * (n - u[1]) * (n - u[2])),
+           float(u[0] * (n - u[1]) * (n - u[2]) + (n - u[0]) * u[1] * (n - u[2]) + (n - u[0]) * (n - u[1]) * u[2]),
+           float(u[0] * u[1] * (n - u[2]) + u[0] * (n - u[1]) * u[2] + (n - u[0]) * u[1] * u[2]),
+           float(u[0] * u[1] * u[2])]
+    assert abs(sum(pop) - P) < 1.0 and all((count == c).sum() > 0 for c in range(4))
+    assert (count == 3).sum() == pop[3]          # the grid holds every point of the innermost stratum
+    idx = [torch.as_tensor(s, device="cuda") for s in S]
+    planes = [torch.as_tensor(inp.stratified_indices(n, 16, 6005 + a), device="cuda") for a in range(3)]
+    out = torch.empty_like(x)
+    kept = None
+    for mode in (lib.DFT3D_FFT, lib.DFT3D_KDFT):
+        plan = lib.Plan(*shape, mode=mode, workspace_limit=4 * 2 ** 30)
+        plan(x, out)
+        _finish(plan)
+        plan.destroy()
+        got = out[idx[0]][:, idx[1]][:, :, idx[2]].cpu().numpy()
+        d2 = np.abs(got - ref) ** 2
+        strata = [pop[c] * d2[count == c].mean() for c in range(4)]
+        est = sum(strata) / (P * ex)
+        assert est < TOL ** 2, (mode, np.sqrt(est), [np.sqrt(v / (P * ex)) for v in strata])
+        for pp in peak_pos:
+            assert abs(got[pp] - ref[pp]) < TOL * abs(ref[pp]), (mode, pp, got[pp], ref[pp])
+        ey = sum(float((torch.view_as_real(out[i]).double() ** 2).sum()) for i in range(n))
+        assert abs(ey / (P * ex) - 1.0) < TOL, (mode, ey / (P * ex))
+        sampled = [out[planes[0]].clone(), out[:, planes[1]].clone(), out[:, :, planes[2]].clone()]
+        if kept is None:
+            kept = sampled
+        else:
+            for a, b in zip(sampled, kept):      # KDFT against FFT on planes that cross every output tile
+                num = float(((a.to(torch.complex128) - b.to(torch.complex128)).abs() ** 2).sum())
+                den = float((b.to(torch.complex128).abs() ** 2).sum())
+                # planes that miss the peaks hold only the noise floor, which fp32 accumulation cannot resolve to
+                # 1e-5 of itself; the error is measured against the mean |X|^2 of the full spectrum, which by
+                # Parseval is sum|x|^2
+                assert num / a.numel() < (TOL ** 2) * ex, (num / a.numel(), den / a.numel(), ex)
+    del kept
