@@ -89,7 +89,7 @@ struct FftAxis {
   long long n = 0;
   int R = 0, RX = 1;       // n = RX*R*R, RX = 1 or 2
   int cols = 16;           // lines per STRIDED stage
-  float* d_w = nullptr;    // stacked [W_hi; W_lo] of F_R as 2R/32 panels of [4R rows][32 floats]
+  float* d_w = nullptr;    // real form of F_R: [piece hi|lo][2R/32 panels][2R rows][32 floats]
   float2* d_tw = nullptr;  // T[k1][beta], R*R complex64
   float2* d_tw2 = nullptr; // RX == 2: exp(s*2*pi*i*m/n), m < R*R
   CUtensorMap map_w;
@@ -264,17 +264,16 @@ int build_fft_axis(dft3d_plan_s* p, int a, const int split[2]) {
   ax.RX = RX;
   ax.cols = (R == 32 && RX == 2) ? 8 : 16;
   const bool scaled = (p->sign > 0) && !(p->flags & DFT3D_UNSCALED_INVERSE);
-  const int K = 2 * R, NB = 4 * R, panels = K / 32;
+  const int K = 2 * R, NB = 2 * R, panels = K / 32;
   std::vector<double> M(size_t(2) * R * R), T(size_t(2) * R * R);
-  std::vector<float> hi(size_t(K) * K), lo(size_t(K) * K), W(size_t(panels) * NB * 32), tw(size_t(2) * R * R);
+  std::vector<float> hi(size_t(K) * K), lo(size_t(K) * K), W(size_t(2) * panels * NB * 32), tw(size_t(2) * R * R);
   dft3d::gen::axis_matrix(R, p->sign, scaled ? 1.0 / R : 1.0, nullptr, false, M.data());
   dft3d::gen::real_table_from_matrix(R, M.data(), hi.data(), lo.data());
-  for (int pn = 0; pn < panels; ++pn)
-    for (int r = 0; r < NB; ++r)
-      for (int c = 0; c < 32; ++c) {
-        const std::vector<float>& piece = (r < K) ? hi : lo;
-        W[(size_t(pn) * NB + r) * 32 + c] = piece[size_t(r % K) * K + pn * 32 + c];
-      }
+  for (int pc = 0; pc < 2; ++pc)            // layout [piece][panel][2R rows][32 floats]
+    for (int pn = 0; pn < panels; ++pn)
+      for (int r = 0; r < NB; ++r)
+        for (int c = 0; c < 32; ++c)
+          W[((size_t(pc) * panels + pn) * NB + r) * 32 + c] = (pc ? lo : hi)[size_t(r) * K + pn * 32 + c];
   dft3d::gen::twiddle(R, R, p->sign, T.data());
   const double tscale = scaled ? 1.0 / RX : 1.0;
   for (size_t i = 0; i < T.size(); ++i) tw[i] = float(T[i] * tscale);
@@ -294,7 +293,7 @@ int build_fft_axis(dft3d_plan_s* p, int a, const int split[2]) {
     DFT3D_CUDA(cudaMalloc(&ax.d_tw2, tw2.size() * sizeof(float)));
     DFT3D_CUDA(cudaMemcpy(ax.d_tw2, tw2.data(), tw2.size() * sizeof(float), cudaMemcpyHostToDevice));
   }
-  const unsigned long long dims[2] = {32ull, (unsigned long long)(panels * NB)};
+  const unsigned long long dims[2] = {32ull, (unsigned long long)(2 * panels * NB)};
   const unsigned long long strides[1] = {128ull};
   const unsigned box[2] = {32u, unsigned(NB)};
   return encode_f32(&ax.map_w, ax.d_w, 2, dims, strides, box, 128);
@@ -308,6 +307,7 @@ int fft_axis_pass(dft3d_plan_s* p, int axis, const float* in, float* out, cudaSt
   fp.N = N;
   fp.twiddle = ax.d_tw;
   fp.twiddle2 = ax.d_tw2;
+  fp.profile = p->d_profile;
   fp.out = out;
   fp.status = p->d_status;
   CUtensorMap map_data;
@@ -391,7 +391,7 @@ const char* dft3d_last_error(void) { return g_last_error; }
 #ifdef DFT3D_PROFILE_WAITS
 // diagnostic builds only: copies the MMA issuer's cycle counters [grid][4] = {total, wait acc, wait W, wait data}
 int dft3d_debug_read_profile(dft3d_plan_t p, long long* host, int ctas) {
-  return cudaMemcpy(host, p->d_profile, sizeof(long long) * 4 * ctas, cudaMemcpyDeviceToHost) == cudaSuccess ? 0 : 4;
+  return cudaMemcpy(host, p->d_profile, sizeof(long long) * ctas, cudaMemcpyDeviceToHost) == cudaSuccess ? 0 : 4;
 }
 #endif
 
@@ -485,7 +485,8 @@ int dft3d_plan_create_ex(dft3d_plan_t* out, long long n0, long long n1, long lon
     if (e == cudaSuccess) e = cudaMemset(p->d_status, 0, sizeof(unsigned int));
     if (e != cudaSuccess) { rc = fail(DFT3D_ERR_ALLOC, "cudaMalloc(status): %s", cudaGetErrorString(e)); break; }
 #ifdef DFT3D_PROFILE_WAITS
-    e = cudaMalloc(&p->d_profile, sizeof(long long) * 4 * 1024);
+    e = cudaMalloc(&p->d_profile, sizeof(long long) * 128 * 256);
+    if (e == cudaSuccess) e = cudaMemset(p->d_profile, 0, sizeof(long long) * 128 * 256);
     if (e != cudaSuccess) { rc = fail(DFT3D_ERR_ALLOC, "cudaMalloc(profile)"); break; }
 #endif
     if (mode == DFT3D_KDFT) {

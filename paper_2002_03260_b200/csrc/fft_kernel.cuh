@@ -10,10 +10,9 @@
 // directly in the operand layout stage 2's MMA reads.  HBM traffic is one read and one write of the data.
 //
 // Both stages use the same complex-as-real mapping as the KDFT kernel (interleaved re/im, real 2R x 2R
-// matrix W).  fp32 accuracy from TF32: the data is split x = hi + lo (two MMAs per K step) and the two
-// table pieces are stacked along N, B = [W_hi ; W_lo] (4R rows), so that the accumulator's column halves
-// hold x*W_hi and x*W_lo; the halves are added when the accumulator is drained.  A chain is at most 16 MMAs
-// long, so the truncation bias of the tensor-core accumulator stays far below fp32 rounding.
+// matrix W).  fp32 accuracy from TF32 as in the KDFT kernel: x = hi + lo, W = W_hi + W_lo and three MMAs per
+// K step (hi*hi, lo*hi, hi*lo) into one 2R-column accumulator.  A chain is at most 24 MMAs long, so the
+// truncation bias of the tensor-core accumulator stays far below fp32 rounding.
 //
 // Tile geometry.  An "M-tile" is 128 accumulator lanes.
 //   stage 1 lanes = (line g, beta)  : 128/R lines of the tile, all beta
@@ -27,8 +26,9 @@
 // (a radix-2 butterfly on the CUDA cores), treat a and b as two lines of length R*R, and the final store
 // interleaves them: X[2k] from a, X[2k+1] from b.
 //
-// Warp roles (512 threads): warp 0 TMA producer, warp 1 MMA issuer, warps 4-7 split (smem -> hi/lo -> tensor
-// memory), warps 8-11 drain stage 1 (+twiddle, write stage-2 operand), warps 12-15 drain stage 2 (+store).
+// Warp roles (512 threads): warp 0 TMA producer, warps 1 and 2 MMA issuers (stage 1, stage 2), warps 4-7 split (smem -> hi/lo -> tensor
+// memory), warps 8-15 drain stage 1 (+twiddle, write stage-2 operand; two groups, 16 values of k1 each),
+// warps 16-19 drain stage 2 (+store).
 #pragma once
 #include <cstdint>
 #include <cuda.h>
@@ -40,7 +40,7 @@ namespace dft3d {
 
 enum : int { FFT_CONTIG = 0, FFT_STRIDED = 1 };
 
-constexpr int kFftThreads = 512;
+constexpr int kFftThreads = 640;      // 5 warp groups: {producer, 2 MMA issuers}, split, drain 1 (x2), drain 2
 constexpr int kFftRawBytes = 128 * 1024;       // ring of raw-data stages
 // STRIDED stages hold COLS neighbouring lines: 16 (128-byte rows, 128B swizzle) or 8 (64-byte rows, 64B swizzle)
 constexpr int kFftTmemD1 = 0, kFftTmemD2 = 128, kFftTmemA1 = 256;   // tensor-memory column map (A1: two buffers of 128)
@@ -60,6 +60,7 @@ struct FftParams {
   const float2* twiddle2;// RX == 2: [R*R] complex64, exp(s*2*pi*i*m/N)
   float* out;
   unsigned int* status;
+  long long* profile;    // optional cycle counters (builds with DFT3D_PROFILE_WAITS): [grid][16][8]
 };
 
 struct FftShared {
@@ -73,24 +74,39 @@ struct FftShared {
   volatile int abort_flag;
 };
 
-// shared memory: [W: 4R rows x 2R floats, as 2R/32 panels of 4R x 128 B] [A2: hi panels, lo panels] [raw ring] [barriers]
+// shared memory: [W: 2 pieces x 2R/32 panels of 2R rows x 128 B] [A2: hi panels, lo panels] [raw ring] [barriers]
 __host__ __device__ constexpr int fft_w_bytes(int R) { return (2 * R / 32) * 4 * R * 128; }
 __host__ __device__ constexpr int fft_a2_piece_bytes(int R) { return (2 * R / 32) * 128 * 128; }
 __host__ __device__ constexpr size_t fft_smem_bytes(int R) {
   return size_t(fft_w_bytes(R)) + 2 * size_t(fft_a2_piece_bytes(R)) + kFftRawBytes + 1024 + 512;
 }
 
+#ifdef DFT3D_PROFILE_WAITS
+#define FFT_PROF_BEGIN const long long prof_t0_ = clock64();
+#define FFT_PROF_END(code) prof_wait[(code) >> 8] [(code) & 7] += clock64() - prof_t0_;
+#else
+#define FFT_PROF_BEGIN
+#define FFT_PROF_END(code)
+#endif
 #define FFT_WAIT(bar, parity, code)                                 \
-  if (!bounded_wait((bar), (parity), &sh.abort_flag)) {             \
-    sh.abort_flag = 1;                                              \
-    atomicCAS(p.status, 0u, (unsigned)(code));                      \
-    goto role_done;                                                 \
+  {                                                                 \
+    FFT_PROF_BEGIN                                                  \
+    if (!bounded_wait((bar), (parity), &sh.abort_flag)) {           \
+      sh.abort_flag = 1;                                            \
+      atomicCAS(p.status, 0u, (unsigned)(code));                    \
+      goto role_done;                                               \
+    }                                                               \
+    FFT_PROF_END(code)                                              \
   }
-#define FFT_WAIT_WARP(bar, parity, code)                                                \
-  if (!__all_sync(0xffffffffu, bounded_wait((bar), (parity), &sh.abort_flag) ? 1 : 0)) { \
-    sh.abort_flag = 1;                                                                  \
-    atomicCAS(p.status, 0u, (unsigned)(code));                                          \
-    goto role_done;                                                                     \
+#define FFT_WAIT_WARP(bar, parity, code)                                                  \
+  {                                                                                       \
+    FFT_PROF_BEGIN                                                                        \
+    if (!__all_sync(0xffffffffu, bounded_wait((bar), (parity), &sh.abort_flag) ? 1 : 0)) { \
+      sh.abort_flag = 1;                                                                  \
+      atomicCAS(p.status, 0u, (unsigned)(code));                                          \
+      goto role_done;                                                                     \
+    }                                                                                     \
+    FFT_PROF_END(code)                                                                    \
   }
 
 template <int MODE, int R, int RX, int COLS>
@@ -100,7 +116,8 @@ fft_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_const
   extern __shared__ uint8_t smem_raw_[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw_) + 1023) & ~uintptr_t(1023));
   constexpr int K = 2 * R;             // reals per contraction
-  constexpr int NB = 4 * R;            // MMA N: stacked [W_hi; W_lo]
+  constexpr int NB = 2 * R;            // MMA N: the 2R output reals (k, re/im) of one stage
+  constexpr int kWPiece = (K / 32) * NB * 128;   // bytes of one table piece in shared memory
   constexpr int panels = K / 32;
   uint8_t* smem_w = smem;
   uint8_t* smem_a2 = smem_w + fft_w_bytes(R);
@@ -109,6 +126,11 @@ fft_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_const
   FftShared& sh = *reinterpret_cast<FftShared*>(smem_rawring + kFftRawBytes);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+#ifdef DFT3D_PROFILE_WAITS
+  long long prof_wait[16][8];
+  for (int i = 0; i < 16; ++i) for (int j = 0; j < 8; ++j) prof_wait[i][j] = 0;
+  const long long prof_start = clock64();
+#endif
   constexpr int SL = 128 / R;          // lines of length R*R per M-tile (sub-lines when RX == 2)
   constexpr int Lg = SL / RX;          // lines of the cube per M-tile
   constexpr int NL = R * R;            // length of a (sub-)line
@@ -117,8 +139,8 @@ fft_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_const
   if (tid == 0) {
     for (int i = 0; i < 4; ++i) { ptx::mbar_init(&sh.raw_full[i], 1); ptx::mbar_init(&sh.raw_empty[i], 4 * p.mtiles_per_stage); }
     for (int i = 0; i < 2; ++i) { ptx::mbar_init(&sh.a1_full[i], 4); ptx::mbar_init(&sh.a1_empty[i], 1); }
-    ptx::mbar_init(&sh.d1_full, 1); ptx::mbar_init(&sh.d1_empty, 4);
-    ptx::mbar_init(&sh.a2_full, 4); ptx::mbar_init(&sh.a2_empty, 1);
+    ptx::mbar_init(&sh.d1_full, 1); ptx::mbar_init(&sh.d1_empty, 4 * (K / 32));
+    ptx::mbar_init(&sh.a2_full, 4 * (K / 32)); ptx::mbar_init(&sh.a2_empty, 1);
     ptx::mbar_init(&sh.d2_full, 1); ptx::mbar_init(&sh.d2_empty, 4);
     ptx::mbar_init(&sh.w_full, 1);
     sh.abort_flag = 0;
@@ -142,11 +164,13 @@ fft_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_const
   if ((long long)blockIdx.x < p.num_stages) my_stages = (p.num_stages - 1 - blockIdx.x) / gridDim.x + 1;
   const long long my_mtiles = my_stages * p.mtiles_per_stage;
 
+  // 640 threads x 96 registers: every role fits its share, so the register file is not re-split here
+
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
     if (lane == 0) {
       ptx::mbar_arrive_expect_tx(&sh.w_full, uint32_t(fft_w_bytes(R)));
-      for (int pn = 0; pn < panels; ++pn)
+      for (int pn = 0; pn < 2 * panels; ++pn)       // [piece][panel][2R rows][32 floats]
         ptx::tma_load_2d(smem_w + pn * NB * 128, &map_w, &sh.w_full, 0, pn * NB);
       long long i = 0;
       for (long long sidx = blockIdx.x; sidx < p.num_stages; sidx += gridDim.x, ++i) {
@@ -164,43 +188,70 @@ fft_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_const
       }
     }
   } else if (warp == 1) {
-    // ------------------------------------------------------------ MMA issuer (stage 1 of M-tile t, then stage 2 of t-1)
+    // ------------------------------------------------------------ MMA issuer, stage 1 (A from tensor memory)
+    // Two issuing threads (this one and warp 2 for stage 2) keep the tensor pipe fed: every operand of the
+    // unrolled MMAs below is loop-invariant (the two A1 buffers alternate, hence the unroll by two), so the
+    // issue loop is a handful of instructions per MMA.
+    if (lane == 0) {
+      const uint32_t idesc = ptx::make_idesc_tf32(128, NB);
+      const uint32_t w_addr = ptx::smem_u32(smem_w);
+      uint64_t wh[K / 8], wl[K / 8];                 // loop-invariant operand descriptors, kept in registers
+#pragma unroll
+      for (int k8 = 0; k8 < K / 8; ++k8) {
+        wh[k8] = ptx::make_kmajor_sw128_desc(w_addr + (k8 >> 2) * NB * 128 + (k8 & 3) * 32);
+        wl[k8] = ptx::make_kmajor_sw128_desc(w_addr + kWPiece + (k8 >> 2) * NB * 128 + (k8 & 3) * 32);
+      }
+      FFT_WAIT(&sh.w_full, 0, 0x601);
+      for (long long t = 0; t < my_mtiles; t += 2) {
+#pragma unroll
+        for (int b = 0; b < 2; ++b) {
+          if (t + b < my_mtiles) {
+            const uint32_t phb = uint32_t(t >> 1) & 1;
+            FFT_WAIT(&sh.a1_full[b], phb, 0x602);
+            FFT_WAIT(&sh.d1_empty, uint32_t(b) ^ 1, 0x603);
+            ptx::tc_fence_after();
+            const uint32_t a_hi = tmem + kFftTmemA1 + b * 128, a_lo = a_hi + K;
+#pragma unroll
+            for (int k8 = 0; k8 < K / 8; ++k8) {
+              ptx::mma_tf32_ts(tmem + kFftTmemD1, a_hi + k8 * 8, wh[k8], idesc, k8 != 0);
+              ptx::mma_tf32_ts(tmem + kFftTmemD1, a_lo + k8 * 8, wh[k8], idesc, 1);
+              ptx::mma_tf32_ts(tmem + kFftTmemD1, a_hi + k8 * 8, wl[k8], idesc, 1);
+            }
+            ptx::tc_commit(&sh.a1_empty[b]);
+            ptx::tc_commit(&sh.d1_full);
+          }
+        }
+      }
+    }
+  } else if (warp == 2) {
+    // ------------------------------------------------------------ MMA issuer, stage 2 (A from shared memory)
     if (lane == 0) {
       const uint32_t idesc = ptx::make_idesc_tf32(128, NB);
       const uint32_t w_addr = ptx::smem_u32(smem_w);
       const uint32_t a2_addr = ptx::smem_u32(smem_a2);
-      FFT_WAIT(&sh.w_full, 0, 0x601);
-      for (long long t = 0; t <= my_mtiles; ++t) {
-        if (t < my_mtiles) {
-          const uint32_t b = uint32_t(t & 1), phb = uint32_t(t >> 1) & 1;
-          FFT_WAIT(&sh.a1_full[b], phb, 0x602);
-          FFT_WAIT(&sh.d1_empty, (uint32_t(t) & 1) ^ 1, 0x603);
-          ptx::tc_fence_after();
-          const uint32_t a_hi = tmem + kFftTmemA1 + b * 128, a_lo = a_hi + K;
+      uint64_t wh[K / 8], wl[K / 8], ah[K / 8], al[K / 8];
 #pragma unroll
-          for (int k8 = 0; k8 < K / 8; ++k8) {
-            const uint64_t wd = ptx::make_kmajor_sw128_desc(w_addr + (k8 >> 2) * NB * 128 + (k8 & 3) * 32);
-            ptx::mma_tf32_ts(tmem + kFftTmemD1, a_hi + k8 * 8, wd, idesc, k8 != 0);
-            ptx::mma_tf32_ts(tmem + kFftTmemD1, a_lo + k8 * 8, wd, idesc, 1);
-          }
-          ptx::tc_commit(&sh.a1_empty[b]);
-          ptx::tc_commit(&sh.d1_full);
-        }
-        if (t >= 1) {
-          const uint32_t u = uint32_t(t - 1);
-          FFT_WAIT(&sh.a2_full, u & 1, 0x604);
-          FFT_WAIT(&sh.d2_empty, (u & 1) ^ 1, 0x605);
-          ptx::tc_fence_after();
+      for (int k8 = 0; k8 < K / 8; ++k8) {
+        const uint32_t off = (k8 >> 2) * 128 * 128 + (k8 & 3) * 32;
+        wh[k8] = ptx::make_kmajor_sw128_desc(w_addr + (k8 >> 2) * NB * 128 + (k8 & 3) * 32);
+        wl[k8] = ptx::make_kmajor_sw128_desc(w_addr + kWPiece + (k8 >> 2) * NB * 128 + (k8 & 3) * 32);
+        ah[k8] = ptx::make_kmajor_sw128_desc(a2_addr + off);
+        al[k8] = ptx::make_kmajor_sw128_desc(a2_addr + a2_piece + off);
+      }
+      FFT_WAIT(&sh.w_full, 0, 0x611);
+      for (long long t = 0; t < my_mtiles; ++t) {
+        const uint32_t u = uint32_t(t);
+        FFT_WAIT(&sh.a2_full, u & 1, 0x604);
+        FFT_WAIT(&sh.d2_empty, (u & 1) ^ 1, 0x605);
+        ptx::tc_fence_after();
 #pragma unroll
-          for (int k8 = 0; k8 < K / 8; ++k8) {
-            const uint32_t off = (k8 >> 2) * 128 * 128 + (k8 & 3) * 32;
-            const uint64_t wd = ptx::make_kmajor_sw128_desc(w_addr + (k8 >> 2) * NB * 128 + (k8 & 3) * 32);
-            ptx::mma_tf32_ss(tmem + kFftTmemD2, ptx::make_kmajor_sw128_desc(a2_addr + off), wd, idesc, k8 != 0);
-            ptx::mma_tf32_ss(tmem + kFftTmemD2, ptx::make_kmajor_sw128_desc(a2_addr + a2_piece + off), wd, idesc, 1);
-          }
-          ptx::tc_commit(&sh.a2_empty);
-          ptx::tc_commit(&sh.d2_full);
+        for (int k8 = 0; k8 < K / 8; ++k8) {
+          ptx::mma_tf32_ss(tmem + kFftTmemD2, ah[k8], wh[k8], idesc, k8 != 0);
+          ptx::mma_tf32_ss(tmem + kFftTmemD2, al[k8], wh[k8], idesc, 1);
+          ptx::mma_tf32_ss(tmem + kFftTmemD2, ah[k8], wl[k8], idesc, 1);
         }
+        ptx::tc_commit(&sh.a2_empty);
+        ptx::tc_commit(&sh.d2_full);
       }
     }
   } else if (warp >= 4 && warp < 8) {
@@ -273,63 +324,66 @@ fft_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_const
         }
       }
     }
-  } else if (warp >= 8 && warp < 12) {
+  } else if (warp >= 8 && warp < 16) {
     // ------------------------------------------------------------ drain stage 1: sum halves, twiddle, split, write A2
-    const int q = warp & 3;
-    const int m = q * 32 + lane;
-    const int sl = m / R, beta = m % R;
-    const uint32_t lane_addr = tmem + (uint32_t(q * 32) << 16) + kFftTmemD1;
-    // A2 row of (sl, k1): CONTIG sl*R + k1 ; STRIDED k1*SL + sl (so that stage-2 stores of one k2 touch neighbouring lines)
-    const int row_mul_k1 = (MODE == FFT_CONTIG) ? 1 : SL;
-    const int row_base = (MODE == FFT_CONTIG) ? sl * R : sl;
-    // K column (beta, q) -> panel beta/16, 16-byte chunk (beta%16)/2, half beta%2
-    const uint32_t a2_col = uint32_t(beta >> 4) * (128u * 128u) + uint32_t(beta & 1) * 8u;
-    const uint32_t a2_chunk = uint32_t(beta & 15) >> 1;
-    const float2* tw = p.twiddle + beta;
-    for (long long t = 0; t < my_mtiles; ++t) {
-      FFT_WAIT_WARP(&sh.d1_full, uint32_t(t) & 1, 0x801);
-      ptx::tc_fence_after();
-      float cre[R], cim[R];                         // C[k1] for this lane's beta
+    // Two warp groups share the work by k1: group c takes the 16 values k1 = 16c .. 16c+15 (one 32-column chunk of
+    // each accumulator half).  For R = 16 there is one chunk and the second group has nothing to do.
+    const int grp = (warp - 8) >> 2;
+    if (grp < K / 32) {
+      const int q = warp & 3;
+      const int m = q * 32 + lane;
+      const int sl = m / R, beta = m % R;
+      const uint32_t lane_addr = tmem + (uint32_t(q * 32) << 16) + kFftTmemD1 + grp * 32;
+      // A2 row of (sl, k1): CONTIG sl*R + k1 ; STRIDED k1*SL + sl (so that stage-2 stores of one k2 touch neighbouring lines)
+      const int row_mul_k1 = (MODE == FFT_CONTIG) ? 1 : SL;
+      const int row_base = ((MODE == FFT_CONTIG) ? sl * R : sl) + grp * 16 * row_mul_k1;
+      // K column (beta, q) -> panel beta/16, 16-byte chunk (beta%16)/2, half beta%2
+      const uint32_t a2_col = uint32_t(beta >> 4) * (128u * 128u) + uint32_t(beta & 1) * 8u;
+      const uint32_t a2_chunk = uint32_t(beta & 15) >> 1;
+      float twr[16], twi[16];                        // T[16*grp + j][beta], kept for the whole kernel
 #pragma unroll
-      for (int ch = 0; ch < K / 32; ++ch) {         // 32 reals = 16 values of k1 per chunk
-        uint32_t v0[32], v1[32];
-        ptx::tmem_ld_32x32(lane_addr + ch * 32, v0);
-        ptx::tmem_ld_32x32(lane_addr + K + ch * 32, v1);
+      for (int j = 0; j < 16; ++j) {
+        const float2 w = __ldg(p.twiddle + (grp * 16 + j) * R + beta);
+        twr[j] = w.x; twi[j] = w.y;
+      }
+      for (long long t = 0; t < my_mtiles; ++t) {
+        FFT_WAIT_WARP(&sh.d1_full, uint32_t(t) & 1, 0x801);
+        ptx::tc_fence_after();
+        uint32_t v0[32];
+        ptx::tmem_ld_32x32(lane_addr, v0);
         ptx::tc_wait_ld();
-        if (ch == K / 32 - 1) {
-          ptx::tc_fence_before();
-          __syncwarp();
-          if (lane == 0) ptx::mbar_arrive(&sh.d1_empty);
-        }
+        ptx::tc_fence_before();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(&sh.d1_empty);
+        float cre[16], cim[16];                       // C[k1] for this lane's beta
 #pragma unroll
         for (int j = 0; j < 16; ++j) {
-          const float br = __uint_as_float(v0[2 * j]) + __uint_as_float(v1[2 * j]);
-          const float bi = __uint_as_float(v0[2 * j + 1]) + __uint_as_float(v1[2 * j + 1]);
-          const float2 w = __ldg(tw + (ch * 16 + j) * R);
-          cre[ch * 16 + j] = br * w.x - bi * w.y;
-          cim[ch * 16 + j] = br * w.y + bi * w.x;
+          const float br = __uint_as_float(v0[2 * j]);
+          const float bi = __uint_as_float(v0[2 * j + 1]);
+          cre[j] = br * twr[j] - bi * twi[j];
+          cim[j] = br * twi[j] + bi * twr[j];
         }
-      }
-      // stage 2 of the previous M-tile must be done reading A2
-      FFT_WAIT_WARP(&sh.a2_empty, (uint32_t(t) & 1) ^ 1, 0x802);
+        // stage 2 of the previous M-tile must be done reading A2
+        FFT_WAIT_WARP(&sh.a2_empty, (uint32_t(t) & 1) ^ 1, 0x802);
+        int rb = row_base;
+        asm volatile("" : "+r"(rb));                  // recompute the 16 store addresses per tile instead of keeping them live
 #pragma unroll
-      for (int k1 = 0; k1 < R; ++k1) {
-        {
-          const int row = row_base + k1 * row_mul_k1;
+        for (int j = 0; j < 16; ++j) {
+          const int row = rb + j * row_mul_k1;
           const uint32_t off = a2_col + uint32_t(row) * 128u + ((a2_chunk ^ uint32_t(row & 7)) << 4);
-          const uint32_t hr = __float_as_uint(cre[k1]), hi_ = __float_as_uint(cim[k1]);
-          const float lr = cre[k1] - __uint_as_float(hr & 0xffffe000u);
-          const float li = cim[k1] - __uint_as_float(hi_ & 0xffffe000u);
+          const uint32_t hr = __float_as_uint(cre[j]), hi_ = __float_as_uint(cim[j]);
+          const float lr = cre[j] - __uint_as_float(hr & 0xffffe000u);
+          const float li = cim[j] - __uint_as_float(hi_ & 0xffffe000u);
           *reinterpret_cast<uint2*>(smem_a2 + off) = make_uint2(hr, hi_);
           *reinterpret_cast<uint2*>(smem_a2 + a2_piece + off) =
               make_uint2((__float_as_uint(lr) + 0x1000u) & 0xffffe000u, (__float_as_uint(li) + 0x1000u) & 0xffffe000u);
         }
+        ptx::fence_proxy_async_smem();                // generic writes -> visible to the MMA's shared-memory reads
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(&sh.a2_full);
       }
-      ptx::fence_proxy_async_smem();                // generic writes -> visible to the MMA's shared-memory reads
-      __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(&sh.a2_full);
     }
-  } else if (warp >= 12) {
+  } else if (warp >= 16) {
     // ------------------------------------------------------------ drain stage 2: sum halves, store in natural order
     const int q = warp & 3;
     const int m = q * 32 + lane;
@@ -359,9 +413,8 @@ fft_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_const
         ptx::tc_fence_after();
 #pragma unroll
         for (int ch = 0; ch < K / 32; ++ch) {
-          uint32_t v0[32], v1[32];
+          uint32_t v0[32];
           ptx::tmem_ld_32x32(lane_addr + ch * 32, v0);
-          ptx::tmem_ld_32x32(lane_addr + K + ch * 32, v1);
           ptx::tc_wait_ld();
           if (ch == K / 32 - 1) {
             ptx::tc_fence_before();
@@ -369,11 +422,12 @@ fft_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_const
             if (lane == 0) ptx::mbar_arrive(&sh.d2_empty);
           }
           if (ok) {
+            float2* pd = dst + (long long)(ch * 16) * k2_stride;
 #pragma unroll
             for (int j = 0; j < 16; ++j) {
-              const float yr = __uint_as_float(v0[2 * j]) + __uint_as_float(v1[2 * j]);
-              const float yi = __uint_as_float(v0[2 * j + 1]) + __uint_as_float(v1[2 * j + 1]);
-              dst[(long long)(ch * 16 + j) * k2_stride] = make_float2(yr, yi);
+              *pd = make_float2(__uint_as_float(v0[2 * j]), __uint_as_float(v0[2 * j + 1]));
+              pd += k2_stride;
+              asm volatile("" : "+l"(pd));            // one running pointer, not sixteen precomputed ones
             }
           }
         }
@@ -382,6 +436,16 @@ fft_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_const
   }
 
 role_done:
+#ifdef DFT3D_PROFILE_WAITS
+  if (p.profile && lane == 0 && (warp <= 2 || (warp & 3) == 0)) {
+    // one reporter per role: codes 0x5xx producer, 0x6xx MMA, 0x7xx split, 0x8xx drain 1, 0x9xx drain 2
+    long long* dst = p.profile + size_t(blockIdx.x) * 128;
+    for (int i = 5; i < 10; ++i)
+      for (int j = 0; j < 8; ++j)
+        if (prof_wait[i][j]) dst[i * 8 + j] = prof_wait[i][j];
+    if (warp == 0) dst[0] = clock64() - prof_start;
+  }
+#endif
   if (warp == 0 && lane == 0 && sh.abort_flag) {
     const long long t0 = clock64();
     while (clock64() - t0 < 2000000LL) { }
