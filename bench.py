@@ -50,6 +50,13 @@ def conv_flops(n):
     return 5.0 * P * math.log2(P)
 
 
+# DRAM bytes per point per launch (dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture divided by the
+# points of that launch; smaller cases than the bench workload, traffic grows in proportion to the points):
+#   profiles/fft_axis_kernel_256x1024x1024.md : (2.148 + 2.094) GB / 268.4 M points
+#   profiles/kdft_axis_kernel_512.md          : (1.084 + 1.035) GB / 134.2 M points
+NCU_DRAM_BYTES_PER_POINT = {"fft_axis_kernel": 15.80, "kdft_axis_kernel": 15.79}
+
+
 def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -249,7 +256,8 @@ def main():
             tf32_peak = peaks["bf16_tflops_sustained"] * (1.1 / 2.25)
             ach = issued / (ms * 1e-3) * 1e-12
             return {"bound": "tensor", "kernel": "kdft_axis_kernel", "achieved": ach, "peak": tf32_peak, "unit": "TFLOP/s",
-                    "frac": ach / tf32_peak, "traffic": None,
+                    "frac": ach / tf32_peak, "traffic": NCU_DRAM_BYTES_PER_POINT["kdft_axis_kernel"] * P,
+                    "traffic_note": "DRAM bytes per launch, ncu capture at 512^3 scaled by points (algorithmic: 16 B/point)",
                     "peak_source": "%s bf16 sustained x nominal TF32/bf16 ratio (1.1/2.25)" % peak_kind,
                     "flops": "issued TF32 tensor flops = 3 split products x 8*n_a flops per point per axis",
                     "useful_gemm_tflops": algo_flops / (ms * 1e-3) * 1e-12, "avg_launch_ms": ms / nlaunch}
@@ -261,7 +269,9 @@ def main():
             algo_bytes = 3 * 16.0 * P
             achieved = algo_bytes / (ms_step * 1e-3) * 1e-9
             roofline = {"bound": "hbm", "kernel": "fft_axis_kernel", "achieved": achieved, "peak": peaks["hbm_gbs"],
-                        "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "traffic": None,
+                        "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
+                        "traffic": NCU_DRAM_BYTES_PER_POINT["fft_axis_kernel"] * P,
+                        "traffic_note": "DRAM bytes per launch, ncu capture at 256x1024x1024 scaled by points",
                         "peak_source": "%s STREAM-style copy" % peak_kind, "avg_launch_ms": ms_step / launches,
                         "bytes": "8 B read + 8 B written per point per axis pass"}
         if kdft_info is not None:
