@@ -56,6 +56,9 @@ typedef struct dft3d_options_s {
   unsigned flags;         /* DFT3D_NODES_ON_OUTPUT | DFT3D_UNSCALED_INVERSE */
   int fft_split[3][2];    /* FFT mode: {N1, N2} per axis with N1*N2 = n_a; {0,0} = default split */
   size_t workspace_limit; /* KDFT mode: upper bound in bytes for the plan-owned workspace; 0 = default */
+  unsigned axes;          /* bit a set = transform axis a; 0 = all three.  6 (axes 1 and 2) is a batch of n0
+                             two-dimensional transforms (Eq. 5), 4 a batch of n0*n1 one-dimensional ones (Eq. 2).
+                             An axis that is not transformed may have any length >= 1 if it is axis 0. */
 } dft3d_options_t;
 
 /*
@@ -76,8 +79,9 @@ typedef struct dft3d_options_s {
  * reduced phases and rounded once to the stored float32 pieces.  The plan owns its
  * device tables and workspace (allocated on the current device during this call).
  *
- * Supported sizes: every n_a a multiple of 64, n_a <= 8192 (KDFT) ; FFT additionally needs
- * N1 and N2 multiples of 16.  Other sizes return DFT3D_ERR_UNSUPPORTED.
+ * Supported sizes: KDFT: every n_a a multiple of 64, n_a <= 8192.  FFT: every transformed n_a in
+ * {256, 512, 1024, 2048} (N = R*R or 2*R*R with R = 16 or 32), the others multiples of 64.
+ * Other sizes return DFT3D_ERR_UNSUPPORTED.
  */
 int dft3d_plan_create(dft3d_plan_t* out, long long n0, long long n1, long long n2, int mode, int sign,
                       const double* nodes0, const double* nodes1, const double* nodes2);

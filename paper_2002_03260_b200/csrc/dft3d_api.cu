@@ -101,6 +101,7 @@ struct dft3d_plan_s {
   long long n[3] = {0, 0, 0};
   int mode = 0, sign = 0;
   unsigned flags = 0;
+  unsigned axes = 7;            // bit a: axis a is transformed
   int device = 0;
   int sm_count = 0;
   KdftAxis kax[3];
@@ -448,9 +449,13 @@ int dft3d_plan_create_ex(dft3d_plan_t* out, long long n0, long long n1, long lon
     memcpy(&opt, options, options->struct_size);
   }
   if (opt.flags & ~(DFT3D_NODES_ON_OUTPUT | DFT3D_UNSCALED_INVERSE)) return fail(DFT3D_ERR_INVALID_ARG, "unknown flag");
+  if (opt.axes > 7) return fail(DFT3D_ERR_INVALID_ARG, "axes must be a mask of bits 0..2");
+  const unsigned axes = opt.axes ? opt.axes : 7u;
   for (int a = 0; a < 3; ++a) {
+    const bool transformed = (axes >> a) & 1u;
+    if (a == 0 && !transformed) continue;   // a pure batch index
     if (nn[a] % 64 != 0) return fail(DFT3D_ERR_UNSUPPORTED, "n%d = %lld is not a multiple of 64", a, nn[a]);
-    if (nn[a] > 8192) return fail(DFT3D_ERR_UNSUPPORTED, "n%d = %lld exceeds 8192", a, nn[a]);
+    if (transformed && nn[a] > 8192) return fail(DFT3D_ERR_UNSUPPORTED, "n%d = %lld exceeds 8192", a, nn[a]);
   }
   if (mode == DFT3D_FFT && (nodes0 || nodes1 || nodes2))
     return fail(DFT3D_ERR_UNSUPPORTED, "the FFT formulation needs a uniform grid (no nodes)");
@@ -465,6 +470,7 @@ int dft3d_plan_create_ex(dft3d_plan_t* out, long long n0, long long n1, long lon
     p->mode = mode;
     p->sign = sign;
     p->flags = opt.flags;
+    p->axes = axes;
     cudaDeviceProp prop;
     if (cudaGetDevice(&p->device) != cudaSuccess || cudaGetDeviceProperties(&prop, p->device) != cudaSuccess) {
       rc = fail(DFT3D_ERR_CUDA, "cannot query the current device");
@@ -490,7 +496,8 @@ int dft3d_plan_create_ex(dft3d_plan_t* out, long long n0, long long n1, long lon
     if (e != cudaSuccess) { rc = fail(DFT3D_ERR_ALLOC, "cudaMalloc(profile)"); break; }
 #endif
     if (mode == DFT3D_KDFT) {
-      for (int a = 0; a < 3 && rc == DFT3D_OK; ++a) rc = build_kdft_axis(p, a, nodes[a]);
+      for (int a = 0; a < 3 && rc == DFT3D_OK; ++a)
+        if ((axes >> a) & 1u) rc = build_kdft_axis(p, a, nodes[a]);
       if (rc != DFT3D_OK) break;
       // workspace: whole cube when it fits the limit, else a group of n0-planes with at least ~8 waves of tiles
       const size_t plane_bytes = size_t(n1) * n2 * 8;
@@ -501,12 +508,21 @@ int dft3d_plan_create_ex(dft3d_plan_t* out, long long n0, long long n1, long lon
         if (g < 1) g = 1;
         while (n0 % g) --g;   // groups of equal size
       }
-      p->group_planes = g;
+      if (g != n0 && (axes == 3u || axes == 5u)) {
+        rc = fail(DFT3D_ERR_UNSUPPORTED, "transforming axis 0 and one other axis needs a workspace as large as the cube "
+                  "(%zu bytes); raise workspace_limit", size_t(n0) * plane_bytes);
+        break;
+      }
+      if (axes == 1u || axes == 2u || axes == 4u) g = 0;   // a single axis goes straight from in to out
+      p->group_planes = g ? g : n0;
       p->workspace_bytes = size_t(g) * plane_bytes;
-      e = cudaMalloc(&p->workspace, p->workspace_bytes);
-      if (e != cudaSuccess) { rc = fail(DFT3D_ERR_ALLOC, "cudaMalloc(workspace %zu bytes): %s", p->workspace_bytes, cudaGetErrorString(e)); break; }
+      if (g != 0) {
+        e = cudaMalloc(&p->workspace, p->workspace_bytes);
+        if (e != cudaSuccess) { rc = fail(DFT3D_ERR_ALLOC, "cudaMalloc(workspace %zu bytes): %s", p->workspace_bytes, cudaGetErrorString(e)); break; }
+      }
     } else {
-      for (int a = 0; a < 3 && rc == DFT3D_OK; ++a) rc = build_fft_axis(p, a, opt.fft_split[a]);
+      for (int a = 0; a < 3 && rc == DFT3D_OK; ++a)
+        if ((axes >> a) & 1u) rc = build_fft_axis(p, a, opt.fft_split[a]);
       if (rc != DFT3D_OK) break;
     }
   } while (0);
@@ -530,6 +546,7 @@ int dft3d_execute_axis(dft3d_plan_t p, int axis, const void* in, void* out, void
   int rc = check_io(p, in, out);
   if (rc != DFT3D_OK) return rc;
   if (axis < 0 || axis > 2) return fail(DFT3D_ERR_INVALID_ARG, "axis must be 0, 1 or 2");
+  if (!((p->axes >> axis) & 1u)) return fail(DFT3D_ERR_INVALID_ARG, "axis %d is not among the plan's axes", axis);
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   if (p->mode == DFT3D_KDFT)
     return kdft_axis_pass(p, axis, static_cast<const float*>(in), static_cast<float*>(out), p->n[0], stream);
@@ -542,24 +559,44 @@ int dft3d_execute(dft3d_plan_t p, const void* in, void* out, void* cuda_stream) 
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   const float* fin = static_cast<const float*>(in);
   float* fout = static_cast<float*>(out);
+  const unsigned axes = p->axes;
   if (p->mode == DFT3D_KDFT) {
-    // axis 0: in -> out; then per group of n0-planes: axis 1 out -> workspace, axis 2 workspace -> out
-    if ((rc = kdft_axis_pass(p, 0, fin, fout, p->n[0], stream)) != DFT3D_OK) return rc;
     const long long g = p->group_planes;
     const long long plane_floats = p->n[1] * p->n[2] * 2;
     float* ws = static_cast<float*>(p->workspace);
-    for (long long a = 0; a < p->n[0]; a += g) {
-      float* slab = fout + a * plane_floats;
-      if ((rc = kdft_axis_pass(p, 1, slab, ws, g, stream)) != DFT3D_OK) return rc;
-      if ((rc = kdft_axis_pass(p, 2, ws, slab, g, stream)) != DFT3D_OK) return rc;
+    if (axes == 7u) {
+      // axis 0: in -> out; then per group of n0-planes: axis 1 out -> workspace, axis 2 workspace -> out
+      if ((rc = kdft_axis_pass(p, 0, fin, fout, p->n[0], stream)) != DFT3D_OK) return rc;
+      for (long long a = 0; a < p->n[0]; a += g) {
+        float* slab = fout + a * plane_floats;
+        if ((rc = kdft_axis_pass(p, 1, slab, ws, g, stream)) != DFT3D_OK) return rc;
+        if ((rc = kdft_axis_pass(p, 2, ws, slab, g, stream)) != DFT3D_OK) return rc;
+      }
+    } else if (axes == 6u) {
+      // batch of 2D transforms: per group axis 1 in -> workspace, axis 2 workspace -> out
+      for (long long a = 0; a < p->n[0]; a += g) {
+        if ((rc = kdft_axis_pass(p, 1, fin + a * plane_floats, ws, g, stream)) != DFT3D_OK) return rc;
+        if ((rc = kdft_axis_pass(p, 2, ws, fout + a * plane_floats, g, stream)) != DFT3D_OK) return rc;
+      }
+    } else if (axes == 3u || axes == 5u) {
+      // axis 0 and one more: the other axis in -> workspace (whole cube), then axis 0 workspace -> out
+      if ((rc = kdft_axis_pass(p, axes == 3u ? 1 : 2, fin, ws, p->n[0], stream)) != DFT3D_OK) return rc;
+      if ((rc = kdft_axis_pass(p, 0, ws, fout, p->n[0], stream)) != DFT3D_OK) return rc;
+    } else {
+      const int a = axes == 1u ? 0 : (axes == 2u ? 1 : 2);
+      if ((rc = kdft_axis_pass(p, a, fin, fout, p->n[0], stream)) != DFT3D_OK) return rc;
     }
     return DFT3D_OK;
   }
-  // FFT: axis 2 in -> out, then axes 1 and 0 in place on out (a CTA loads a group of lines completely into
-  // shared memory before it stores any of their results, and groups are disjoint)
-  if ((rc = fft_axis_pass(p, 2, fin, fout, stream)) != DFT3D_OK) return rc;
-  if ((rc = fft_axis_pass(p, 1, fout, fout, stream)) != DFT3D_OK) return rc;
-  return fft_axis_pass(p, 0, fout, fout, stream);
+  // FFT: the first transformed axis (last axis first) in -> out, the others in place on out (a CTA loads a group of
+  // lines completely into shared memory before it stores any of their results, and groups are disjoint)
+  const float* src = fin;
+  for (int a = 2; a >= 0; --a) {
+    if (!((axes >> a) & 1u)) continue;
+    if ((rc = fft_axis_pass(p, a, src, fout, stream)) != DFT3D_OK) return rc;
+    src = fout;
+  }
+  return DFT3D_OK;
 }
 
 int dft3d_execute_host(dft3d_plan_t p, const void* host_in, void* host_out, void* cuda_stream) {
@@ -589,8 +626,10 @@ size_t dft3d_plan_workspace_bytes(dft3d_plan_t p) { return p ? p->workspace_byte
 
 int dft3d_plan_launches(dft3d_plan_t p) {
   if (!p) return 0;
-  if (p->mode == DFT3D_KDFT) return int(1 + 2 * (p->n[0] / p->group_planes));
-  return 3;
+  const int count = int((p->axes & 1u) + ((p->axes >> 1) & 1u) + ((p->axes >> 2) & 1u));
+  if (p->mode == DFT3D_KDFT && p->axes == 7u) return int(1 + 2 * (p->n[0] / p->group_planes));
+  if (p->mode == DFT3D_KDFT && p->axes == 6u) return int(2 * (p->n[0] / p->group_planes));
+  return count;
 }
 
 int dft3d_plan_destroy(dft3d_plan_t p) {

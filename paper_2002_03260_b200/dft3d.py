@@ -33,7 +33,8 @@ class Dft3dError(RuntimeError):
 
 class _Options(ctypes.Structure):
     _fields_ = [("struct_size", ctypes.c_size_t), ("flags", ctypes.c_uint),
-                ("fft_split", (ctypes.c_int * 2) * 3), ("workspace_limit", ctypes.c_size_t)]
+                ("fft_split", (ctypes.c_int * 2) * 3), ("workspace_limit", ctypes.c_size_t),
+                ("axes", ctypes.c_uint)]
 
 
 def library_path():
@@ -138,10 +139,11 @@ class Plan:
 
     plan = Plan(n0, n1, n2, mode=DFT3D_KDFT, sign=DFT3D_FORWARD, nodes=(None, None, None))
     y = plan(x)            # x: complex64 CUDA tensor [n0, n1, n2]; y: new tensor (or pass out=)
+    Plan(b, n1, n2, axes=(1, 2)) is a batch of b two-dimensional transforms, axes=(2,) a batch of 1D ones.
     """
 
     def __init__(self, n0, n1, n2, mode=DFT3D_KDFT, sign=DFT3D_FORWARD, nodes=None, flags=0, fft_split=None,
-                 workspace_limit=0):
+                 workspace_limit=0, axes=None):
         self.shape = (int(n0), int(n1), int(n2))
         self.mode, self.sign = mode, sign
         self._h = ctypes.c_void_p()
@@ -151,6 +153,7 @@ class Plan:
         opt.struct_size = ctypes.sizeof(_Options)
         opt.flags = flags
         opt.workspace_limit = workspace_limit
+        opt.axes = 0 if axes is None else sum(1 << int(a) for a in set(axes))   # e.g. axes=(1, 2): batch of 2D transforms
         if fft_split is not None:
             for a in range(3):
                 if fft_split[a] is not None:

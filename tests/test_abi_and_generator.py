@@ -58,6 +58,18 @@ def test_argument_validation_needs_no_gpu(dft):
         with pytest.raises(dft.Dft3dError) as e:
             dft.Plan(*n, **kw)
         assert e.value.status == status, (n, kw, str(e.value))
+    # axis subsets: an untransformed axis 0 may have any length; the other axes still need multiples of 64
+    with pytest.raises(dft.Dft3dError) as e:
+        dft.Plan(3, 100, 64, axes=(1, 2))
+    assert e.value.status == 2
+    with pytest.raises(dft.Dft3dError) as e:
+        dft.Plan(3, 128, 64, axes=(0, 1, 2))
+    assert e.value.status == 2
+    import torch
+    if not torch.cuda.is_available():
+        with pytest.raises(dft.Dft3dError) as e:
+            dft.Plan(3, 128, 64, axes=(1, 2))      # valid sizes: the first failure is the missing device
+        assert e.value.status == 4
     from paper_2002_03260_b200 import dft3d as b
     assert b._lib.dft3d_plan_create(None, 64, 64, 64, 0, -1, None, None, None) == 1
     assert b._lib.dft3d_plan_destroy(None) == 0

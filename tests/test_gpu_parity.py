@@ -406,3 +406,53 @@ def test_config5_2048_exponentials_both_modes(lib, oracle):
                 # Parseval is sum|x|^2
                 assert num / a.numel() < (TOL ** 2) * ex, (num / a.numel(), den / a.numel(), ex)
     del kept
+
+
+# ------------------------------------------------------------------ batched 2D / 1D transforms (subset of the axes)
+
+def _oracle_axes(oracle, xh, axes, **kw):
+    y = xh.astype(np.complex128)
+    for a in axes:
+        y = oracle.dft_axis(y, a, **kw)
+    return y
+
+
+@pytest.mark.parametrize("mode_name,shape", [("kdft", (3, 128, 192)), ("kdft", (1, 64, 256)), ("fft", (5, 256, 512))])
+def test_batched_2d(lib, oracle, mode_name, shape):
+    """axes=(1,2): n0 independent 2D transforms X = V1 x V2^T (Eq. 5); n0 need not be a multiple of 64."""
+    mode = lib.DFT3D_KDFT if mode_name == "kdft" else lib.DFT3D_FFT
+    x = _inputs().cube(shape, "normal", 81, device="cuda")
+    plan = lib.Plan(*shape, mode=mode, axes=(1, 2))
+    y = plan(x)
+    _finish(plan)
+    assert plan.launches == 2
+    plan.destroy()
+    err = oracle.rel_l2(y.cpu().numpy(), _oracle_axes(oracle, x.cpu().numpy(), (1, 2)))
+    assert err < SANITY, (mode_name, shape, err)
+
+
+@pytest.mark.parametrize("axes", [(2,), (1,), (0,), (0, 1), (0, 2)])
+def test_axis_subsets_kdft(lib, oracle, axes):
+    shape = (64, 128, 64)
+    x = _inputs().cube(shape, "uniform", 82, device="cuda")
+    plan = lib.Plan(*shape, axes=axes, sign=lib.DFT3D_INVERSE)
+    y = plan(x)
+    _finish(plan)
+    assert plan.launches == len(axes)
+    with pytest.raises(lib.Dft3dError):
+        plan.execute_axis([a for a in range(3) if a not in axes][0], x)
+    plan.destroy()
+    ref = x.cpu().numpy().astype(np.complex128)
+    for a in axes:
+        ref = oracle.dft_axis(ref, a, sign=+1, scale=1.0 / shape[a])
+    assert oracle.rel_l2(y.cpu().numpy(), ref) < SANITY, axes
+
+
+def test_batched_1d_fft(lib, oracle):
+    shape = (7, 64, 1024)
+    x = _inputs().cube(shape, "normal", 83, device="cuda")
+    plan = lib.Plan(*shape, mode=lib.DFT3D_FFT, axes=(2,))
+    y = plan(x)
+    _finish(plan)
+    plan.destroy()
+    assert oracle.rel_l2(y.cpu().numpy(), _oracle_axes(oracle, x.cpu().numpy(), (2,))) < SANITY_AXIS
