@@ -128,17 +128,18 @@ int set_kernel_attributes() {
                                   cudaFuncAttributeMaxDynamicSharedMemorySize, int(dft3d::kKdftSmemBytes)));
   DFT3D_CUDA(cudaFuncSetAttribute(dft3d::kdft_axis_kernel<dft3d::KDFT_STRIDED>,
                                   cudaFuncAttributeMaxDynamicSharedMemorySize, int(dft3d::kKdftSmemBytes)));
-#define DFT3D_FFT_ATTR(MODE, R, RX, COLS)                                                                     \
-  DFT3D_CUDA(cudaFuncSetAttribute(dft3d::fft_axis_kernel<MODE, R, RX, COLS>,                                   \
-                                  cudaFuncAttributeMaxDynamicSharedMemorySize, int(dft3d::fft_smem_bytes(R))))
-  DFT3D_FFT_ATTR(dft3d::FFT_CONTIG, 32, 1, 16);
-  DFT3D_FFT_ATTR(dft3d::FFT_CONTIG, 16, 1, 16);
-  DFT3D_FFT_ATTR(dft3d::FFT_CONTIG, 32, 2, 16);
-  DFT3D_FFT_ATTR(dft3d::FFT_CONTIG, 16, 2, 16);
-  DFT3D_FFT_ATTR(dft3d::FFT_STRIDED, 32, 1, 16);
-  DFT3D_FFT_ATTR(dft3d::FFT_STRIDED, 16, 1, 16);
-  DFT3D_FFT_ATTR(dft3d::FFT_STRIDED, 32, 2, 8);
-  DFT3D_FFT_ATTR(dft3d::FFT_STRIDED, 16, 2, 16);
+#define DFT3D_FFT_ATTR(MODE, R, RX, COLS, NB2)                                                                \
+  DFT3D_CUDA(cudaFuncSetAttribute(dft3d::fft_axis_kernel<MODE, R, RX, COLS, NB2>,                              \
+                                  cudaFuncAttributeMaxDynamicSharedMemorySize, int(dft3d::fft_smem_bytes(R, NB2))))
+  DFT3D_FFT_ATTR(dft3d::FFT_CONTIG, 32, 1, 16, 2);
+  DFT3D_FFT_ATTR(dft3d::FFT_CONTIG, 16, 1, 16, 2);
+  DFT3D_FFT_ATTR(dft3d::FFT_CONTIG, 32, 2, 16, 2);
+  DFT3D_FFT_ATTR(dft3d::FFT_CONTIG, 16, 2, 16, 2);
+  DFT3D_FFT_ATTR(dft3d::FFT_STRIDED, 32, 1, 16, 1);
+  DFT3D_FFT_ATTR(dft3d::FFT_STRIDED, 32, 1, 8, 2);
+  DFT3D_FFT_ATTR(dft3d::FFT_STRIDED, 16, 1, 16, 2);
+  DFT3D_FFT_ATTR(dft3d::FFT_STRIDED, 32, 2, 8, 1);
+  DFT3D_FFT_ATTR(dft3d::FFT_STRIDED, 16, 2, 16, 2);
 #undef DFT3D_FFT_ATTR
   done = true;
   return DFT3D_OK;
@@ -263,7 +264,7 @@ int build_fft_axis(dft3d_plan_s* p, int a, const int split[2]) {
   ax.n = n;
   ax.R = R;
   ax.RX = RX;
-  ax.cols = (R == 32 && RX == 2) ? 8 : 16;
+  ax.cols = (R == 32 && RX == 2) ? 8 : 16;   // default; fft_axis_pass may pick 8 for R = 32, RX = 1 (see there)
   const bool scaled = (p->sign > 0) && !(p->flags & DFT3D_UNSCALED_INVERSE);
   const int K = 2 * R, NB = 2 * R, panels = K / 32;
   std::vector<double> M(size_t(2) * R * R), T(size_t(2) * R * R);
@@ -303,6 +304,15 @@ int build_fft_axis(dft3d_plan_s* p, int a, const int split[2]) {
 int fft_axis_pass(dft3d_plan_s* p, int axis, const float* in, float* out, cudaStream_t stream) {
   const FftAxis& ax = p->fax[axis];
   const int R = ax.R, RX = ax.RX, N = int(ax.n), Lg = 128 / (R * RX);
+  int cols = ax.cols;
+  if (axis != 2 && R == 32 && RX == 1) {
+    // 1024-point strided axes: 16 lines per stage (128-byte rows) leave room for one stage-2 operand buffer only;
+    // 8 lines per stage (64-byte rows) allow two.  Rows far apart (large strides) favour the wider rows.
+    const long long C = (axis == 0) ? p->n[1] * p->n[2] : p->n[2];
+    const char* env = getenv("DFT3D_FFT_COLS");
+    cols = env ? atoi(env) : ((C * 8 >= (1ll << 20)) ? 16 : 8);
+    if (cols != 8 && cols != 16) cols = 16;
+  }
   dft3d::FftParams fp;
   memset(&fp, 0, sizeof(fp));
   fp.N = N;
@@ -327,32 +337,40 @@ int fft_axis_pass(dft3d_plan_s* p, int axis, const float* in, float* out, cudaSt
     const long long batches = (axis == 0) ? 1 : p->n[0];
     const long long C = (axis == 0) ? p->n[1] * p->n[2] : p->n[2];
     fp.C = C;
-    fp.c_tiles = C / ax.cols;
-    fp.mtiles_per_stage = ax.cols / Lg;
-    fp.stage_bytes = N * ax.cols * 8;
+    fp.c_tiles = C / cols;
+    {
+      // prefetching helps while rows are close (axis 1); with rows MiBs apart (axis 0) the pass is bound by the
+      // rate of address translations and every extra request costs more than it hides (measured: 10.0 -> 12.2 ms)
+      const char* env = getenv("DFT3D_FFT_L2_PREFETCH");
+      fp.l2_prefetch = env ? atoi(env) : (C * 8 < (1ll << 20) ? 1 : 0);
+    }
+    fp.mtiles_per_stage = cols / Lg;
+    fp.stage_bytes = N * cols * 8;
     fp.num_stages = batches * fp.c_tiles;
     const unsigned long long dims[3] = {(unsigned long long)(2 * C), (unsigned long long)N, (unsigned long long)batches};
     const unsigned long long strides[2] = {(unsigned long long)(C * 8), (unsigned long long)N * C * 8ull};
-    const unsigned box[3] = {unsigned(2 * ax.cols), 256u, 1u};
-    rc = encode_f32(&map_data, in, 3, dims, strides, box, ax.cols * 8);
+    const unsigned box[3] = {unsigned(2 * cols), 256u, 1u};
+    rc = encode_f32(&map_data, in, 3, dims, strides, box, cols * 8);
   }
   if (rc != DFT3D_OK) return rc;
-  fp.raw_stages = dft3d::kFftRawBytes / fp.stage_bytes;
+  const int nb2 = (axis == 2 || R == 16 || (R == 32 && RX == 1 && cols == 8)) ? 2 : 1;
+  fp.raw_stages = dft3d::fft_raw_bytes(R, nb2) / fp.stage_bytes;
   if (fp.raw_stages > 4) fp.raw_stages = 4;
   const int grid = int(fp.num_stages < p->sm_count ? fp.num_stages : p->sm_count);
-  const size_t smem = dft3d::fft_smem_bytes(R);
-#define DFT3D_FFT_LAUNCH(MODE, R_, RX_, COLS_)                                                              \
-  dft3d::fft_axis_kernel<MODE, R_, RX_, COLS_><<<grid, dft3d::kFftThreads, smem, stream>>>(map_data, ax.map_w, fp)
+  const size_t smem = dft3d::fft_smem_bytes(R, nb2);
+#define DFT3D_FFT_LAUNCH(MODE, R_, RX_, COLS_, NB2_)                                                          \
+  dft3d::fft_axis_kernel<MODE, R_, RX_, COLS_, NB2_><<<grid, dft3d::kFftThreads, smem, stream>>>(map_data, ax.map_w, fp)
   if (axis == 2) {
-    if (R == 32 && RX == 1) DFT3D_FFT_LAUNCH(dft3d::FFT_CONTIG, 32, 1, 16);
-    else if (R == 16 && RX == 1) DFT3D_FFT_LAUNCH(dft3d::FFT_CONTIG, 16, 1, 16);
-    else if (R == 32) DFT3D_FFT_LAUNCH(dft3d::FFT_CONTIG, 32, 2, 16);
-    else DFT3D_FFT_LAUNCH(dft3d::FFT_CONTIG, 16, 2, 16);
+    if (R == 32 && RX == 1) DFT3D_FFT_LAUNCH(dft3d::FFT_CONTIG, 32, 1, 16, 2);
+    else if (R == 16 && RX == 1) DFT3D_FFT_LAUNCH(dft3d::FFT_CONTIG, 16, 1, 16, 2);
+    else if (R == 32) DFT3D_FFT_LAUNCH(dft3d::FFT_CONTIG, 32, 2, 16, 2);
+    else DFT3D_FFT_LAUNCH(dft3d::FFT_CONTIG, 16, 2, 16, 2);
   } else {
-    if (R == 32 && RX == 1) DFT3D_FFT_LAUNCH(dft3d::FFT_STRIDED, 32, 1, 16);
-    else if (R == 16 && RX == 1) DFT3D_FFT_LAUNCH(dft3d::FFT_STRIDED, 16, 1, 16);
-    else if (R == 32) DFT3D_FFT_LAUNCH(dft3d::FFT_STRIDED, 32, 2, 8);
-    else DFT3D_FFT_LAUNCH(dft3d::FFT_STRIDED, 16, 2, 16);
+    if (R == 32 && RX == 1 && cols == 16) DFT3D_FFT_LAUNCH(dft3d::FFT_STRIDED, 32, 1, 16, 1);
+    else if (R == 32 && RX == 1) DFT3D_FFT_LAUNCH(dft3d::FFT_STRIDED, 32, 1, 8, 2);
+    else if (R == 16 && RX == 1) DFT3D_FFT_LAUNCH(dft3d::FFT_STRIDED, 16, 1, 16, 2);
+    else if (R == 32) DFT3D_FFT_LAUNCH(dft3d::FFT_STRIDED, 32, 2, 8, 1);
+    else DFT3D_FFT_LAUNCH(dft3d::FFT_STRIDED, 16, 2, 16, 2);
   }
 #undef DFT3D_FFT_LAUNCH
   DFT3D_CUDA(cudaGetLastError());

@@ -41,8 +41,8 @@ namespace dft3d {
 enum : int { FFT_CONTIG = 0, FFT_STRIDED = 1 };
 
 constexpr int kFftThreads = 640;      // 5 warp groups: {producer, 2 MMA issuers}, split, drain 1 (x2), drain 2
-constexpr int kFftRawBytes = 128 * 1024;       // ring of raw-data stages
 // STRIDED stages hold COLS neighbouring lines: 16 (128-byte rows, 128B swizzle) or 8 (64-byte rows, 64B swizzle)
+// NB2 = buffers of the stage-2 operand (2 lets drain 1 write the next M-tile while stage 2 still reads this one)
 constexpr int kFftTmemD1 = 0, kFftTmemD2 = 128, kFftTmemA1 = 256;   // tensor-memory column map (A1: two buffers of 128)
 
 struct FftParams {
@@ -56,6 +56,7 @@ struct FftParams {
   // STRIDED: view [batches][N][C] complex
   long long C;
   long long c_tiles;     // C / COLS
+  int l2_prefetch;       // STRIDED: prefetch the next stage's rows into L2
   const float2* twiddle; // [R][R] complex64, T[k1][beta] (times 1/RX for a scaled inverse)
   const float2* twiddle2;// RX == 2: [R*R] complex64, exp(s*2*pi*i*m/N)
   float* out;
@@ -67,7 +68,7 @@ struct FftShared {
   uint64_t raw_full[4], raw_empty[4];
   uint64_t a1_full[2], a1_empty[2];
   uint64_t d1_full, d1_empty;
-  uint64_t a2_full, a2_empty;
+  uint64_t a2_full[2], a2_empty[2];
   uint64_t d2_full, d2_empty;
   uint64_t w_full;
   uint32_t tmem_base;
@@ -77,8 +78,10 @@ struct FftShared {
 // shared memory: [W: 2 pieces x 2R/32 panels of 2R rows x 128 B] [A2: hi panels, lo panels] [raw ring] [barriers]
 __host__ __device__ constexpr int fft_w_bytes(int R) { return (2 * R / 32) * 4 * R * 128; }
 __host__ __device__ constexpr int fft_a2_piece_bytes(int R) { return (2 * R / 32) * 128 * 128; }
-__host__ __device__ constexpr size_t fft_smem_bytes(int R) {
-  return size_t(fft_w_bytes(R)) + 2 * size_t(fft_a2_piece_bytes(R)) + kFftRawBytes + 1024 + 512;
+// the stage-2 operand has NB2 = 1 or 2 buffers; with two of them for R = 32 the raw ring shrinks to 64 KB
+__host__ __device__ constexpr int fft_raw_bytes(int R, int NB2) { return (R == 32 && NB2 == 2) ? 64 * 1024 : 128 * 1024; }
+__host__ __device__ constexpr size_t fft_smem_bytes(int R, int NB2) {
+  return size_t(fft_w_bytes(R)) + size_t(2 * NB2) * fft_a2_piece_bytes(R) + fft_raw_bytes(R, NB2) + 1024 + 512;
 }
 
 #ifdef DFT3D_PROFILE_WAITS
@@ -109,7 +112,7 @@ __host__ __device__ constexpr size_t fft_smem_bytes(int R) {
     FFT_PROF_END(code)                                                                    \
   }
 
-template <int MODE, int R, int RX, int COLS>
+template <int MODE, int R, int RX, int COLS, int NB2>
 __global__ void __launch_bounds__(kFftThreads, 1)
 fft_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_constant__ CUtensorMap map_w,
                 const FftParams p) {
@@ -122,8 +125,8 @@ fft_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_const
   uint8_t* smem_w = smem;
   uint8_t* smem_a2 = smem_w + fft_w_bytes(R);
   constexpr int a2_piece = fft_a2_piece_bytes(R);
-  uint8_t* smem_rawring = smem_a2 + 2 * a2_piece;
-  FftShared& sh = *reinterpret_cast<FftShared*>(smem_rawring + kFftRawBytes);
+  uint8_t* smem_rawring = smem_a2 + 2 * NB2 * a2_piece;     // A2 buffer i = [hi piece][lo piece] at i * 2 * a2_piece
+  FftShared& sh = *reinterpret_cast<FftShared*>(smem_rawring + fft_raw_bytes(R, NB2));
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 #ifdef DFT3D_PROFILE_WAITS
@@ -140,7 +143,7 @@ fft_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_const
     for (int i = 0; i < 4; ++i) { ptx::mbar_init(&sh.raw_full[i], 1); ptx::mbar_init(&sh.raw_empty[i], 4 * p.mtiles_per_stage); }
     for (int i = 0; i < 2; ++i) { ptx::mbar_init(&sh.a1_full[i], 4); ptx::mbar_init(&sh.a1_empty[i], 1); }
     ptx::mbar_init(&sh.d1_full, 1); ptx::mbar_init(&sh.d1_empty, 4 * (K / 32));
-    ptx::mbar_init(&sh.a2_full, 4 * (K / 32)); ptx::mbar_init(&sh.a2_empty, 1);
+    for (int i = 0; i < 2; ++i) { ptx::mbar_init(&sh.a2_full[i], 4 * (K / 32)); ptx::mbar_init(&sh.a2_empty[i], 1); }
     ptx::mbar_init(&sh.d2_full, 1); ptx::mbar_init(&sh.d2_empty, 4);
     ptx::mbar_init(&sh.w_full, 1);
     sh.abort_flag = 0;
@@ -184,6 +187,14 @@ fft_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_const
           const long long ct = sidx % p.c_tiles, bt = sidx / p.c_tiles;
           for (int r0 = 0; r0 < p.N; r0 += 256)
             ptx::tma_load_3d(dst + size_t(r0) * kRowBytes, &map_data, &sh.raw_full[s], int(ct * 2 * COLS), r0, int(bt));
+          // the ring is short on the strided axes (one or two stages), so the loads of the next stage cannot be
+          // issued yet; pull its rows into L2 meanwhile (rows are far apart: this also absorbs the TLB misses)
+          const long long nidx = sidx + gridDim.x;
+          if (p.l2_prefetch && nidx < p.num_stages) {
+            const long long nct = nidx % p.c_tiles, nbt = nidx / p.c_tiles;
+            for (int r0 = 0; r0 < p.N; r0 += 256)
+              ptx::tma_prefetch_l2_3d(&map_data, int(nct * 2 * COLS), r0, int(nbt));
+          }
         }
       }
     }
@@ -238,19 +249,21 @@ fft_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_const
         ah[k8] = ptx::make_kmajor_sw128_desc(a2_addr + off);
         al[k8] = ptx::make_kmajor_sw128_desc(a2_addr + a2_piece + off);
       }
+      constexpr uint64_t kBufStep = uint64_t(2 * a2_piece) >> 4;   // second A2 buffer, in descriptor address units
       FFT_WAIT(&sh.w_full, 0, 0x611);
       for (long long t = 0; t < my_mtiles; ++t) {
-        const uint32_t u = uint32_t(t);
-        FFT_WAIT(&sh.a2_full, u & 1, 0x604);
-        FFT_WAIT(&sh.d2_empty, (u & 1) ^ 1, 0x605);
+        const uint32_t bi = uint32_t(t % NB2), u = uint32_t(t / NB2);
+        FFT_WAIT(&sh.a2_full[bi], u & 1, 0x604);
+        FFT_WAIT(&sh.d2_empty, (uint32_t(t) & 1) ^ 1, 0x605);
         ptx::tc_fence_after();
+        const uint64_t bstep = bi ? kBufStep : 0;
 #pragma unroll
         for (int k8 = 0; k8 < K / 8; ++k8) {
-          ptx::mma_tf32_ss(tmem + kFftTmemD2, ah[k8], wh[k8], idesc, k8 != 0);
-          ptx::mma_tf32_ss(tmem + kFftTmemD2, al[k8], wh[k8], idesc, 1);
-          ptx::mma_tf32_ss(tmem + kFftTmemD2, ah[k8], wl[k8], idesc, 1);
+          ptx::mma_tf32_ss(tmem + kFftTmemD2, ah[k8] + bstep, wh[k8], idesc, k8 != 0);
+          ptx::mma_tf32_ss(tmem + kFftTmemD2, al[k8] + bstep, wh[k8], idesc, 1);
+          ptx::mma_tf32_ss(tmem + kFftTmemD2, ah[k8] + bstep, wl[k8], idesc, 1);
         }
-        ptx::tc_commit(&sh.a2_empty);
+        ptx::tc_commit(&sh.a2_empty[bi]);
         ptx::tc_commit(&sh.d2_full);
       }
     }
@@ -364,7 +377,9 @@ fft_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_const
           cim[j] = br * twi[j] + bi * twr[j];
         }
         // stage 2 of the previous M-tile must be done reading A2
-        FFT_WAIT_WARP(&sh.a2_empty, (uint32_t(t) & 1) ^ 1, 0x802);
+        const uint32_t bi = uint32_t(t % NB2), u = uint32_t(t / NB2);
+        FFT_WAIT_WARP(&sh.a2_empty[bi], (u & 1) ^ 1, 0x802);
+        uint8_t* a2buf = smem_a2 + size_t(bi) * 2 * a2_piece;
         int rb = row_base;
         asm volatile("" : "+r"(rb));                  // recompute the 16 store addresses per tile instead of keeping them live
 #pragma unroll
@@ -374,13 +389,13 @@ fft_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_const
           const uint32_t hr = __float_as_uint(cre[j]), hi_ = __float_as_uint(cim[j]);
           const float lr = cre[j] - __uint_as_float(hr & 0xffffe000u);
           const float li = cim[j] - __uint_as_float(hi_ & 0xffffe000u);
-          *reinterpret_cast<uint2*>(smem_a2 + off) = make_uint2(hr, hi_);
-          *reinterpret_cast<uint2*>(smem_a2 + a2_piece + off) =
+          *reinterpret_cast<uint2*>(a2buf + off) = make_uint2(hr, hi_);
+          *reinterpret_cast<uint2*>(a2buf + a2_piece + off) =
               make_uint2((__float_as_uint(lr) + 0x1000u) & 0xffffe000u, (__float_as_uint(li) + 0x1000u) & 0xffffe000u);
         }
         ptx::fence_proxy_async_smem();                // generic writes -> visible to the MMA's shared-memory reads
         __syncwarp();
-        if (lane == 0) ptx::mbar_arrive(&sh.a2_full);
+        if (lane == 0) ptx::mbar_arrive(&sh.a2_full[bi]);
       }
     }
   } else if (warp >= 16) {
