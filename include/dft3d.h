@@ -79,8 +79,9 @@ typedef struct dft3d_options_s {
  * reduced phases and rounded once to the stored float32 pieces.  The plan owns its
  * device tables and workspace (allocated on the current device during this call).
  *
- * Supported sizes: KDFT: every n_a a multiple of 64, n_a <= 8192.  FFT: every transformed n_a in
- * {256, 512, 1024, 2048} (N = R*R or 2*R*R with R = 16 or 32), the others multiples of 64.
+ * Supported sizes: KDFT: every n_a even, n_a <= 8192 (tiles that are not full are zero-filled on load
+ * and masked on store, the way the paper's compiler pads to its hardware's preferred shapes).  FFT: every
+ * transformed n_a in {256, 512, 1024, 2048} (N = R*R or 2*R*R with R = 16 or 32), the others multiples of 64.
  * Other sizes return DFT3D_ERR_UNSUPPORTED.
  */
 int dft3d_plan_create(dft3d_plan_t* out, long long n0, long long n1, long long n2, int mode, int sign,

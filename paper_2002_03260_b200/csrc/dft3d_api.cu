@@ -121,8 +121,10 @@ namespace {
 
 long long points(const dft3d_plan_s* p) { return p->n[0] * p->n[1] * p->n[2]; }
 
-int set_kernel_attributes() {
-  static bool done = false;
+// the opt-in to large dynamic shared memory is a per-device property of each kernel
+int set_kernel_attributes(int device) {
+  static bool done_on[64] = {false};
+  bool& done = done_on[device & 63];
   if (done) return DFT3D_OK;
   DFT3D_CUDA(cudaFuncSetAttribute(dft3d::kdft_axis_kernel<dft3d::KDFT_CONTIG>,
                                   cudaFuncAttributeMaxDynamicSharedMemorySize, int(dft3d::kKdftSmemBytes)));
@@ -149,7 +151,7 @@ int build_kdft_axis(dft3d_plan_s* p, int a, const double* nodes) {
   KdftAxis& ax = p->kax[a];
   const long long n = p->n[a];
   ax.n = n;
-  ax.bn = int(2 * n < 256 ? 2 * n : 256);
+  ax.bn = int(2 * n < 256 ? (2 * n + 15) / 16 * 16 : 256);   // MMA N: a multiple of 16, rows beyond 2n are zero-filled
   const bool scaled = (p->sign > 0) && !(p->flags & DFT3D_UNSCALED_INVERSE);
   const double scale = scaled ? 1.0 / double(n) : 1.0;
   std::vector<double> M;
@@ -183,7 +185,7 @@ int launch_kdft_strided(dft3d_plan_s* p, int a, const float* in, float* out, lon
   kp.chunk_kb = p->chunk_kb;
   kp.batches = batches;
   kp.C = C;
-  kp.lpb = int(C < 128 ? C : 128);
+  kp.lpb = C <= 64 ? 64 : 128;   // lanes of one batch in a tile; columns beyond C are zero-filled and masked
   kp.bpt = 128 / kp.lpb;
   kp.c_tiles = (C + kp.lpb - 1) / kp.lpb;
   kp.m_tiles = kp.c_tiles * ((batches + kp.bpt - 1) / kp.bpt);
@@ -382,6 +384,9 @@ int check_io(const dft3d_plan_s* p, const void* in, const void* out) {
   if (!in || !out) return fail(DFT3D_ERR_INVALID_ARG, "in/out must not be NULL");
   if ((reinterpret_cast<uintptr_t>(in) & 15) || (reinterpret_cast<uintptr_t>(out) & 15))
     return fail(DFT3D_ERR_INVALID_ARG, "in/out must be 16-byte aligned");
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev != p->device)
+    return fail(DFT3D_ERR_INVALID_ARG, "the plan was created on device %d but device %d is current", p->device, dev);
   const size_t bytes = size_t(points(p)) * 8;
   const char* a = static_cast<const char*>(in);
   const char* b = static_cast<const char*>(out);
@@ -472,7 +477,11 @@ int dft3d_plan_create_ex(dft3d_plan_t* out, long long n0, long long n1, long lon
   for (int a = 0; a < 3; ++a) {
     const bool transformed = (axes >> a) & 1u;
     if (a == 0 && !transformed) continue;   // a pure batch index
-    if (nn[a] % 64 != 0) return fail(DFT3D_ERR_UNSUPPORTED, "n%d = %lld is not a multiple of 64", a, nn[a]);
+    // KDFT: rows of the table and of the data must start on 16-byte boundaries (TMA), i.e. even lengths;
+    // FFT: the untransformed axes are split into groups of 16 lines
+    const long long quantum = (mode == DFT3D_KDFT) ? 2 : 64;
+    if (nn[a] % quantum != 0)
+      return fail(DFT3D_ERR_UNSUPPORTED, "n%d = %lld is not a multiple of %lld", a, nn[a], quantum);
     if (transformed && nn[a] > 8192) return fail(DFT3D_ERR_UNSUPPORTED, "n%d = %lld exceeds 8192", a, nn[a]);
   }
   if (mode == DFT3D_FFT && (nodes0 || nodes1 || nodes2))
@@ -504,7 +513,7 @@ int dft3d_plan_create_ex(dft3d_plan_t* out, long long n0, long long n1, long lon
       const int v = atoi(env);
       if (v >= 1) p->chunk_kb = v;
     }
-    if ((rc = set_kernel_attributes()) != DFT3D_OK) break;
+    if ((rc = set_kernel_attributes(p->device)) != DFT3D_OK) break;
     cudaError_t e = cudaMalloc(&p->d_status, sizeof(unsigned int));
     if (e == cudaSuccess) e = cudaMemset(p->d_status, 0, sizeof(unsigned int));
     if (e != cudaSuccess) { rc = fail(DFT3D_ERR_ALLOC, "cudaMalloc(status): %s", cudaGetErrorString(e)); break; }

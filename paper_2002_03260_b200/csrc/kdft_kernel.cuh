@@ -161,7 +161,7 @@ kdft_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_cons
   const uint32_t tmem = sh.tmem_base;
 
   const long long total_tiles = p.m_tiles * p.n_tiles;
-  const int num_kb = p.k2 / kBlockK;
+  const int num_kb = (p.k2 + kBlockK - 1) / kBlockK;   // a ragged last stage is zero-filled by TMA on both operands
   const uint32_t bytes_b = 2u * uint32_t(p.bn) * kBlockK * 4u;
 
   if (warp < 4) {
@@ -368,7 +368,8 @@ kdft_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_cons
           if (row < p.rows) {
             float4* dst = reinterpret_cast<float4*>(p.out + row * (long long)p.k2 + c0);
 #pragma unroll
-            for (int i = 0; i < 32; ++i) dst[i] = make_float4(acc[4 * i], acc[4 * i + 1], acc[4 * i + 2], acc[4 * i + 3]);
+            for (int i = 0; i < 32; ++i)
+              if (c0 + 4 * i < p.k2) dst[i] = make_float4(acc[4 * i], acc[4 * i + 1], acc[4 * i + 2], acc[4 * i + 3]);
           }
         } else {
           const long long ct = mt % p.c_tiles;
@@ -381,7 +382,7 @@ kdft_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_cons
             float* dst = p.out + 2 * ((batch * J + c0 / 2) * p.C + cc);
 #pragma unroll
             for (int i = 0; i < 64; ++i)
-              *reinterpret_cast<float2*>(dst + i * k_stride) = make_float2(acc[2 * i], acc[2 * i + 1]);
+              if (c0 / 2 + i < J) *reinterpret_cast<float2*>(dst + i * k_stride) = make_float2(acc[2 * i], acc[2 * i + 1]);
           }
         }
       }

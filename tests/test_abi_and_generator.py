@@ -49,7 +49,7 @@ def test_argument_validation_needs_no_gpu(dft):
     cases = [
         (dict(n=(0, 64, 64)), 1), (dict(n=(64, -64, 64)), 1), (dict(n=(64, 64, 64), mode=7), 1),
         (dict(n=(64, 64, 64), sign=0), 1), (dict(n=(64, 64, 64), flags=64), 1),
-        (dict(n=(64, 64, 100)), 2), (dict(n=(16384, 64, 64)), 2),
+        (dict(n=(64, 64, 101)), 2), (dict(n=(16384, 64, 64)), 2), (dict(n=(256, 256, 100), mode=1), 2),
         (dict(n=(64, 64, 64), nodes=(np.array([np.nan] * 64), None, None)), 1),
         (dict(n=(64, 64, 64), mode=1, nodes=(np.arange(64) / 64.0, None, None)), 2),
     ]
@@ -60,10 +60,10 @@ def test_argument_validation_needs_no_gpu(dft):
         assert e.value.status == status, (n, kw, str(e.value))
     # axis subsets: an untransformed axis 0 may have any length; the other axes still need multiples of 64
     with pytest.raises(dft.Dft3dError) as e:
-        dft.Plan(3, 100, 64, axes=(1, 2))
+        dft.Plan(3, 101, 64, axes=(1, 2))
     assert e.value.status == 2
     with pytest.raises(dft.Dft3dError) as e:
-        dft.Plan(3, 128, 64, axes=(0, 1, 2))
+        dft.Plan(3, 128, 64, axes=(0, 1, 2))      # axis 0 is transformed here: its length must be even
     assert e.value.status == 2
     import torch
     if not torch.cuda.is_available():

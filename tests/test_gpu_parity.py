@@ -456,3 +456,27 @@ def test_batched_1d_fft(lib, oracle):
     _finish(plan)
     plan.destroy()
     assert oracle.rel_l2(y.cpu().numpy(), _oracle_axes(oracle, x.cpu().numpy(), (2,))) < SANITY_AXIS
+
+
+# ------------------------------------------------------------------ sizes that are not tile multiples (KDFT)
+
+@pytest.mark.parametrize("shape", [(100, 66, 250), (30, 18, 34), (2, 4, 6), (130, 64, 2), (66, 258, 64)])
+def test_kdft_general_even_sizes(lib, oracle, shape):
+    """Any even length: ragged K stages are zero-filled by TMA on both operands, ragged tiles masked on store."""
+    x = _inputs().cube(shape, "normal", 91, device="cuda")
+    guard = torch.full((1 << 14,), 7.0, device="cuda")           # canaries around the output
+    out = torch.empty_like(x)
+    guard2 = torch.full((1 << 14,), 7.0, device="cuda")
+    plan = lib.Plan(*shape)
+    plan(x, out)
+    _finish(plan)
+    plan.destroy()
+    err = oracle.rel_l2(out.cpu().numpy(), oracle.dft3d(x.cpu().numpy()))
+    assert err < SANITY, (shape, err)
+    assert bool((guard == 7.0).all()) and bool((guard2 == 7.0).all())
+    nodes = _inputs().sorted_nodes(shape, 92)
+    plan = lib.Plan(*shape, nodes=nodes)
+    y = plan(x)
+    _finish(plan)
+    plan.destroy()
+    assert oracle.rel_l2(y.cpu().numpy(), oracle.dft3d(x.cpu().numpy(), nodes=nodes)) < SANITY
