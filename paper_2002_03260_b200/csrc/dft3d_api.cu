@@ -56,14 +56,14 @@ int get_encoder(EncodeTiledFn* fn) {
   return DFT3D_OK;
 }
 
-// float32 tensor map with up to 3 dimensions; dims/box innermost first; strides in bytes for dims 1..rank-1
+// float32 tensor map with up to 4 dimensions; dims/box innermost first; strides in bytes for dims 1..rank-1
 int encode_f32(CUtensorMap* map, const void* base, int rank, const unsigned long long* dims,
                const unsigned long long* strides_bytes, const unsigned* box, int swizzle_bytes) {
   EncodeTiledFn enc;
   int rc = get_encoder(&enc);
   if (rc != DFT3D_OK) return rc;
-  cuuint64_t d[3], s[2];
-  cuuint32_t b[3], es[3];
+  cuuint64_t d[4], s[3];
+  cuuint32_t b[4], es[4];
   for (int i = 0; i < rank; ++i) { d[i] = dims[i]; b[i] = box[i]; es[i] = 1; }
   for (int i = 0; i + 1 < rank; ++i) s[i] = strides_bytes[i];
   CUresult cr = enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, rank, const_cast<void*>(base), d, s, b, es,
@@ -130,18 +130,25 @@ int set_kernel_attributes(int device) {
                                   cudaFuncAttributeMaxDynamicSharedMemorySize, int(dft3d::kKdftSmemBytes)));
   DFT3D_CUDA(cudaFuncSetAttribute(dft3d::kdft_axis_kernel<dft3d::KDFT_STRIDED>,
                                   cudaFuncAttributeMaxDynamicSharedMemorySize, int(dft3d::kKdftSmemBytes)));
-#define DFT3D_FFT_ATTR(MODE, R, RX, COLS, NB2)                                                                \
-  DFT3D_CUDA(cudaFuncSetAttribute(dft3d::fft_axis_kernel<MODE, R, RX, COLS, NB2>,                              \
+#define DFT3D_FFT_ATTR(MODE, R, RX, COLS, NB2, SO)                                                            \
+  DFT3D_CUDA(cudaFuncSetAttribute(dft3d::fft_axis_kernel<MODE, R, RX, COLS, NB2, SO>,                          \
                                   cudaFuncAttributeMaxDynamicSharedMemorySize, int(dft3d::fft_smem_bytes(R, NB2))))
-  DFT3D_FFT_ATTR(dft3d::FFT_CONTIG, 32, 1, 16, 2);
-  DFT3D_FFT_ATTR(dft3d::FFT_CONTIG, 16, 1, 16, 2);
-  DFT3D_FFT_ATTR(dft3d::FFT_CONTIG, 32, 2, 16, 2);
-  DFT3D_FFT_ATTR(dft3d::FFT_CONTIG, 16, 2, 16, 2);
-  DFT3D_FFT_ATTR(dft3d::FFT_STRIDED, 32, 1, 16, 1);
-  DFT3D_FFT_ATTR(dft3d::FFT_STRIDED, 32, 1, 8, 2);
-  DFT3D_FFT_ATTR(dft3d::FFT_STRIDED, 16, 1, 16, 2);
-  DFT3D_FFT_ATTR(dft3d::FFT_STRIDED, 32, 2, 8, 1);
-  DFT3D_FFT_ATTR(dft3d::FFT_STRIDED, 16, 2, 16, 2);
+  DFT3D_FFT_ATTR(dft3d::FFT_CONTIG, 32, 1, 16, 2, 0);
+  DFT3D_FFT_ATTR(dft3d::FFT_CONTIG, 16, 1, 16, 2, 0);
+  DFT3D_FFT_ATTR(dft3d::FFT_CONTIG, 32, 2, 16, 2, 0);
+  DFT3D_FFT_ATTR(dft3d::FFT_CONTIG, 16, 2, 16, 2, 0);
+  DFT3D_FFT_ATTR(dft3d::FFT_STRIDED, 32, 1, 16, 1, 0);
+  DFT3D_FFT_ATTR(dft3d::FFT_STRIDED, 32, 1, 8, 2, 0);
+  DFT3D_FFT_ATTR(dft3d::FFT_STRIDED, 16, 1, 16, 2, 0);
+  DFT3D_FFT_ATTR(dft3d::FFT_STRIDED, 32, 2, 8, 1, 0);
+  DFT3D_FFT_ATTR(dft3d::FFT_STRIDED, 16, 2, 16, 2, 0);
+  DFT3D_FFT_ATTR(dft3d::FFT_STRIDED, 32, 1, 16, 1, 1);
+  DFT3D_FFT_ATTR(dft3d::FFT_STRIDED, 32, 1, 8, 1, 0);
+  DFT3D_FFT_ATTR(dft3d::FFT_STRIDED, 32, 1, 8, 1, 1);
+  DFT3D_FFT_ATTR(dft3d::FFT_STRIDED, 32, 1, 8, 2, 1);
+  DFT3D_FFT_ATTR(dft3d::FFT_STRIDED, 16, 1, 16, 2, 1);
+  DFT3D_FFT_ATTR(dft3d::FFT_STRIDED, 32, 2, 8, 1, 1);
+  DFT3D_FFT_ATTR(dft3d::FFT_STRIDED, 16, 2, 16, 2, 1);
 #undef DFT3D_FFT_ATTR
   done = true;
   return DFT3D_OK;
@@ -303,18 +310,34 @@ int build_fft_axis(dft3d_plan_s* p, int a, const int split[2]) {
   return encode_f32(&ax.map_w, ax.d_w, 2, dims, strides, box, 128);
 }
 
-int fft_axis_pass(dft3d_plan_s* p, int axis, const float* in, float* out, cudaStream_t stream) {
+// layout: 0 = `in` and `out` in the natural [n0][n1][n2] order.
+//         1 = axis 0 only: `out` receives the blocked order T[column tile][k0][cols] (one contiguous block per stage)
+//         2 = axis 1 only: `in` is in that blocked order (written by a layout-1 pass), `out` natural
+// The blocked order exists because a pass along axis 0 touches rows that are n1*n2*8 bytes apart: reading them
+// piecewise is cheap, writing them piecewise is not (1024^3: 3.7 ms without the stores, 9-11 ms with them).
+enum { FFT_NATURAL = 0, FFT_OUT_BLOCKED = 1, FFT_IN_BLOCKED = 2 };
+
+int fft_cols_for(const dft3d_plan_s* p, int axis, int layout) {
   const FftAxis& ax = p->fax[axis];
-  const int R = ax.R, RX = ax.RX, N = int(ax.n), Lg = 128 / (R * RX);
   int cols = ax.cols;
-  if (axis != 2 && R == 32 && RX == 1) {
+  if (axis != 2 && ax.R == 32 && ax.RX == 1) {
     // 1024-point strided axes: 16 lines per stage (128-byte rows) leave room for one stage-2 operand buffer only;
     // 8 lines per stage (64-byte rows) allow two.  Rows far apart (large strides) favour the wider rows.
     const long long C = (axis == 0) ? p->n[1] * p->n[2] : p->n[2];
-    const char* env = getenv("DFT3D_FFT_COLS");
-    cols = env ? atoi(env) : ((C * 8 >= (1ll << 20)) ? 16 : 8);
+    const char* env = getenv(axis == 0 ? "DFT3D_FFT_COLS0" : "DFT3D_FFT_COLS1");
+    if (!env) env = getenv("DFT3D_FFT_COLS");
+    // measured at 1024^3: natural layout, rows >= 1 MiB apart: 16; otherwise (close rows, or the blocked layout
+    // where every stage is one contiguous block) 8-line stages, which leave room to load the next stage early
+    cols = env ? atoi(env) : ((layout == FFT_NATURAL && C * 8 >= (1ll << 20)) ? 16 : 8);
     if (cols != 8 && cols != 16) cols = 16;
   }
+  return cols;
+}
+
+int fft_axis_pass(dft3d_plan_s* p, int axis, const float* in, float* out, cudaStream_t stream, int layout = FFT_NATURAL) {
+  const FftAxis& ax = p->fax[axis];
+  const int R = ax.R, RX = ax.RX, N = int(ax.n), Lg = 128 / (R * RX);
+  const int cols = fft_cols_for(p, axis, layout);
   dft3d::FftParams fp;
   memset(&fp, 0, sizeof(fp));
   fp.N = N;
@@ -323,8 +346,9 @@ int fft_axis_pass(dft3d_plan_s* p, int axis, const float* in, float* out, cudaSt
   fp.profile = p->d_profile;
   fp.out = out;
   fp.status = p->d_status;
-  CUtensorMap map_data;
+  CUtensorMap map_data, map_out;
   int rc;
+  int stage_out = 0;
   if (axis == 2) {
     const long long rows = p->n[0] * p->n[1];
     fp.rows = rows;
@@ -335,6 +359,7 @@ int fft_axis_pass(dft3d_plan_s* p, int axis, const float* in, float* out, cudaSt
     const unsigned long long strides[2] = {1024ull, (unsigned long long)N * 8ull};
     const unsigned box[3] = {256u, unsigned(N / 128), unsigned(Lg)};
     rc = encode_f32(&map_data, in, 3, dims, strides, box, 0);
+    map_out = map_data;   // unused on this axis
   } else {
     const long long batches = (axis == 0) ? 1 : p->n[0];
     const long long C = (axis == 0) ? p->n[1] * p->n[2] : p->n[2];
@@ -352,27 +377,70 @@ int fft_axis_pass(dft3d_plan_s* p, int axis, const float* in, float* out, cudaSt
     const unsigned long long dims[3] = {(unsigned long long)(2 * C), (unsigned long long)N, (unsigned long long)batches};
     const unsigned long long strides[2] = {(unsigned long long)(C * 8), (unsigned long long)N * C * 8ull};
     const unsigned box[3] = {unsigned(2 * cols), 256u, 1u};
-    rc = encode_f32(&map_data, in, 3, dims, strides, box, cols * 8);
+    if (layout == FFT_IN_BLOCKED) {
+      // `in` = T[tile][k0][colsA] written by the axis-0 pass; this stage is (k0 = batch, n2 tile) and its rows are n1
+      const int colsA = fft_cols_for(p, 0, FFT_OUT_BLOCKED);
+      const long long n0 = p->n[0], n1 = p->n[1], n2 = p->n[2];
+      const unsigned long long bdims[4] = {(unsigned long long)(2 * colsA), (unsigned long long)n0,
+                                           (unsigned long long)(n2 / colsA), (unsigned long long)n1};
+      const unsigned long long bstr[3] = {(unsigned long long)(colsA * 8), (unsigned long long)(n0 * colsA * 8),
+                                          (unsigned long long)(n2 * n0 * 8)};
+      const unsigned bbox[4] = {unsigned(2 * cols), 1u, 1u, 256u};
+      rc = encode_f32(&map_data, in, 4, bdims, bstr, bbox, cols * 8);
+      fp.in_blocked = 1;
+      fp.blk_ratio = colsA / cols;
+      fp.l2_prefetch = 0;
+    } else {
+      rc = encode_f32(&map_data, in, 3, dims, strides, box, cols * 8);
+    }
+    if (layout == FFT_OUT_BLOCKED) {
+      const unsigned long long bdims[3] = {(unsigned long long)(2 * cols), (unsigned long long)N, (unsigned long long)(C / cols)};
+      const unsigned long long bstr[2] = {(unsigned long long)(cols * 8), (unsigned long long)N * cols * 8ull};
+      if (rc == DFT3D_OK) rc = encode_f32(&map_out, out, 3, bdims, bstr, box, cols * 8);
+      fp.out_blocked = 1;
+      stage_out = 1;
+    } else {
+      if (rc == DFT3D_OK) rc = encode_f32(&map_out, out, 3, dims, strides, box, cols * 8);
+      // rows MiBs apart: send the results out as full rows through TMA stores instead of 32-byte pieces
+      const char* env = getenv("DFT3D_FFT_STAGE_OUT");
+      stage_out = env ? atoi(env) : (C * 8 >= (1ll << 20) ? 1 : 0);
+    }
   }
   if (rc != DFT3D_OK) return rc;
-  const int nb2 = (axis == 2 || R == 16 || (R == 32 && RX == 1 && cols == 8)) ? 2 : 1;
+  int nb2 = (axis == 2 || R == 16 || (R == 32 && RX == 1 && cols == 8)) ? 2 : 1;
+  if (axis != 2 && R == 32 && RX == 1 && cols == 8) {
+    // 8-line stages: two stage-2 operand buffers and one raw stage (best with direct stores), or one operand
+    // buffer and two raw stages (best when the results return through the raw stage, which then stays busy longer)
+    const char* env = getenv("DFT3D_FFT_NB2");
+    nb2 = env ? atoi(env) : (layout != FFT_NATURAL ? 1 : 2);
+    if (nb2 != 1 && nb2 != 2) nb2 = 2;
+  }
   fp.raw_stages = dft3d::fft_raw_bytes(R, nb2) / fp.stage_bytes;
   if (fp.raw_stages > 4) fp.raw_stages = 4;
   const int grid = int(fp.num_stages < p->sm_count ? fp.num_stages : p->sm_count);
   const size_t smem = dft3d::fft_smem_bytes(R, nb2);
-#define DFT3D_FFT_LAUNCH(MODE, R_, RX_, COLS_, NB2_)                                                          \
-  dft3d::fft_axis_kernel<MODE, R_, RX_, COLS_, NB2_><<<grid, dft3d::kFftThreads, smem, stream>>>(map_data, ax.map_w, fp)
+#define DFT3D_FFT_LAUNCH(MODE, R_, RX_, COLS_, NB2_, SO_)                                                     \
+  dft3d::fft_axis_kernel<MODE, R_, RX_, COLS_, NB2_, SO_>                                                      \
+      <<<grid, dft3d::kFftThreads, smem, stream>>>(map_data, ax.map_w, map_out, fp)
   if (axis == 2) {
-    if (R == 32 && RX == 1) DFT3D_FFT_LAUNCH(dft3d::FFT_CONTIG, 32, 1, 16, 2);
-    else if (R == 16 && RX == 1) DFT3D_FFT_LAUNCH(dft3d::FFT_CONTIG, 16, 1, 16, 2);
-    else if (R == 32) DFT3D_FFT_LAUNCH(dft3d::FFT_CONTIG, 32, 2, 16, 2);
-    else DFT3D_FFT_LAUNCH(dft3d::FFT_CONTIG, 16, 2, 16, 2);
+    if (R == 32 && RX == 1) DFT3D_FFT_LAUNCH(dft3d::FFT_CONTIG, 32, 1, 16, 2, 0);
+    else if (R == 16 && RX == 1) DFT3D_FFT_LAUNCH(dft3d::FFT_CONTIG, 16, 1, 16, 2, 0);
+    else if (R == 32) DFT3D_FFT_LAUNCH(dft3d::FFT_CONTIG, 32, 2, 16, 2, 0);
+    else DFT3D_FFT_LAUNCH(dft3d::FFT_CONTIG, 16, 2, 16, 2, 0);
+  } else if (!stage_out) {
+    if (R == 32 && RX == 1 && cols == 16) DFT3D_FFT_LAUNCH(dft3d::FFT_STRIDED, 32, 1, 16, 1, 0);
+    else if (R == 32 && RX == 1 && nb2 == 1) DFT3D_FFT_LAUNCH(dft3d::FFT_STRIDED, 32, 1, 8, 1, 0);
+    else if (R == 32 && RX == 1) DFT3D_FFT_LAUNCH(dft3d::FFT_STRIDED, 32, 1, 8, 2, 0);
+    else if (R == 16 && RX == 1) DFT3D_FFT_LAUNCH(dft3d::FFT_STRIDED, 16, 1, 16, 2, 0);
+    else if (R == 32) DFT3D_FFT_LAUNCH(dft3d::FFT_STRIDED, 32, 2, 8, 1, 0);
+    else DFT3D_FFT_LAUNCH(dft3d::FFT_STRIDED, 16, 2, 16, 2, 0);
   } else {
-    if (R == 32 && RX == 1 && cols == 16) DFT3D_FFT_LAUNCH(dft3d::FFT_STRIDED, 32, 1, 16, 1);
-    else if (R == 32 && RX == 1) DFT3D_FFT_LAUNCH(dft3d::FFT_STRIDED, 32, 1, 8, 2);
-    else if (R == 16 && RX == 1) DFT3D_FFT_LAUNCH(dft3d::FFT_STRIDED, 16, 1, 16, 2);
-    else if (R == 32) DFT3D_FFT_LAUNCH(dft3d::FFT_STRIDED, 32, 2, 8, 1);
-    else DFT3D_FFT_LAUNCH(dft3d::FFT_STRIDED, 16, 2, 16, 2);
+    if (R == 32 && RX == 1 && cols == 16) DFT3D_FFT_LAUNCH(dft3d::FFT_STRIDED, 32, 1, 16, 1, 1);
+    else if (R == 32 && RX == 1 && nb2 == 1) DFT3D_FFT_LAUNCH(dft3d::FFT_STRIDED, 32, 1, 8, 1, 1);
+    else if (R == 32 && RX == 1) DFT3D_FFT_LAUNCH(dft3d::FFT_STRIDED, 32, 1, 8, 2, 1);
+    else if (R == 16 && RX == 1) DFT3D_FFT_LAUNCH(dft3d::FFT_STRIDED, 16, 1, 16, 2, 1);
+    else if (R == 32) DFT3D_FFT_LAUNCH(dft3d::FFT_STRIDED, 32, 2, 8, 1, 1);
+    else DFT3D_FFT_LAUNCH(dft3d::FFT_STRIDED, 16, 2, 16, 2, 1);
   }
 #undef DFT3D_FFT_LAUNCH
   DFT3D_CUDA(cudaGetLastError());
@@ -551,6 +619,15 @@ int dft3d_plan_create_ex(dft3d_plan_t* out, long long n0, long long n1, long lon
       for (int a = 0; a < 3 && rc == DFT3D_OK; ++a)
         if ((axes >> a) & 1u) rc = build_fft_axis(p, a, opt.fft_split[a]);
       if (rc != DFT3D_OK) break;
+      // a cube of workspace, if it fits the limit, lets the axis-0 pass avoid piecewise writes to far-apart rows;
+      // without it the three passes run in place on `out`
+      const size_t cube_bytes = size_t(n0) * n1 * n2 * 8;
+      const size_t limit = opt.workspace_limit ? opt.workspace_limit : (size_t(16) << 30);
+      if (axes == 7u && cube_bytes <= limit && fft_cols_for(p, 0, FFT_OUT_BLOCKED) % fft_cols_for(p, 1, FFT_IN_BLOCKED) == 0) {
+        e = cudaMalloc(&p->workspace, cube_bytes);
+        if (e == cudaSuccess) p->workspace_bytes = cube_bytes;
+        else { p->workspace = nullptr; (void)cudaGetLastError(); }   // fall back to the in-place schedule
+      }
     }
   } while (0);
   if (rc != DFT3D_OK) {
@@ -617,6 +694,14 @@ int dft3d_execute(dft3d_plan_t p, const void* in, void* out, void* cuda_stream) 
   }
   // FFT: the first transformed axis (last axis first) in -> out, the others in place on out (a CTA loads a group of
   // lines completely into shared memory before it stores any of their results, and groups are disjoint)
+  if (axes == 7u && p->workspace && !getenv("DFT3D_FFT_INPLACE")) {
+    // with a cube of workspace: axis 0 in -> out (blocked order: its far-apart rows are only read, never written
+    // piecewise), axis 1 out -> workspace (natural order), axis 2 workspace -> out
+    float* ws = static_cast<float*>(p->workspace);
+    if ((rc = fft_axis_pass(p, 0, fin, fout, stream, FFT_OUT_BLOCKED)) != DFT3D_OK) return rc;
+    if ((rc = fft_axis_pass(p, 1, fout, ws, stream, FFT_IN_BLOCKED)) != DFT3D_OK) return rc;
+    return fft_axis_pass(p, 2, ws, fout, stream);
+  }
   const float* src = fin;
   for (int a = 2; a >= 0; --a) {
     if (!((axes >> a) & 1u)) continue;

@@ -42,6 +42,10 @@ enum : int { FFT_CONTIG = 0, FFT_STRIDED = 1 };
 
 constexpr int kFftThreads = 640;      // 5 warp groups: {producer, 2 MMA issuers}, split, drain 1 (x2), drain 2
 // STRIDED stages hold COLS neighbouring lines: 16 (128-byte rows, 128B swizzle) or 8 (64-byte rows, 64B swizzle)
+// STAGE_OUT (STRIDED only): results go back into the raw stage they came from (each M-tile owns its columns there) and
+//   leave as full rows through TMA stores, instead of 32-byte pieces from registers; pays off when the rows are so far
+//   apart that every piece costs an address translation (1024^3 axis 0: 11.0 ms with direct stores, 3.7 ms without
+//   any stores)
 // NB2 = buffers of the stage-2 operand (2 lets drain 1 write the next M-tile while stage 2 still reads this one)
 constexpr int kFftTmemD1 = 0, kFftTmemD2 = 128, kFftTmemA1 = 256;   // tensor-memory column map (A1: two buffers of 128)
 
@@ -57,6 +61,11 @@ struct FftParams {
   long long C;
   long long c_tiles;     // C / COLS
   int l2_prefetch;       // STRIDED: prefetch the next stage's rows into L2
+  // Blocked intermediate layout T[column tile][row][COLS] (one contiguous block per stage), used between the axis-0
+  // and the axis-1 pass of a 3D transform so that the far-apart rows of axis 0 are only ever READ piecewise:
+  int out_blocked;       // STAGE_OUT: store the stage as block number `column tile` of T (map_out is T's 3D map)
+  int blk_ratio;         // in_blocked: columns of a block of T / COLS of this pass
+  int in_blocked;        // load rows from T through a 4D map {COLS, row-in-block, tile, block row}; batch = row-in-block
   const float2* twiddle; // [R][R] complex64, T[k1][beta] (times 1/RX for a scaled inverse)
   const float2* twiddle2;// RX == 2: [R*R] complex64, exp(s*2*pi*i*m/N)
   float* out;
@@ -71,6 +80,7 @@ struct FftShared {
   uint64_t a2_full[2], a2_empty[2];
   uint64_t d2_full, d2_empty;
   uint64_t w_full;
+  uint64_t out_ready;      // STAGE_OUT: the four drain-2 warps have written the stage's last M-tile
   uint32_t tmem_base;
   volatile int abort_flag;
 };
@@ -112,10 +122,10 @@ __host__ __device__ constexpr size_t fft_smem_bytes(int R, int NB2) {
     FFT_PROF_END(code)                                                                    \
   }
 
-template <int MODE, int R, int RX, int COLS, int NB2>
+template <int MODE, int R, int RX, int COLS, int NB2, int STAGE_OUT>
 __global__ void __launch_bounds__(kFftThreads, 1)
 fft_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_constant__ CUtensorMap map_w,
-                const FftParams p) {
+                const __grid_constant__ CUtensorMap map_out, const FftParams p) {
   extern __shared__ uint8_t smem_raw_[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw_) + 1023) & ~uintptr_t(1023));
   constexpr int K = 2 * R;             // reals per contraction
@@ -140,7 +150,11 @@ fft_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_const
   constexpr int kRowBytes = COLS * 8;  // STRIDED: bytes of one row of a raw stage
 
   if (tid == 0) {
-    for (int i = 0; i < 4; ++i) { ptx::mbar_init(&sh.raw_full[i], 1); ptx::mbar_init(&sh.raw_empty[i], 4 * p.mtiles_per_stage); }
+    for (int i = 0; i < 4; ++i) {
+      ptx::mbar_init(&sh.raw_full[i], 1);
+      ptx::mbar_init(&sh.raw_empty[i], 4 * p.mtiles_per_stage + (STAGE_OUT ? 1 : 0));
+    }
+    ptx::mbar_init(&sh.out_ready, 4);
     for (int i = 0; i < 2; ++i) { ptx::mbar_init(&sh.a1_full[i], 4); ptx::mbar_init(&sh.a1_empty[i], 1); }
     ptx::mbar_init(&sh.d1_full, 1); ptx::mbar_init(&sh.d1_empty, 4 * (K / 32));
     for (int i = 0; i < 2; ++i) { ptx::mbar_init(&sh.a2_full[i], 4 * (K / 32)); ptx::mbar_init(&sh.a2_empty[i], 1); }
@@ -185,8 +199,13 @@ fft_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_const
           ptx::tma_load_3d(dst, &map_data, &sh.raw_full[s], 0, 0, int(sidx * Lg));
         } else {
           const long long ct = sidx % p.c_tiles, bt = sidx / p.c_tiles;
-          for (int r0 = 0; r0 < p.N; r0 += 256)
-            ptx::tma_load_3d(dst + size_t(r0) * kRowBytes, &map_data, &sh.raw_full[s], int(ct * 2 * COLS), r0, int(bt));
+          for (int r0 = 0; r0 < p.N; r0 += 256) {
+            if (p.in_blocked)
+              ptx::tma_load_4d(dst + size_t(r0) * kRowBytes, &map_data, &sh.raw_full[s],
+                               int(ct % p.blk_ratio) * 2 * COLS, int(bt), int(ct / p.blk_ratio), r0);
+            else
+              ptx::tma_load_3d(dst + size_t(r0) * kRowBytes, &map_data, &sh.raw_full[s], int(ct * 2 * COLS), r0, int(bt));
+          }
           // the ring is short on the strided axes (one or two stages), so the loads of the next stage cannot be
           // issued yet; pull its rows into L2 meanwhile (rows are far apart: this also absorbs the TLB misses)
           const long long nidx = sidx + gridDim.x;
@@ -406,8 +425,9 @@ fft_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_const
     const int k1 = (MODE == FFT_CONTIG) ? m % R : m / SL;
     const int g = sl / RX, bsel = sl % RX;
     const uint32_t lane_addr = tmem + (uint32_t(q * 32) << 16) + kFftTmemD2;
-    long long t = 0;
-    for (long long sidx = blockIdx.x; sidx < p.num_stages; sidx += gridDim.x) {
+    long long t = 0, istage = 0;
+    for (long long sidx = blockIdx.x; sidx < p.num_stages; sidx += gridDim.x, ++istage) {
+      uint8_t* stage = smem_rawring + size_t(istage % p.raw_stages) * p.stage_bytes;   // STAGE_OUT: results return here
       for (int mt = 0; mt < p.mtiles_per_stage; ++mt, ++t) {
         float2* dst;              // &out[line][RX*k1 + bsel]; output k = RX*(k1 + R*k2) + bsel is k2*k2_stride further
         long long k2_stride;
@@ -436,7 +456,17 @@ fft_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_const
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(&sh.d2_empty);
           }
-          if (ok) {
+          if (STAGE_OUT) {
+            // element (row k, column c) of the stage, in the layout TMA wrote the input in (same swizzle)
+            const int c = mt * Lg + g;
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              const int k = RX * (k1 + R * (ch * 16 + j)) + bsel;
+              const uint32_t swz = (COLS == 16) ? uint32_t(k & 7) : uint32_t((k >> 1) & 3);
+              const uint32_t off = uint32_t(k) * kRowBytes + ((uint32_t(c >> 1) ^ swz) << 4) + uint32_t(c & 1) * 8u;
+              *reinterpret_cast<uint2*>(stage + off) = make_uint2(v0[2 * j], v0[2 * j + 1]);
+            }
+          } else if (ok) {
             float2* pd = dst + (long long)(ch * 16) * k2_stride;
 #pragma unroll
             for (int j = 0; j < 16; ++j) {
@@ -447,7 +477,31 @@ fft_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_const
           }
         }
       }
+      if (STAGE_OUT) {
+        // all M-tiles of the stage are back in shared memory: one thread sends the rows out and, once the copy
+        // engine has read them, hands the stage to the producer for the next load
+        ptx::fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(&sh.out_ready);
+        if (warp == 16) {
+          FFT_WAIT_WARP(&sh.out_ready, uint32_t(istage) & 1, 0x902);
+          if (lane == 0) {
+            const long long ct = sidx % p.c_tiles, bt = sidx / p.c_tiles;
+            for (int r0 = 0; r0 < p.N; r0 += 256) {
+              if (p.out_blocked)
+                ptx::tma_store_3d(&map_out, stage + size_t(r0) * kRowBytes, 0, r0, int(ct));
+              else
+                ptx::tma_store_3d(&map_out, stage + size_t(r0) * kRowBytes, int(ct * 2 * COLS), r0, int(bt));
+            }
+            ptx::tma_store_commit();
+            ptx::tma_store_wait_read();
+            ptx::mbar_arrive(&sh.raw_empty[istage % p.raw_stages]);
+          }
+          __syncwarp();
+        }
+      }
     }
+    if (STAGE_OUT && warp == 16 && lane == 0) ptx::tma_store_wait_all();
   }
 
 role_done:

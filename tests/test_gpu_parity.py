@@ -219,6 +219,22 @@ def test_fft_256_forward_inverse_and_kdft_agreement(lib, oracle):
         p.destroy()
 
 
+def test_fft_schedules_agree(lib, oracle):
+    """With a cube of workspace the 3D FFT goes in -> out (blocked order) -> workspace -> out; without it the
+    three passes run in place on out.  Both against the oracle."""
+    shape = (256, 512, 256)
+    x = _inputs().cube(shape, "normal", 66, device="cuda")
+    ref = oracle.dft3d(x.cpu().numpy())
+    with_ws = lib.Plan(*shape, mode=lib.DFT3D_FFT)
+    in_place = lib.Plan(*shape, mode=lib.DFT3D_FFT, workspace_limit=1 << 20)
+    assert with_ws.workspace_bytes == x.numel() * 8 and in_place.workspace_bytes == 0
+    for plan in (with_ws, in_place):
+        y = plan(x)
+        _finish(plan)
+        assert oracle.rel_l2(y.cpu().numpy(), ref) < SANITY
+        plan.destroy()
+
+
 def test_fft_mixed_axis_lengths(lib, oracle):
     shape = (256, 1024, 256)
     x = _inputs().cube(shape, "normal", 63, device="cuda")
