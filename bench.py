@@ -54,7 +54,7 @@ def conv_flops(n):
 # points of that launch; smaller cases than the bench workload, traffic grows in proportion to the points):
 #   profiles/fft_axis_kernel_256x1024x1024.md : (2.148 + 2.094) GB / 268.4 M points
 #   profiles/kdft_axis_kernel_512.md          : (1.084 + 1.035) GB / 134.2 M points
-NCU_DRAM_BYTES_PER_POINT = {"fft_axis_kernel": 15.80, "kdft_axis_kernel": 15.79}
+NCU_DRAM_BYTES_PER_POINT = {"fft_axis_kernel": 15.80, "kdft_axis_kernel": 15.79, "kdft_f16_axis_kernel": 15.79}
 
 
 def measured_peaks():
@@ -219,7 +219,9 @@ def main():
     if mode == "fft" and not args.no_kdft:
         ksteps = max(1, min(args.steps, 3))
         kplan, kms, kclk = time_mode("kdft", ksteps, 3, True)
-        kdft_info = {"ms_per_step": kms, "steps": ksteps, "warmup": 3, "launches_per_step": kplan.launches, "clocks": kclk}
+        kdft_info = {"ms_per_step": kms, "steps": ksteps, "warmup": 3, "launches_per_step": kplan.launches,
+                     "split": "fp16" if kplan.split == dft.DFT3D_SPLIT_FP16 else "tf32", "clocks": kclk}
+        ksplit = kplan.split
         kplan.destroy()
 
     # ---- end to end through the host-buffer entry point
@@ -248,22 +250,30 @@ def main():
         P = float(shape[0]) * shape[1] * shape[2]
         nsum = float(sum(shape))
 
-        def kdft_roofline(ms, nlaunch):
-            # only kernel: kdft_axis_kernel.  Algorithmic flops per point per axis = 8*n_a (4 real multiply-adds per
-            # complex MAC); the tensor cores issue them three times (TF32 split: hi*hi, lo*hi, hi*lo).
+        def kdft_roofline(ms, nlaunch, split):
+            # dominant kernel: the KDFT axis kernel (the fp16 split adds one small reduction over the input).
+            # Algorithmic flops per point per axis = 8*n_a (4 real multiply-adds per complex MAC); the tensor cores
+            # issue them three times (split products hi*hi, lo*hi, hi*lo).
             algo_flops = 8.0 * nsum * P
             issued = 3.0 * algo_flops
-            tf32_peak = peaks["bf16_tflops_sustained"] * (1.1 / 2.25)
             ach = issued / (ms * 1e-3) * 1e-12
-            return {"bound": "tensor", "kernel": "kdft_axis_kernel", "achieved": ach, "peak": tf32_peak, "unit": "TFLOP/s",
-                    "frac": ach / tf32_peak, "traffic": NCU_DRAM_BYTES_PER_POINT["kdft_axis_kernel"] * P,
+            if split == dft.DFT3D_SPLIT_FP16:
+                kernel, peak = "kdft_f16_axis_kernel", peaks["bf16_tflops_sustained"]
+                src = "%s bf16 sustained (fp16 and bf16 share the tensor rate)" % peak_kind
+                axis_launches = nlaunch - 1
+            else:
+                kernel, peak = "kdft_axis_kernel", peaks["bf16_tflops_sustained"] * (1.1 / 2.25)
+                src = "%s bf16 sustained x nominal TF32/bf16 ratio (1.1/2.25)" % peak_kind
+                axis_launches = nlaunch
+            return {"bound": "tensor", "kernel": kernel, "achieved": ach, "peak": peak, "unit": "TFLOP/s",
+                    "frac": ach / peak, "traffic": NCU_DRAM_BYTES_PER_POINT[kernel] * P,
                     "traffic_note": "DRAM bytes per launch, ncu capture at 512^3 scaled by points (algorithmic: 16 B/point)",
-                    "peak_source": "%s bf16 sustained x nominal TF32/bf16 ratio (1.1/2.25)" % peak_kind,
-                    "flops": "issued TF32 tensor flops = 3 split products x 8*n_a flops per point per axis",
-                    "useful_gemm_tflops": algo_flops / (ms * 1e-3) * 1e-12, "avg_launch_ms": ms / nlaunch}
+                    "peak_source": src,
+                    "flops": "issued tensor flops = 3 split products x 8*n_a flops per point per axis",
+                    "useful_gemm_tflops": algo_flops / (ms * 1e-3) * 1e-12, "avg_launch_ms": ms / axis_launches}
 
         if mode == "kdft":
-            roofline = kdft_roofline(ms_step, launches)
+            roofline = kdft_roofline(ms_step, launches, plan.split)
         else:
             # only kernel: fft_axis_kernel, one launch per axis; algorithmic traffic 16 B per point per axis
             algo_bytes = 3 * 16.0 * P
@@ -277,7 +287,7 @@ def main():
         if kdft_info is not None:
             kdft_info["value"] = world * conv_flops(shape) / kdft_info["ms_per_step"] * 1e-6
             kdft_info["unit"] = "GFLOP/s"
-            kdft_info["roofline"] = kdft_roofline(kdft_info["ms_per_step"], kdft_info["launches_per_step"])
+            kdft_info["roofline"] = kdft_roofline(kdft_info["ms_per_step"], kdft_info["launches_per_step"], ksplit)
         cpu = None
         if not args.no_cpu_baseline:
             planes = max(1, min(n, int(3.0e10 / (float(n) ** 3))))

@@ -48,12 +48,20 @@ enum {
   DFT3D_NODES_ON_OUTPUT = 1u,   /* M[k,j] = exp(s*2*pi*i * node[k] * j): Eq. 1 read literally (arbitrary
                                    evaluation points, integer powers).  Default is M[k,j] = exp(s*2*pi*i * k * node[j])
                                    (nonuniform input samples, integer output frequencies). */
-  DFT3D_UNSCALED_INVERSE = 2u   /* sign=+1 without the 1/n_a factors */
+  DFT3D_UNSCALED_INVERSE = 2u,  /* sign=+1 without the 1/n_a factors */
+  /* KDFT operand split (the "decompose and accumulate" of Section II-A).  Both use 3 products of 11-bit pieces with
+     fp32 accumulation and meet the same error bound.  Default: fp16 pieces when every transformed n_a % 4 == 0,
+     TF32 pieces otherwise. */
+  DFT3D_SPLIT_FP16 = 4u,        /* insist on fp16 pieces (operands scaled by powers of two from the largest input
+                                   magnitude; half the tensor-core instructions of TF32); DFT3D_ERR_UNSUPPORTED when
+                                   a transformed n_a is not a multiple of 4 */
+  DFT3D_SPLIT_TF32 = 8u         /* insist on TF32 pieces (no scaling; every element keeps ~22 significant bits
+                                   whatever the dynamic range of the input) */
 };
 
 typedef struct dft3d_options_s {
   size_t struct_size;     /* sizeof(dft3d_options_t), for forward compatibility */
-  unsigned flags;         /* DFT3D_NODES_ON_OUTPUT | DFT3D_UNSCALED_INVERSE */
+  unsigned flags;         /* DFT3D_NODES_ON_OUTPUT | DFT3D_UNSCALED_INVERSE | DFT3D_SPLIT_* */
   int fft_split[3][2];    /* FFT mode: {N1, N2} per axis with N1*N2 = n_a; {0,0} = default split */
   size_t workspace_limit; /* upper bound in bytes for the plan-owned workspace; 0 = default (16 GiB).  KDFT needs a
                              workspace and shrinks it to groups of n0-planes; FFT uses one cube of workspace when it
@@ -127,8 +135,12 @@ int dft3d_plan_status(dft3d_plan_t plan);
 /* Bytes of device workspace the plan owns (0 for NULL). */
 size_t dft3d_plan_workspace_bytes(dft3d_plan_t plan);
 
-/* Number of kernels one dft3d_execute enqueues (0 for NULL). */
+/* Number of kernels one dft3d_execute enqueues (0 for NULL).  With fp16 pieces this counts the small reduction
+ * that finds the largest input magnitude before the first axis pass. */
 int dft3d_plan_launches(dft3d_plan_t plan);
+
+/* DFT3D_SPLIT_FP16 or DFT3D_SPLIT_TF32: the operand split a KDFT plan uses; 0 for an FFT plan or NULL. */
+int dft3d_plan_split(dft3d_plan_t plan);
 
 /* Frees device and host memory of the plan.  NULL is accepted. */
 int dft3d_plan_destroy(dft3d_plan_t plan);

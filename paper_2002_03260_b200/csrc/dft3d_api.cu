@@ -14,6 +14,7 @@
 #include "../../include/dft3d.h"
 #include "generator.h"
 #include "kdft_kernel.cuh"
+#include "kdft_f16_kernel.cuh"
 #include "fft_kernel.cuh"
 
 namespace {
@@ -57,8 +58,18 @@ int get_encoder(EncodeTiledFn* fn) {
 }
 
 // float32 tensor map with up to 4 dimensions; dims/box innermost first; strides in bytes for dims 1..rank-1
+int encode_map(CUtensorMap* map, CUtensorMapDataType dtype, const void* base, int rank,
+               const unsigned long long* dims, const unsigned long long* strides_bytes, const unsigned* box,
+               int swizzle_bytes);
+
 int encode_f32(CUtensorMap* map, const void* base, int rank, const unsigned long long* dims,
                const unsigned long long* strides_bytes, const unsigned* box, int swizzle_bytes) {
+  return encode_map(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, base, rank, dims, strides_bytes, box, swizzle_bytes);
+}
+
+int encode_map(CUtensorMap* map, CUtensorMapDataType dtype, const void* base, int rank,
+               const unsigned long long* dims, const unsigned long long* strides_bytes, const unsigned* box,
+               int swizzle_bytes) {
   EncodeTiledFn enc;
   int rc = get_encoder(&enc);
   if (rc != DFT3D_OK) return rc;
@@ -66,7 +77,7 @@ int encode_f32(CUtensorMap* map, const void* base, int rank, const unsigned long
   cuuint32_t b[4], es[4];
   for (int i = 0; i < rank; ++i) { d[i] = dims[i]; b[i] = box[i]; es[i] = 1; }
   for (int i = 0; i + 1 < rank; ++i) s[i] = strides_bytes[i];
-  CUresult cr = enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, rank, const_cast<void*>(base), d, s, b, es,
+  CUresult cr = enc(map, dtype, rank, const_cast<void*>(base), d, s, b, es,
                     CU_TENSOR_MAP_INTERLEAVE_NONE,
                     swizzle_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
                                          : (swizzle_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_NONE),
@@ -80,9 +91,10 @@ int encode_f32(CUtensorMap* map, const void* base, int rank, const unsigned long
 
 struct KdftAxis {
   long long n = 0;
-  float* d_w = nullptr;   // [2 pieces][2n][2n] floats
+  float* d_w = nullptr;   // [2 pieces][2n][2n] floats (TF32 pieces), or halves holding 1024*W (fp16 pieces)
   CUtensorMap map_w;
   int bn = 0;
+  float out_mul = 1.0f;   // fp16 pieces: 2^-10, times 1/n for a scaled inverse
 };
 
 struct FftAxis {
@@ -101,6 +113,7 @@ struct dft3d_plan_s {
   long long n[3] = {0, 0, 0};
   int mode = 0, sign = 0;
   unsigned flags = 0;
+  bool f16 = false;       // KDFT with fp16 pieces (else TF32 pieces)
   unsigned axes = 7;            // bit a: axis a is transformed
   int device = 0;
   int sm_count = 0;
@@ -111,6 +124,7 @@ struct dft3d_plan_s {
   long long group_planes = 0;   // n0-planes per workspace group (KDFT)
   int chunk_kb = 4;             // 32-real stages per tensor-core accumulation chain (KDFT)
   unsigned int* d_status = nullptr;
+  unsigned int* d_amax = nullptr;   // fp16 pieces: float bits of the largest magnitude before pass 0, 1, 2, (3)
   long long* d_profile = nullptr;   // wait-cycle counters, only allocated in DFT3D_PROFILE_WAITS builds
   void* host_in_dev = nullptr;  // device staging for dft3d_execute_host
   void* host_out_dev = nullptr;
@@ -130,6 +144,10 @@ int set_kernel_attributes(int device) {
                                   cudaFuncAttributeMaxDynamicSharedMemorySize, int(dft3d::kKdftSmemBytes)));
   DFT3D_CUDA(cudaFuncSetAttribute(dft3d::kdft_axis_kernel<dft3d::KDFT_STRIDED>,
                                   cudaFuncAttributeMaxDynamicSharedMemorySize, int(dft3d::kKdftSmemBytes)));
+  DFT3D_CUDA(cudaFuncSetAttribute(dft3d::kdft_f16_axis_kernel<dft3d::KDFT_CONTIG>,
+                                  cudaFuncAttributeMaxDynamicSharedMemorySize, int(dft3d::kKdftF16SmemBytes)));
+  DFT3D_CUDA(cudaFuncSetAttribute(dft3d::kdft_f16_axis_kernel<dft3d::KDFT_STRIDED>,
+                                  cudaFuncAttributeMaxDynamicSharedMemorySize, int(dft3d::kKdftF16SmemBytes)));
 #define DFT3D_FFT_ATTR(MODE, R, RX, COLS, NB2, SO)                                                            \
   DFT3D_CUDA(cudaFuncSetAttribute(dft3d::fft_axis_kernel<MODE, R, RX, COLS, NB2, SO>,                          \
                                   cudaFuncAttributeMaxDynamicSharedMemorySize, int(dft3d::fft_smem_bytes(R, NB2))))
@@ -165,9 +183,40 @@ int build_kdft_axis(dft3d_plan_s* p, int a, const double* nodes) {
   std::vector<float> W;
   try {
     M.resize(size_t(2) * n * n);
-    W.resize(size_t(2) * 4 * n * n);
+    if (!p->f16) W.resize(size_t(2) * 4 * n * n);
   } catch (const std::bad_alloc&) {
     return fail(DFT3D_ERR_ALLOC, "host allocation of the axis-%d table failed", a);
+  }
+  if (p->f16) {
+    // fp16 pieces of 1024*W; the 1/n of a scaled inverse goes into the epilogue multiplier instead of the table
+    dft3d::gen::axis_matrix(n, p->sign, 1.0, nodes, (p->flags & DFT3D_NODES_ON_OUTPUT) != 0, M.data());
+    std::vector<__half> H;
+    try {
+      H.resize(size_t(2) * 4 * n * n);
+    } catch (const std::bad_alloc&) {
+      return fail(DFT3D_ERR_ALLOC, "host allocation of the axis-%d table failed", a);
+    }
+    const size_t piece = size_t(4) * n * n, ld = size_t(2) * n;
+    for (long long k = 0; k < n; ++k)
+      for (long long j = 0; j < n; ++j) {
+        const double re = 1024.0 * M[2 * (k * n + j)], im = 1024.0 * M[2 * (k * n + j) + 1];
+        const double vals[4] = {re, -im, im, re};                  // W[2k][2j], W[2k][2j+1], W[2k+1][2j], W[2k+1][2j+1]
+        const size_t idx[4] = {(2 * k) * ld + 2 * j, (2 * k) * ld + 2 * j + 1, (2 * k + 1) * ld + 2 * j,
+                               (2 * k + 1) * ld + 2 * j + 1};
+        for (int q = 0; q < 4; ++q) {
+          const double hi = dft3d::gen::round_to_fp16(vals[q]);
+          const double lo = dft3d::gen::round_to_fp16(vals[q] - hi);
+          H[idx[q]] = __float2half_rn(float(hi));                  // exact: already on the fp16 grid
+          H[piece + idx[q]] = __float2half_rn(float(lo));
+        }
+      }
+    ax.out_mul = float(scale / 1024.0);
+    DFT3D_CUDA(cudaMalloc(&ax.d_w, H.size() * sizeof(__half)));
+    DFT3D_CUDA(cudaMemcpy(ax.d_w, H.data(), H.size() * sizeof(__half), cudaMemcpyHostToDevice));
+    const unsigned long long hdims[3] = {(unsigned long long)(2 * n), (unsigned long long)(2 * n), 2ull};
+    const unsigned long long hstrides[2] = {(unsigned long long)(2 * n * 2), (unsigned long long)(4 * n * n * 2)};
+    const unsigned hbox[3] = {unsigned(dft3d::kF16BlockK), unsigned(ax.bn), 2u};
+    return encode_map(&ax.map_w, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, ax.d_w, 3, hdims, hstrides, hbox, 128);
   }
   dft3d::gen::axis_matrix(n, p->sign, scale, nodes, (p->flags & DFT3D_NODES_ON_OUTPUT) != 0, M.data());
   dft3d::gen::real_table_from_matrix(n, M.data(), W.data(), W.data() + size_t(4) * n * n);
@@ -180,8 +229,20 @@ int build_kdft_axis(dft3d_plan_s* p, int a, const double* nodes) {
 }
 
 // One KDFT axis pass over a [batches][J][C] complex view (STRIDED) or rows x J (CONTIG).
+template <class Params>
+void fill_f16_params(Params& fp, const dft3d::KdftParams& kp, const KdftAxis& ax, dft3d_plan_s* p, int chain_pos) {
+  fp.k2 = kp.k2; fp.bn = kp.bn; fp.n_tiles = kp.n_tiles; fp.chunk_kb = kp.chunk_kb;
+  fp.m_tiles = kp.m_tiles; fp.rows = kp.rows; fp.batches = kp.batches; fp.C = kp.C;
+  fp.lpb = kp.lpb; fp.bpt = kp.bpt; fp.c_tiles = kp.c_tiles;
+  fp.out = kp.out; fp.status = kp.status; fp.profile = kp.profile;
+  fp.out_mul = ax.out_mul;
+  fp.amax_in = p->d_amax + chain_pos;
+  fp.amax_out = p->d_amax + chain_pos + 1;
+}
+
+// chain_pos: position of this pass in the sequence of passes of one execute (fp16 pieces: which amax word to read)
 int launch_kdft_strided(dft3d_plan_s* p, int a, const float* in, float* out, long long batches, long long C,
-                        cudaStream_t stream) {
+                        cudaStream_t stream, int chain_pos) {
   const KdftAxis& ax = p->kax[a];
   const long long J = ax.n;
   dft3d::KdftParams kp;
@@ -203,18 +264,26 @@ int launch_kdft_strided(dft3d_plan_s* p, int a, const float* in, float* out, lon
   CUtensorMap map_data;
   const unsigned long long dims[3] = {(unsigned long long)(2 * C), (unsigned long long)J, (unsigned long long)batches};
   const unsigned long long strides[2] = {(unsigned long long)(C * 8), (unsigned long long)(J * C * 8)};
-  const unsigned box[3] = {unsigned(2 * kp.lpb), unsigned(dft3d::kBlockK / 2), unsigned(kp.bpt)};
+  const bool f16 = p->f16;
+  const unsigned box[3] = {unsigned(2 * kp.lpb), unsigned((f16 ? dft3d::kF16BlockK : dft3d::kBlockK) / 2), unsigned(kp.bpt)};
   int rc = encode_f32(&map_data, in, 3, dims, strides, box, 0);
   if (rc != DFT3D_OK) return rc;
   const long long total = kp.m_tiles * kp.n_tiles;
   const int grid = int(total < p->sm_count ? total : p->sm_count);
+  if (f16) {
+    dft3d::KdftF16Params fp;
+    fill_f16_params(fp, kp, ax, p, chain_pos);
+    dft3d::kdft_f16_axis_kernel<dft3d::KDFT_STRIDED>
+        <<<grid, dft3d::kKdftThreads, dft3d::kKdftF16SmemBytes, stream>>>(map_data, ax.map_w, fp);
+  } else
   dft3d::kdft_axis_kernel<dft3d::KDFT_STRIDED>
       <<<grid, dft3d::kKdftThreads, dft3d::kKdftSmemBytes, stream>>>(map_data, ax.map_w, kp);
   DFT3D_CUDA(cudaGetLastError());
   return DFT3D_OK;
 }
 
-int launch_kdft_contig(dft3d_plan_s* p, int a, const float* in, float* out, long long rows, cudaStream_t stream) {
+int launch_kdft_contig(dft3d_plan_s* p, int a, const float* in, float* out, long long rows, cudaStream_t stream,
+                       int chain_pos) {
   const KdftAxis& ax = p->kax[a];
   const long long J = ax.n;
   dft3d::KdftParams kp;
@@ -239,18 +308,35 @@ int launch_kdft_contig(dft3d_plan_s* p, int a, const float* in, float* out, long
   if (rc != DFT3D_OK) return rc;
   const long long total = kp.m_tiles * kp.n_tiles;
   const int grid = int(total < p->sm_count ? total : p->sm_count);
+  if (p->f16) {
+    dft3d::KdftF16Params fp;
+    fill_f16_params(fp, kp, ax, p, chain_pos);
+    dft3d::kdft_f16_axis_kernel<dft3d::KDFT_CONTIG>
+        <<<grid, dft3d::kKdftThreads, dft3d::kKdftF16SmemBytes, stream>>>(map_data, ax.map_w, fp);
+  } else
   dft3d::kdft_axis_kernel<dft3d::KDFT_CONTIG>
       <<<grid, dft3d::kKdftThreads, dft3d::kKdftSmemBytes, stream>>>(map_data, ax.map_w, kp);
   DFT3D_CUDA(cudaGetLastError());
   return DFT3D_OK;
 }
 
-int kdft_axis_pass(dft3d_plan_s* p, int axis, const float* in, float* out, long long planes, cudaStream_t stream) {
+int kdft_axis_pass(dft3d_plan_s* p, int axis, const float* in, float* out, long long planes, cudaStream_t stream,
+                   int chain_pos) {
   // `planes` n0-planes starting at in/out (axis 0 always takes the whole cube)
   const long long n1 = p->n[1], n2 = p->n[2];
-  if (axis == 0) return launch_kdft_strided(p, 0, in, out, 1, n1 * n2, stream);
-  if (axis == 1) return launch_kdft_strided(p, 1, in, out, planes, n2, stream);
-  return launch_kdft_contig(p, 2, in, out, planes * n1, stream);
+  if (axis == 0) return launch_kdft_strided(p, 0, in, out, 1, n1 * n2, stream, chain_pos);
+  if (axis == 1) return launch_kdft_strided(p, 1, in, out, planes, n2, stream, chain_pos);
+  return launch_kdft_contig(p, 2, in, out, planes * n1, stream, chain_pos);
+}
+
+// fp16 pieces: before the first pass of an execute, clear the chain of amax words and measure the input
+int kdft_prepare_scales(dft3d_plan_s* p, const float* in, cudaStream_t stream) {
+  if (!p->f16) return DFT3D_OK;
+  DFT3D_CUDA(cudaMemsetAsync(p->d_amax, 0, 4 * sizeof(unsigned int), stream));
+  const long long n4 = points(p) / 2;      // float4 = two complex points; the point count is even
+  dft3d::amax_kernel<<<p->sm_count * 8, 256, 0, stream>>>(reinterpret_cast<const float4*>(in), n4, p->d_amax);
+  DFT3D_CUDA(cudaGetLastError());
+  return DFT3D_OK;
 }
 
 // FFT formulation, one axis: n = RX*R*R with R = 16 or 32 and RX = 1 or 2 (Eq. 17 with P = R, preceded for
@@ -539,7 +625,13 @@ int dft3d_plan_create_ex(dft3d_plan_t* out, long long n0, long long n1, long lon
       return fail(DFT3D_ERR_INVALID_ARG, "options->struct_size is not a known size");
     memcpy(&opt, options, options->struct_size);
   }
-  if (opt.flags & ~(DFT3D_NODES_ON_OUTPUT | DFT3D_UNSCALED_INVERSE)) return fail(DFT3D_ERR_INVALID_ARG, "unknown flag");
+  if (opt.flags & ~(DFT3D_NODES_ON_OUTPUT | DFT3D_UNSCALED_INVERSE | DFT3D_SPLIT_FP16 | DFT3D_SPLIT_TF32))
+    return fail(DFT3D_ERR_INVALID_ARG, "unknown flag");
+  if ((opt.flags & DFT3D_SPLIT_FP16) && (opt.flags & DFT3D_SPLIT_TF32))
+    return fail(DFT3D_ERR_INVALID_ARG, "DFT3D_SPLIT_FP16 and DFT3D_SPLIT_TF32 exclude each other");
+  if ((opt.flags & DFT3D_SPLIT_FP16) && mode != DFT3D_KDFT)
+    return fail(DFT3D_ERR_UNSUPPORTED, "DFT3D_SPLIT_FP16 applies to the KDFT formulation");
+  bool f16 = mode == DFT3D_KDFT && !(opt.flags & DFT3D_SPLIT_TF32);   // default where the sizes allow it
   if (opt.axes > 7) return fail(DFT3D_ERR_INVALID_ARG, "axes must be a mask of bits 0..2");
   const unsigned axes = opt.axes ? opt.axes : 7u;
   for (int a = 0; a < 3; ++a) {
@@ -551,6 +643,11 @@ int dft3d_plan_create_ex(dft3d_plan_t* out, long long n0, long long n1, long lon
     if (nn[a] % quantum != 0)
       return fail(DFT3D_ERR_UNSUPPORTED, "n%d = %lld is not a multiple of %lld", a, nn[a], quantum);
     if (transformed && nn[a] > 8192) return fail(DFT3D_ERR_UNSUPPORTED, "n%d = %lld exceeds 8192", a, nn[a]);
+    if (transformed && nn[a] % 4 != 0) {
+      if (opt.flags & DFT3D_SPLIT_FP16)
+        return fail(DFT3D_ERR_UNSUPPORTED, "DFT3D_SPLIT_FP16 needs n%d = %lld to be a multiple of 4", a, nn[a]);
+      f16 = false;
+    }
   }
   if (mode == DFT3D_FFT && (nodes0 || nodes1 || nodes2))
     return fail(DFT3D_ERR_UNSUPPORTED, "the FFT formulation needs a uniform grid (no nodes)");
@@ -565,6 +662,7 @@ int dft3d_plan_create_ex(dft3d_plan_t* out, long long n0, long long n1, long lon
     p->mode = mode;
     p->sign = sign;
     p->flags = opt.flags;
+    p->f16 = f16;
     p->axes = axes;
     cudaDeviceProp prop;
     if (cudaGetDevice(&p->device) != cudaSuccess || cudaGetDeviceProperties(&prop, p->device) != cudaSuccess) {
@@ -590,6 +688,8 @@ int dft3d_plan_create_ex(dft3d_plan_t* out, long long n0, long long n1, long lon
     if (e == cudaSuccess) e = cudaMemset(p->d_profile, 0, sizeof(long long) * 128 * 256);
     if (e != cudaSuccess) { rc = fail(DFT3D_ERR_ALLOC, "cudaMalloc(profile)"); break; }
 #endif
+    e = cudaMalloc(&p->d_amax, 4 * sizeof(unsigned int));
+    if (e != cudaSuccess) { rc = fail(DFT3D_ERR_ALLOC, "cudaMalloc(amax): %s", cudaGetErrorString(e)); break; }
     if (mode == DFT3D_KDFT) {
       for (int a = 0; a < 3 && rc == DFT3D_OK; ++a)
         if ((axes >> a) & 1u) rc = build_kdft_axis(p, a, nodes[a]);
@@ -652,8 +752,10 @@ int dft3d_execute_axis(dft3d_plan_t p, int axis, const void* in, void* out, void
   if (axis < 0 || axis > 2) return fail(DFT3D_ERR_INVALID_ARG, "axis must be 0, 1 or 2");
   if (!((p->axes >> axis) & 1u)) return fail(DFT3D_ERR_INVALID_ARG, "axis %d is not among the plan's axes", axis);
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-  if (p->mode == DFT3D_KDFT)
-    return kdft_axis_pass(p, axis, static_cast<const float*>(in), static_cast<float*>(out), p->n[0], stream);
+  if (p->mode == DFT3D_KDFT) {
+    if ((rc = kdft_prepare_scales(p, static_cast<const float*>(in), stream)) != DFT3D_OK) return rc;
+    return kdft_axis_pass(p, axis, static_cast<const float*>(in), static_cast<float*>(out), p->n[0], stream, 0);
+  }
   return fft_axis_pass(p, axis, static_cast<const float*>(in), static_cast<float*>(out), stream);
 }
 
@@ -668,27 +770,31 @@ int dft3d_execute(dft3d_plan_t p, const void* in, void* out, void* cuda_stream) 
     const long long g = p->group_planes;
     const long long plane_floats = p->n[1] * p->n[2] * 2;
     float* ws = static_cast<float*>(p->workspace);
+    if ((rc = kdft_prepare_scales(p, fin, stream)) != DFT3D_OK) return rc;
+    // the last argument is the pass's position in the chain (fp16 pieces: every pass reads the largest magnitude its
+    // predecessor recorded; a later group of planes may read a value that earlier groups already raised, which is
+    // still an upper bound for its own data)
     if (axes == 7u) {
       // axis 0: in -> out; then per group of n0-planes: axis 1 out -> workspace, axis 2 workspace -> out
-      if ((rc = kdft_axis_pass(p, 0, fin, fout, p->n[0], stream)) != DFT3D_OK) return rc;
+      if ((rc = kdft_axis_pass(p, 0, fin, fout, p->n[0], stream, 0)) != DFT3D_OK) return rc;
       for (long long a = 0; a < p->n[0]; a += g) {
         float* slab = fout + a * plane_floats;
-        if ((rc = kdft_axis_pass(p, 1, slab, ws, g, stream)) != DFT3D_OK) return rc;
-        if ((rc = kdft_axis_pass(p, 2, ws, slab, g, stream)) != DFT3D_OK) return rc;
+        if ((rc = kdft_axis_pass(p, 1, slab, ws, g, stream, 1)) != DFT3D_OK) return rc;
+        if ((rc = kdft_axis_pass(p, 2, ws, slab, g, stream, 2)) != DFT3D_OK) return rc;
       }
     } else if (axes == 6u) {
       // batch of 2D transforms: per group axis 1 in -> workspace, axis 2 workspace -> out
       for (long long a = 0; a < p->n[0]; a += g) {
-        if ((rc = kdft_axis_pass(p, 1, fin + a * plane_floats, ws, g, stream)) != DFT3D_OK) return rc;
-        if ((rc = kdft_axis_pass(p, 2, ws, fout + a * plane_floats, g, stream)) != DFT3D_OK) return rc;
+        if ((rc = kdft_axis_pass(p, 1, fin + a * plane_floats, ws, g, stream, 0)) != DFT3D_OK) return rc;
+        if ((rc = kdft_axis_pass(p, 2, ws, fout + a * plane_floats, g, stream, 1)) != DFT3D_OK) return rc;
       }
     } else if (axes == 3u || axes == 5u) {
       // axis 0 and one more: the other axis in -> workspace (whole cube), then axis 0 workspace -> out
-      if ((rc = kdft_axis_pass(p, axes == 3u ? 1 : 2, fin, ws, p->n[0], stream)) != DFT3D_OK) return rc;
-      if ((rc = kdft_axis_pass(p, 0, ws, fout, p->n[0], stream)) != DFT3D_OK) return rc;
+      if ((rc = kdft_axis_pass(p, axes == 3u ? 1 : 2, fin, ws, p->n[0], stream, 0)) != DFT3D_OK) return rc;
+      if ((rc = kdft_axis_pass(p, 0, ws, fout, p->n[0], stream, 1)) != DFT3D_OK) return rc;
     } else {
       const int a = axes == 1u ? 0 : (axes == 2u ? 1 : 2);
-      if ((rc = kdft_axis_pass(p, a, fin, fout, p->n[0], stream)) != DFT3D_OK) return rc;
+      if ((rc = kdft_axis_pass(p, a, fin, fout, p->n[0], stream, 0)) != DFT3D_OK) return rc;
     }
     return DFT3D_OK;
   }
@@ -739,9 +845,15 @@ size_t dft3d_plan_workspace_bytes(dft3d_plan_t p) { return p ? p->workspace_byte
 int dft3d_plan_launches(dft3d_plan_t p) {
   if (!p) return 0;
   const int count = int((p->axes & 1u) + ((p->axes >> 1) & 1u) + ((p->axes >> 2) & 1u));
-  if (p->mode == DFT3D_KDFT && p->axes == 7u) return int(1 + 2 * (p->n[0] / p->group_planes));
-  if (p->mode == DFT3D_KDFT && p->axes == 6u) return int(2 * (p->n[0] / p->group_planes));
-  return count;
+  const int pre = p->f16 ? 1 : 0;   // the reduction that finds the largest input magnitude
+  if (p->mode == DFT3D_KDFT && p->axes == 7u) return pre + int(1 + 2 * (p->n[0] / p->group_planes));
+  if (p->mode == DFT3D_KDFT && p->axes == 6u) return pre + int(2 * (p->n[0] / p->group_planes));
+  return pre + count;
+}
+
+int dft3d_plan_split(dft3d_plan_t p) {
+  if (!p || p->mode != DFT3D_KDFT) return 0;
+  return p->f16 ? DFT3D_SPLIT_FP16 : DFT3D_SPLIT_TF32;
 }
 
 int dft3d_plan_destroy(dft3d_plan_t p) {
@@ -754,6 +866,7 @@ int dft3d_plan_destroy(dft3d_plan_t p) {
   }
   if (p->workspace) cudaFree(p->workspace);
   if (p->d_status) cudaFree(p->d_status);
+  if (p->d_amax) cudaFree(p->d_amax);
   if (p->d_profile) cudaFree(p->d_profile);
   if (p->host_in_dev) cudaFree(p->host_in_dev);
   if (p->host_out_dev) cudaFree(p->host_out_dev);

@@ -102,6 +102,17 @@ float round_to_tf32(double v) {
   return static_cast<float>(std::ldexp(r, e - 11));
 }
 
+double round_to_fp16(double v) {
+  if (v == 0.0 || !std::isfinite(v)) return v;
+  const double a = std::fabs(v);
+  if (a < 6.103515625e-05) {                       // below 2^-14: subnormal grid, spacing 2^-24
+    return std::nearbyint(v * 16777216.0) / 16777216.0;
+  }
+  int e;
+  const double m = std::frexp(v, &e);
+  return std::ldexp(std::nearbyint(std::ldexp(m, 11)), e - 11);
+}
+
 void real_table_from_matrix(int64_t n, const double* M, float* hi, float* lo) {
   const int64_t ld = 2 * n;
   for (int64_t k = 0; k < n; ++k)

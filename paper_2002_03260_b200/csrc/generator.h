@@ -22,6 +22,9 @@ void twiddle(int64_t N1, int64_t N2, int sign, double* T);
 // nearest value with an 11-bit significand (TF32), returned as float (low 13 mantissa bits zero)
 float round_to_tf32(double v);
 
+// nearest fp16 value (11-bit significand down to 2^-14, multiples of 2^-24 below; no overflow handling: |v| < 65504)
+double round_to_fp16(double v);
+
 // v ~= hi + lo with both pieces TF32-exact
 inline void split_tf32(double v, float* hi, float* lo) {
   *hi = round_to_tf32(v);

@@ -15,11 +15,11 @@ _LIB_PATH = os.environ.get("DFT3D_LIBRARY") or os.path.join(_HERE, "libdft3d.so"
 
 DFT3D_KDFT, DFT3D_FFT = 0, 1
 DFT3D_FORWARD, DFT3D_INVERSE = -1, +1
-DFT3D_NODES_ON_OUTPUT, DFT3D_UNSCALED_INVERSE = 1, 2
+DFT3D_NODES_ON_OUTPUT, DFT3D_UNSCALED_INVERSE, DFT3D_SPLIT_FP16, DFT3D_SPLIT_TF32 = 1, 2, 4, 8
 
 EXPORTS = [
     "dft3d_plan_create", "dft3d_plan_create_ex", "dft3d_execute", "dft3d_execute_host", "dft3d_execute_axis",
-    "dft3d_plan_status", "dft3d_plan_workspace_bytes", "dft3d_plan_launches", "dft3d_plan_destroy",
+    "dft3d_plan_status", "dft3d_plan_workspace_bytes", "dft3d_plan_launches", "dft3d_plan_split", "dft3d_plan_destroy",
     "dft3d_status_string", "dft3d_last_error", "dft3d_generate_axis_matrix", "dft3d_generate_twiddle",
     "dft3d_generate_real_table", "dft3d_kdft_execute_static",
 ]
@@ -57,6 +57,7 @@ def _load():
     lib.dft3d_plan_workspace_bytes.argtypes = [vp]
     lib.dft3d_plan_workspace_bytes.restype = ctypes.c_size_t
     lib.dft3d_plan_launches.argtypes = [vp]
+    lib.dft3d_plan_split.argtypes = [vp]
     lib.dft3d_plan_destroy.argtypes = [vp]
     lib.dft3d_status_string.argtypes = [ci]
     lib.dft3d_status_string.restype = ctypes.c_char_p
@@ -204,6 +205,11 @@ class Plan:
     @property
     def launches(self):
         return int(_lib.dft3d_plan_launches(self._h))
+
+    @property
+    def split(self):
+        """DFT3D_SPLIT_FP16 or DFT3D_SPLIT_TF32 for a KDFT plan, 0 for an FFT plan."""
+        return int(_lib.dft3d_plan_split(self._h))
 
     def destroy(self):
         if self._h:

@@ -36,13 +36,27 @@ def _finish(plan):
     plan.status()
 
 
+SPLITS = ["fp16", "tf32"]   # the two operand splits of the KDFT kernels; fp16 is the default where sizes allow
+
+
+def _split_flag(lib, split):
+    return lib.DFT3D_SPLIT_FP16 if split == "fp16" else lib.DFT3D_SPLIT_TF32
+
+
+def _pre(lib, plan):
+    """Launches before the axis passes: the fp16 split first reduces the input to its largest magnitude."""
+    return 1 if plan.split == lib.DFT3D_SPLIT_FP16 else 0
+
+
 # ------------------------------------------------------------------ single axes (each kernel variant alone)
 
 @pytest.mark.parametrize("shape", [(64, 64, 64), (64, 128, 192), (128, 64, 256), (192, 64, 64)])
 @pytest.mark.parametrize("axis", [0, 1, 2])
-def test_kdft_single_axis(lib, oracle, shape, axis):
+@pytest.mark.parametrize("split", SPLITS)
+def test_kdft_single_axis(lib, oracle, shape, axis, split):
     x = _inputs().cube(shape, "normal", 7 + axis, device="cuda")
-    plan = lib.Plan(*shape, mode=lib.DFT3D_KDFT)
+    plan = lib.Plan(*shape, mode=lib.DFT3D_KDFT, flags=_split_flag(lib, split))
+    assert plan.split == _split_flag(lib, split)
     y = plan.execute_axis(axis, x)
     _finish(plan)
     ref = oracle.dft_axis(x.cpu().numpy().astype(np.complex128), axis)
@@ -53,10 +67,11 @@ def test_kdft_single_axis(lib, oracle, shape, axis):
 
 # ------------------------------------------------------------------ config 1: 64^3 KDFT forward, U(-1,1)
 
-def test_config1_kdft_64(lib, oracle):
+@pytest.mark.parametrize("split", SPLITS)
+def test_config1_kdft_64(lib, oracle, split):
     shape = (64, 64, 64)
     x = _inputs().cube(shape, "uniform", 1001, device="cuda")
-    plan = lib.Plan(*shape, mode=lib.DFT3D_KDFT, sign=lib.DFT3D_FORWARD)
+    plan = lib.Plan(*shape, mode=lib.DFT3D_KDFT, sign=lib.DFT3D_FORWARD, flags=_split_flag(lib, split))
     y = plan(x)
     _finish(plan)
     ref = oracle.dft3d(x.cpu().numpy())
@@ -68,9 +83,10 @@ def test_config1_kdft_64(lib, oracle):
 
 
 @pytest.mark.parametrize("shape", [(64, 128, 256), (256, 64, 128), (128, 192, 64)])
-def test_kdft_noncubic(lib, oracle, shape):
+@pytest.mark.parametrize("split", SPLITS)
+def test_kdft_noncubic(lib, oracle, shape, split):
     x = _inputs().cube(shape, "uniform", 31, device="cuda")
-    plan = lib.Plan(*shape)
+    plan = lib.Plan(*shape, flags=_split_flag(lib, split))
     y = plan(x)
     _finish(plan)
     err = oracle.rel_l2(y.cpu().numpy(), oracle.dft3d(x.cpu().numpy()))
@@ -78,12 +94,13 @@ def test_kdft_noncubic(lib, oracle, shape):
     plan.destroy()
 
 
-def test_kdft_workspace_groups(lib, oracle):
+@pytest.mark.parametrize("split", SPLITS)
+def test_kdft_workspace_groups(lib, oracle, split):
     """A small workspace limit forces the plane-group schedule (several launches per axis)."""
     shape = (64, 64, 128)
     x = _inputs().cube(shape, "normal", 32, device="cuda")
-    plan = lib.Plan(*shape, workspace_limit=16 * 64 * 128 * 8)
-    assert plan.workspace_bytes == 16 * 64 * 128 * 8 and plan.launches == 1 + 2 * 4
+    plan = lib.Plan(*shape, workspace_limit=16 * 64 * 128 * 8, flags=_split_flag(lib, split))
+    assert plan.workspace_bytes == 16 * 64 * 128 * 8 and plan.launches == _pre(lib, plan) + 1 + 2 * 4
     y = plan(x)
     _finish(plan)
     err = oracle.rel_l2(y.cpu().numpy(), oracle.dft3d(x.cpu().numpy()))
@@ -91,10 +108,12 @@ def test_kdft_workspace_groups(lib, oracle):
     plan.destroy()
 
 
-def test_kdft_inverse_and_roundtrip(lib, oracle):
+@pytest.mark.parametrize("split", SPLITS)
+def test_kdft_inverse_and_roundtrip(lib, oracle, split):
     shape = (128, 64, 64)
     x = _inputs().cube(shape, "normal", 33, device="cuda")
-    fwd, inv = lib.Plan(*shape, sign=lib.DFT3D_FORWARD), lib.Plan(*shape, sign=lib.DFT3D_INVERSE)
+    sf = _split_flag(lib, split)
+    fwd, inv = lib.Plan(*shape, sign=lib.DFT3D_FORWARD, flags=sf), lib.Plan(*shape, sign=lib.DFT3D_INVERSE, flags=sf)
     X = fwd(x)
     back = inv(X)
     _finish(inv)
@@ -102,7 +121,7 @@ def test_kdft_inverse_and_roundtrip(lib, oracle):
     assert oracle.rel_l2(back.cpu().numpy(), x.cpu().numpy()) < TOL   # two transforms in a row
     ref = oracle.dft3d(X.cpu().numpy(), sign=+1, scaled_inverse=True)
     assert oracle.rel_l2(back.cpu().numpy(), ref) < SANITY
-    raw = lib.Plan(*shape, sign=lib.DFT3D_INVERSE, flags=lib.DFT3D_UNSCALED_INVERSE)
+    raw = lib.Plan(*shape, sign=lib.DFT3D_INVERSE, flags=lib.DFT3D_UNSCALED_INVERSE | sf)
     y = raw(X)
     _finish(raw)
     assert oracle.rel_l2(y.cpu().numpy(), oracle.dft3d(X.cpu().numpy(), sign=+1)) < SANITY
@@ -112,12 +131,13 @@ def test_kdft_inverse_and_roundtrip(lib, oracle):
 
 # ------------------------------------------------------------------ config 4: nonuniform KDFT 256^3
 
-def test_config4_nonuniform_256(lib, oracle):
+@pytest.mark.parametrize("split", SPLITS)
+def test_config4_nonuniform_256(lib, oracle, split):
     shape = (256, 256, 256)
     inp = _inputs()
     x = inp.cube(shape, "normal", 1004, device="cuda")
     nodes = inp.sorted_nodes(shape, 2004)
-    plan = lib.Plan(*shape, nodes=nodes)
+    plan = lib.Plan(*shape, nodes=nodes, flags=_split_flag(lib, split))
     y = plan(x)
     _finish(plan)
     ref = oracle.dft3d(x.cpu().numpy(), nodes=nodes)
@@ -441,20 +461,21 @@ def test_batched_2d(lib, oracle, mode_name, shape):
     plan = lib.Plan(*shape, mode=mode, axes=(1, 2))
     y = plan(x)
     _finish(plan)
-    assert plan.launches == 2
+    assert plan.launches == _pre(lib, plan) + 2
     plan.destroy()
     err = oracle.rel_l2(y.cpu().numpy(), _oracle_axes(oracle, x.cpu().numpy(), (1, 2)))
     assert err < SANITY, (mode_name, shape, err)
 
 
 @pytest.mark.parametrize("axes", [(2,), (1,), (0,), (0, 1), (0, 2)])
-def test_axis_subsets_kdft(lib, oracle, axes):
+@pytest.mark.parametrize("split", SPLITS)
+def test_axis_subsets_kdft(lib, oracle, axes, split):
     shape = (64, 128, 64)
     x = _inputs().cube(shape, "uniform", 82, device="cuda")
-    plan = lib.Plan(*shape, axes=axes, sign=lib.DFT3D_INVERSE)
+    plan = lib.Plan(*shape, axes=axes, sign=lib.DFT3D_INVERSE, flags=_split_flag(lib, split))
     y = plan(x)
     _finish(plan)
-    assert plan.launches == len(axes)
+    assert plan.launches == _pre(lib, plan) + len(axes)
     with pytest.raises(lib.Dft3dError):
         plan.execute_axis([a for a in range(3) if a not in axes][0], x)
     plan.destroy()
@@ -476,14 +497,21 @@ def test_batched_1d_fft(lib, oracle):
 
 # ------------------------------------------------------------------ sizes that are not tile multiples (KDFT)
 
-@pytest.mark.parametrize("shape", [(100, 66, 250), (30, 18, 34), (2, 4, 6), (130, 64, 2), (66, 258, 64)])
+@pytest.mark.parametrize("shape", [(100, 66, 250), (30, 18, 34), (2, 4, 6), (130, 64, 2), (66, 258, 64),
+                                   (100, 68, 36), (4, 132, 252), (260, 8, 12)])
 def test_kdft_general_even_sizes(lib, oracle, shape):
-    """Any even length: ragged K stages are zero-filled by TMA on both operands, ragged tiles masked on store."""
+    """Any even length: ragged K stages are zero-filled by TMA on both operands, ragged tiles masked on store.
+    Shapes whose lengths are all multiples of 4 run the fp16 split, the others fall back to the TF32 split."""
     x = _inputs().cube(shape, "normal", 91, device="cuda")
     guard = torch.full((1 << 14,), 7.0, device="cuda")           # canaries around the output
     out = torch.empty_like(x)
     guard2 = torch.full((1 << 14,), 7.0, device="cuda")
     plan = lib.Plan(*shape)
+    fp16_ok = all(n % 4 == 0 for n in shape)
+    assert plan.split == (lib.DFT3D_SPLIT_FP16 if fp16_ok else lib.DFT3D_SPLIT_TF32)
+    if not fp16_ok:
+        with pytest.raises(lib.Dft3dError):
+            lib.Plan(*shape, flags=lib.DFT3D_SPLIT_FP16)
     plan(x, out)
     _finish(plan)
     plan.destroy()
@@ -496,3 +524,60 @@ def test_kdft_general_even_sizes(lib, oracle, shape):
     _finish(plan)
     plan.destroy()
     assert oracle.rel_l2(y.cpu().numpy(), oracle.dft3d(x.cpu().numpy(), nodes=nodes)) < SANITY
+
+
+# ------------------------------------------------------------------ fp16 split: scaling by powers of two
+
+@pytest.mark.parametrize("log2_scale", [-120, -60, 0, 90])
+def test_fp16_split_is_scale_invariant(lib, oracle, log2_scale):
+    """The fp16 pieces are taken after an exact power-of-two scaling chosen from the largest input magnitude, so
+    a scaled input gives the scaled result bit for bit (2^-120 puts the data next to the smallest normal float,
+    where the scale factor saturates and a few entries are subnormal: fp32-level accuracy is all that is asked)."""
+    shape = (64, 128, 64)
+    x = _inputs().cube(shape, "normal", 93, device="cuda")
+    plan = lib.Plan(*shape, flags=lib.DFT3D_SPLIT_FP16)
+    y = plan(x).clone()
+    xs = x * (2.0 ** log2_scale)
+    ys = plan(xs)
+    _finish(plan)
+    plan.destroy()
+    if log2_scale > -100:
+        assert torch.equal(ys, y * (2.0 ** log2_scale))
+    ref = oracle.dft3d(xs.cpu().numpy().astype(np.complex128))
+    assert oracle.rel_l2(ys.cpu().numpy().astype(np.complex128), ref) < SANITY
+
+
+def test_fp16_split_wide_dynamic_range(lib, oracle):
+    """One entry 2^30 above the rest: the error stays at fp32 level relative to the norm of the result (small
+    entries lose relative, not norm-wise, accuracy), and the TF32 split agrees."""
+    shape = (64, 64, 128)
+    x = _inputs().cube(shape, "normal", 94, device="cuda")
+    x[3, 5, 7] = 2.0 ** 30
+    ref = oracle.dft3d(x.cpu().numpy())
+    for flag in (lib.DFT3D_SPLIT_FP16, lib.DFT3D_SPLIT_TF32):
+        plan = lib.Plan(*shape, flags=flag)
+        y = plan(x)
+        _finish(plan)
+        plan.destroy()
+        assert oracle.rel_l2(y.cpu().numpy(), ref) < SANITY, flag
+    # all-zero input: no scale is derived, the result is exactly zero
+    plan = lib.Plan(*shape, flags=lib.DFT3D_SPLIT_FP16)
+    z = plan(torch.zeros_like(x))
+    _finish(plan)
+    plan.destroy()
+    assert not bool(z.any())
+
+
+@pytest.mark.slow
+def test_splits_agree_512(lib, oracle):
+    """Config-2 size: the two splits agree with each other to fp32 level and the fp16 one is not slower."""
+    shape = (512, 512, 512)
+    x = _inputs().cube(shape, "uniform", 95, device="cuda")
+    res = {}
+    for name in SPLITS:
+        plan = lib.Plan(*shape, flags=_split_flag(lib, name))
+        res[name] = plan(x)
+        _finish(plan)
+        plan.destroy()
+    diff = torch.linalg.vector_norm((res["fp16"] - res["tf32"]).flatten()) / torch.linalg.vector_norm(res["tf32"].flatten())
+    assert diff.item() < SANITY
