@@ -15,6 +15,7 @@
 #include "generator.h"
 #include "kdft_kernel.cuh"
 #include "kdft_f16_kernel.cuh"
+#include "fft_f16_kernel.cuh"
 #include "fft_kernel.cuh"
 
 namespace {
@@ -104,6 +105,7 @@ struct FftAxis {
   float* d_w = nullptr;    // real form of F_R: [piece hi|lo][2R/32 panels][2R rows][32 floats]
   float2* d_tw = nullptr;  // T[k1][beta], R*R complex64
   float2* d_tw2 = nullptr; // RX == 2: exp(s*2*pi*i*m/n), m < R*R
+  float out_mul = 1.0f;    // fp16 pieces: the factor the store applies (powers of two, 1/n for a scaled inverse)
   CUtensorMap map_w;
 };
 
@@ -168,6 +170,24 @@ int set_kernel_attributes(int device) {
   DFT3D_FFT_ATTR(dft3d::FFT_STRIDED, 32, 2, 8, 1, 1);
   DFT3D_FFT_ATTR(dft3d::FFT_STRIDED, 16, 2, 16, 2, 1);
 #undef DFT3D_FFT_ATTR
+#define DFT3D_FFT16_ATTR(MODE, R, RX, COLS, SO)                                                   \
+  DFT3D_CUDA(cudaFuncSetAttribute(dft3d::fft_f16_axis_kernel<MODE, R, RX, COLS, SO>,              \
+                                  cudaFuncAttributeMaxDynamicSharedMemorySize, int(dft3d::fft16_smem_bytes(R))))
+  DFT3D_FFT16_ATTR(dft3d::FFT_CONTIG, 32, 1, 16, 0);
+  DFT3D_FFT16_ATTR(dft3d::FFT_CONTIG, 16, 1, 16, 0);
+  DFT3D_FFT16_ATTR(dft3d::FFT_CONTIG, 32, 2, 16, 0);
+  DFT3D_FFT16_ATTR(dft3d::FFT_CONTIG, 16, 2, 16, 0);
+  DFT3D_FFT16_ATTR(dft3d::FFT_STRIDED, 32, 1, 16, 0);
+  DFT3D_FFT16_ATTR(dft3d::FFT_STRIDED, 32, 1, 8, 0);
+  DFT3D_FFT16_ATTR(dft3d::FFT_STRIDED, 16, 1, 16, 0);
+  DFT3D_FFT16_ATTR(dft3d::FFT_STRIDED, 32, 2, 8, 0);
+  DFT3D_FFT16_ATTR(dft3d::FFT_STRIDED, 16, 2, 16, 0);
+  DFT3D_FFT16_ATTR(dft3d::FFT_STRIDED, 32, 1, 16, 1);
+  DFT3D_FFT16_ATTR(dft3d::FFT_STRIDED, 32, 1, 8, 1);
+  DFT3D_FFT16_ATTR(dft3d::FFT_STRIDED, 16, 1, 16, 1);
+  DFT3D_FFT16_ATTR(dft3d::FFT_STRIDED, 32, 2, 8, 1);
+  DFT3D_FFT16_ATTR(dft3d::FFT_STRIDED, 16, 2, 16, 1);
+#undef DFT3D_FFT16_ATTR
   done = true;
   return DFT3D_OK;
 }
@@ -330,7 +350,7 @@ int kdft_axis_pass(dft3d_plan_s* p, int axis, const float* in, float* out, long 
 }
 
 // fp16 pieces: before the first pass of an execute, clear the chain of amax words and measure the input
-int kdft_prepare_scales(dft3d_plan_s* p, const float* in, cudaStream_t stream) {
+int prepare_scales(dft3d_plan_s* p, const float* in, cudaStream_t stream) {
   if (!p->f16) return DFT3D_OK;
   DFT3D_CUDA(cudaMemsetAsync(p->d_amax, 0, 4 * sizeof(unsigned int), stream));
   const long long n4 = points(p) / 2;      // float4 = two complex points; the point count is even
@@ -362,6 +382,51 @@ int build_fft_axis(dft3d_plan_s* p, int a, const int split[2]) {
   ax.cols = (R == 32 && RX == 2) ? 8 : 16;   // default; fft_axis_pass may pick 8 for R = 32, RX = 1 (see there)
   const bool scaled = (p->sign > 0) && !(p->flags & DFT3D_UNSCALED_INVERSE);
   const int K = 2 * R, NB = 2 * R, panels = K / 32;
+  if (p->f16) {
+    // fp16 pieces: 1024 * F_R (real form), rows of 64 halves (zero-padded for R = 16), [hi piece; lo piece]; the twiddle
+    // factors carry 2^-(10 + log2(R) - 1); everything else (1/n of a scaled inverse included) is one factor at the store
+    const int sh = (R == 32 ? 5 : 4) - 1;
+    std::vector<double> M(size_t(2) * R * R), T(size_t(2) * R * R);
+    std::vector<__half> W(size_t(2) * NB * 64, __float2half(0.0f));
+    std::vector<float> tw(size_t(2) * R * R);
+    dft3d::gen::axis_matrix(R, p->sign, 1024.0, nullptr, false, M.data());
+    for (int k = 0; k < R; ++k)
+      for (int j = 0; j < R; ++j) {
+        const double re = M[2 * (size_t(k) * R + j)], im = M[2 * (size_t(k) * R + j) + 1];
+        const double v[2][2] = {{re, -im}, {im, re}};
+        for (int pp = 0; pp < 2; ++pp)
+          for (int q = 0; q < 2; ++q) {
+            const double hi = dft3d::gen::round_to_fp16(v[pp][q]);
+            const double lo = dft3d::gen::round_to_fp16(v[pp][q] - hi);
+            const size_t at = size_t(2 * k + pp) * 64 + (2 * j + q);
+            W[at] = __float2half(float(hi));
+            W[size_t(NB) * 64 + at] = __float2half(float(lo));
+          }
+      }
+    dft3d::gen::twiddle(R, R, p->sign, T.data());
+    const double tscale = std::ldexp(1.0, -(10 + sh));
+    for (size_t i = 0; i < T.size(); ++i) tw[i] = float(T[i] * tscale);
+    ax.out_mul = float(std::ldexp(1.0, sh - 10) * (scaled ? 1.0 / double(n) : 1.0));
+    DFT3D_CUDA(cudaMalloc(&ax.d_w, W.size() * sizeof(__half)));
+    DFT3D_CUDA(cudaMemcpy(ax.d_w, W.data(), W.size() * sizeof(__half), cudaMemcpyHostToDevice));
+    DFT3D_CUDA(cudaMalloc(&ax.d_tw, tw.size() * sizeof(float)));
+    DFT3D_CUDA(cudaMemcpy(ax.d_tw, tw.data(), tw.size() * sizeof(float), cudaMemcpyHostToDevice));
+    if (RX == 2) {
+      std::vector<float> tw2(size_t(2) * R * R);
+      for (long long m = 0; m < (long long)R * R; ++m) {
+        double re, im;
+        dft3d::gen::root_of_unity(m, n, p->sign, &re, &im);
+        tw2[2 * m] = float(re);
+        tw2[2 * m + 1] = float(im);
+      }
+      DFT3D_CUDA(cudaMalloc(&ax.d_tw2, tw2.size() * sizeof(float)));
+      DFT3D_CUDA(cudaMemcpy(ax.d_tw2, tw2.data(), tw2.size() * sizeof(float), cudaMemcpyHostToDevice));
+    }
+    const unsigned long long dims[2] = {64ull, (unsigned long long)(2 * NB)};
+    const unsigned long long strides[1] = {128ull};
+    const unsigned box[2] = {64u, unsigned(NB)};
+    return encode_map(&ax.map_w, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, ax.d_w, 2, dims, strides, box, 128);
+  }
   std::vector<double> M(size_t(2) * R * R), T(size_t(2) * R * R);
   std::vector<float> hi(size_t(K) * K), lo(size_t(K) * K), W(size_t(2) * panels * NB * 32), tw(size_t(2) * R * R);
   dft3d::gen::axis_matrix(R, p->sign, scaled ? 1.0 / R : 1.0, nullptr, false, M.data());
@@ -420,7 +485,8 @@ int fft_cols_for(const dft3d_plan_s* p, int axis, int layout) {
   return cols;
 }
 
-int fft_axis_pass(dft3d_plan_s* p, int axis, const float* in, float* out, cudaStream_t stream, int layout = FFT_NATURAL) {
+int fft_axis_pass(dft3d_plan_s* p, int axis, const float* in, float* out, cudaStream_t stream, int chain_pos,
+                  int layout = FFT_NATURAL) {
   const FftAxis& ax = p->fax[axis];
   const int R = ax.R, RX = ax.RX, N = int(ax.n), Lg = 128 / (R * RX);
   const int cols = fft_cols_for(p, axis, layout);
@@ -493,6 +559,40 @@ int fft_axis_pass(dft3d_plan_s* p, int axis, const float* in, float* out, cudaSt
     }
   }
   if (rc != DFT3D_OK) return rc;
+  if (p->f16) {
+    // fp16 pieces: two stage-2 operand buffers and a 128 KB raw ring at every size
+    dft3d::FftF16Params hp;
+    hp.base = fp;
+    hp.out_mul = ax.out_mul;
+    hp.base.raw_stages = dft3d::kFft16RawBytes / fp.stage_bytes;
+    if (hp.base.raw_stages > 4) hp.base.raw_stages = 4;
+    const int grid = int(fp.num_stages < p->sm_count ? fp.num_stages : p->sm_count);
+    const size_t smem = dft3d::fft16_smem_bytes(R);
+#define DFT3D_FFT16_LAUNCH(MODE, R_, RX_, COLS_, SO_)                                         \
+  dft3d::fft_f16_axis_kernel<MODE, R_, RX_, COLS_, SO_>                                        \
+      <<<grid, dft3d::kFftThreads, smem, stream>>>(map_data, ax.map_w, map_out, hp)
+    if (axis == 2) {
+      if (R == 32 && RX == 1) DFT3D_FFT16_LAUNCH(dft3d::FFT_CONTIG, 32, 1, 16, 0);
+      else if (R == 16 && RX == 1) DFT3D_FFT16_LAUNCH(dft3d::FFT_CONTIG, 16, 1, 16, 0);
+      else if (R == 32) DFT3D_FFT16_LAUNCH(dft3d::FFT_CONTIG, 32, 2, 16, 0);
+      else DFT3D_FFT16_LAUNCH(dft3d::FFT_CONTIG, 16, 2, 16, 0);
+    } else if (!stage_out) {
+      if (R == 32 && RX == 1 && cols == 16) DFT3D_FFT16_LAUNCH(dft3d::FFT_STRIDED, 32, 1, 16, 0);
+      else if (R == 32 && RX == 1) DFT3D_FFT16_LAUNCH(dft3d::FFT_STRIDED, 32, 1, 8, 0);
+      else if (R == 16 && RX == 1) DFT3D_FFT16_LAUNCH(dft3d::FFT_STRIDED, 16, 1, 16, 0);
+      else if (R == 32) DFT3D_FFT16_LAUNCH(dft3d::FFT_STRIDED, 32, 2, 8, 0);
+      else DFT3D_FFT16_LAUNCH(dft3d::FFT_STRIDED, 16, 2, 16, 0);
+    } else {
+      if (R == 32 && RX == 1 && cols == 16) DFT3D_FFT16_LAUNCH(dft3d::FFT_STRIDED, 32, 1, 16, 1);
+      else if (R == 32 && RX == 1) DFT3D_FFT16_LAUNCH(dft3d::FFT_STRIDED, 32, 1, 8, 1);
+      else if (R == 16 && RX == 1) DFT3D_FFT16_LAUNCH(dft3d::FFT_STRIDED, 16, 1, 16, 1);
+      else if (R == 32) DFT3D_FFT16_LAUNCH(dft3d::FFT_STRIDED, 32, 2, 8, 1);
+      else DFT3D_FFT16_LAUNCH(dft3d::FFT_STRIDED, 16, 2, 16, 1);
+    }
+#undef DFT3D_FFT16_LAUNCH
+    DFT3D_CUDA(cudaGetLastError());
+    return DFT3D_OK;
+  }
   int nb2 = (axis == 2 || R == 16 || (R == 32 && RX == 1 && cols == 8)) ? 2 : 1;
   if (axis != 2 && R == 32 && RX == 1 && cols == 8) {
     // 8-line stages: two stage-2 operand buffers and one raw stage (best with direct stores), or one operand
@@ -629,9 +729,8 @@ int dft3d_plan_create_ex(dft3d_plan_t* out, long long n0, long long n1, long lon
     return fail(DFT3D_ERR_INVALID_ARG, "unknown flag");
   if ((opt.flags & DFT3D_SPLIT_FP16) && (opt.flags & DFT3D_SPLIT_TF32))
     return fail(DFT3D_ERR_INVALID_ARG, "DFT3D_SPLIT_FP16 and DFT3D_SPLIT_TF32 exclude each other");
-  if ((opt.flags & DFT3D_SPLIT_FP16) && mode != DFT3D_KDFT)
-    return fail(DFT3D_ERR_UNSUPPORTED, "DFT3D_SPLIT_FP16 applies to the KDFT formulation");
-  bool f16 = mode == DFT3D_KDFT && !(opt.flags & DFT3D_SPLIT_TF32);   // default where the sizes allow it
+  // default: fp16 pieces for KDFT where the sizes allow it; the FFT formulation uses them on request
+  bool f16 = mode == DFT3D_KDFT ? !(opt.flags & DFT3D_SPLIT_TF32) : (opt.flags & DFT3D_SPLIT_FP16) != 0;
   if (opt.axes > 7) return fail(DFT3D_ERR_INVALID_ARG, "axes must be a mask of bits 0..2");
   const unsigned axes = opt.axes ? opt.axes : 7u;
   for (int a = 0; a < 3; ++a) {
@@ -753,10 +852,10 @@ int dft3d_execute_axis(dft3d_plan_t p, int axis, const void* in, void* out, void
   if (!((p->axes >> axis) & 1u)) return fail(DFT3D_ERR_INVALID_ARG, "axis %d is not among the plan's axes", axis);
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   if (p->mode == DFT3D_KDFT) {
-    if ((rc = kdft_prepare_scales(p, static_cast<const float*>(in), stream)) != DFT3D_OK) return rc;
+    if ((rc = prepare_scales(p, static_cast<const float*>(in), stream)) != DFT3D_OK) return rc;
     return kdft_axis_pass(p, axis, static_cast<const float*>(in), static_cast<float*>(out), p->n[0], stream, 0);
   }
-  return fft_axis_pass(p, axis, static_cast<const float*>(in), static_cast<float*>(out), stream);
+  return fft_axis_pass(p, axis, static_cast<const float*>(in), static_cast<float*>(out), stream, 0);
 }
 
 int dft3d_execute(dft3d_plan_t p, const void* in, void* out, void* cuda_stream) {
@@ -770,7 +869,7 @@ int dft3d_execute(dft3d_plan_t p, const void* in, void* out, void* cuda_stream) 
     const long long g = p->group_planes;
     const long long plane_floats = p->n[1] * p->n[2] * 2;
     float* ws = static_cast<float*>(p->workspace);
-    if ((rc = kdft_prepare_scales(p, fin, stream)) != DFT3D_OK) return rc;
+    if ((rc = prepare_scales(p, fin, stream)) != DFT3D_OK) return rc;
     // the last argument is the pass's position in the chain (fp16 pieces: every pass reads the largest magnitude its
     // predecessor recorded; a later group of planes may read a value that earlier groups already raised, which is
     // still an upper bound for its own data)
@@ -804,14 +903,15 @@ int dft3d_execute(dft3d_plan_t p, const void* in, void* out, void* cuda_stream) 
     // with a cube of workspace: axis 0 in -> out (blocked order: its far-apart rows are only read, never written
     // piecewise), axis 1 out -> workspace (natural order), axis 2 workspace -> out
     float* ws = static_cast<float*>(p->workspace);
-    if ((rc = fft_axis_pass(p, 0, fin, fout, stream, FFT_OUT_BLOCKED)) != DFT3D_OK) return rc;
-    if ((rc = fft_axis_pass(p, 1, fout, ws, stream, FFT_IN_BLOCKED)) != DFT3D_OK) return rc;
-    return fft_axis_pass(p, 2, ws, fout, stream);
+    if ((rc = fft_axis_pass(p, 0, fin, fout, stream, 0, FFT_OUT_BLOCKED)) != DFT3D_OK) return rc;
+    if ((rc = fft_axis_pass(p, 1, fout, ws, stream, 1, FFT_IN_BLOCKED)) != DFT3D_OK) return rc;
+    return fft_axis_pass(p, 2, ws, fout, stream, 2);
   }
   const float* src = fin;
+  int chain_pos = 0;
   for (int a = 2; a >= 0; --a) {
     if (!((axes >> a) & 1u)) continue;
-    if ((rc = fft_axis_pass(p, a, src, fout, stream)) != DFT3D_OK) return rc;
+    if ((rc = fft_axis_pass(p, a, src, fout, stream, chain_pos++)) != DFT3D_OK) return rc;
     src = fout;
   }
   return DFT3D_OK;
@@ -845,14 +945,14 @@ size_t dft3d_plan_workspace_bytes(dft3d_plan_t p) { return p ? p->workspace_byte
 int dft3d_plan_launches(dft3d_plan_t p) {
   if (!p) return 0;
   const int count = int((p->axes & 1u) + ((p->axes >> 1) & 1u) + ((p->axes >> 2) & 1u));
-  const int pre = p->f16 ? 1 : 0;   // the reduction that finds the largest input magnitude
+  const int pre = (p->f16 && p->mode == DFT3D_KDFT) ? 1 : 0;   // the reduction that finds the largest input magnitude
   if (p->mode == DFT3D_KDFT && p->axes == 7u) return pre + int(1 + 2 * (p->n[0] / p->group_planes));
   if (p->mode == DFT3D_KDFT && p->axes == 6u) return pre + int(2 * (p->n[0] / p->group_planes));
   return pre + count;
 }
 
 int dft3d_plan_split(dft3d_plan_t p) {
-  if (!p || p->mode != DFT3D_KDFT) return 0;
+  if (!p) return 0;
   return p->f16 ? DFT3D_SPLIT_FP16 : DFT3D_SPLIT_TF32;
 }
 
