@@ -38,6 +38,8 @@ def parse_args():
     ap.add_argument("--n", type=int, default=1024)
     ap.add_argument("--shape", type=str, default=None, help="n0,n1,n2 instead of a cube (profiling on smaller cases)")
     ap.add_argument("--no-kdft", action="store_true", help="FFT mode only: skip the KDFT timing of the same cube")
+    ap.add_argument("--split", choices=["default", "fp16", "tf32"], default="default",
+                    help="operand split of the tensor-core products (default: the library's choice per formulation)")
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing leg")
@@ -54,7 +56,8 @@ def conv_flops(n):
 # points of that launch; smaller cases than the bench workload, traffic grows in proportion to the points):
 #   profiles/fft_axis_kernel_256x1024x1024.md : (2.148 + 2.094) GB / 268.4 M points
 #   profiles/kdft_axis_kernel_512.md          : (1.084 + 1.035) GB / 134.2 M points
-NCU_DRAM_BYTES_PER_POINT = {"fft_axis_kernel": 15.80, "kdft_axis_kernel": 15.79, "kdft_f16_axis_kernel": 15.79}
+NCU_DRAM_BYTES_PER_POINT = {"fft_axis_kernel": 15.80, "fft_f16_axis_kernel": 15.82, "kdft_axis_kernel": 15.79,
+                            "kdft_f16_axis_kernel": 15.79}
 
 
 def measured_peaks():
@@ -196,7 +199,9 @@ def main():
 
     def time_mode(mode_name, steps, warmup, sample_clocks):
         """W warm-up steps, then K timed steps between barriers; CUDA events on the launching stream; max over ranks."""
-        plan_ = dft.Plan(*shape, mode=dft.DFT3D_KDFT if mode_name == "kdft" else dft.DFT3D_FFT, sign=dft.DFT3D_FORWARD)
+        flags = {"default": 0, "fp16": dft.DFT3D_SPLIT_FP16, "tf32": dft.DFT3D_SPLIT_TF32}[args.split]
+        plan_ = dft.Plan(*shape, mode=dft.DFT3D_KDFT if mode_name == "kdft" else dft.DFT3D_FFT, sign=dft.DFT3D_FORWARD,
+                         flags=flags)
         for _ in range(warmup):
             plan_.execute(x, y)
         barrier()
@@ -278,9 +283,10 @@ def main():
             # only kernel: fft_axis_kernel, one launch per axis; algorithmic traffic 16 B per point per axis
             algo_bytes = 3 * 16.0 * P
             achieved = algo_bytes / (ms_step * 1e-3) * 1e-9
-            roofline = {"bound": "hbm", "kernel": "fft_axis_kernel", "achieved": achieved, "peak": peaks["hbm_gbs"],
+            fkernel = "fft_f16_axis_kernel" if plan.split == dft.DFT3D_SPLIT_FP16 else "fft_axis_kernel"
+            roofline = {"bound": "hbm", "kernel": fkernel, "achieved": achieved, "peak": peaks["hbm_gbs"],
                         "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
-                        "traffic": NCU_DRAM_BYTES_PER_POINT["fft_axis_kernel"] * P,
+                        "traffic": NCU_DRAM_BYTES_PER_POINT[fkernel] * P,
                         "traffic_note": "DRAM bytes per launch, ncu capture at 256x1024x1024 scaled by points",
                         "peak_source": "%s STREAM-style copy" % peak_kind, "avg_launch_ms": ms_step / launches,
                         "bytes": "8 B read + 8 B written per point per axis pass"}
@@ -296,7 +302,7 @@ def main():
         line = {"metric": "3D C2C DFT GFLOP/s (5*P*log2P) at %s" % wl,
                 "value": world * conv_flops(shape) / ms_step * 1e-6, "unit": "GFLOP/s", "n_gpus": world,
                 "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
-                "scaling": "weak", "vs_baseline": None, "dtype": "tf32x3", "data": "synthetic",
+                "scaling": "weak", "vs_baseline": None, "dtype": "fp16x3" if plan.split == dft.DFT3D_SPLIT_FP16 else "tf32x3", "data": "synthetic",
                 "config": {"workload": "%s forward 3D complex64 DFT %s, re/im iid U(-1,1), seed 1003+rank" % (mode.upper(), wl),
                            "mode": mode, "shape": list(shape),
                            "l2": "input and output (%.2f GiB each) are larger than L2" % (P * 8 / 2**30),

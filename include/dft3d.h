@@ -49,12 +49,12 @@ enum {
                                    evaluation points, integer powers).  Default is M[k,j] = exp(s*2*pi*i * k * node[j])
                                    (nonuniform input samples, integer output frequencies). */
   DFT3D_UNSCALED_INVERSE = 2u,  /* sign=+1 without the 1/n_a factors */
-  /* KDFT operand split (the "decompose and accumulate" of Section II-A).  Both use 3 products of 11-bit pieces with
-     fp32 accumulation and meet the same error bound.  Default: fp16 pieces when every transformed n_a % 4 == 0,
-     TF32 pieces otherwise. */
-  DFT3D_SPLIT_FP16 = 4u,        /* insist on fp16 pieces (operands scaled by powers of two from the largest input
-                                   magnitude; half the tensor-core instructions of TF32); DFT3D_ERR_UNSUPPORTED when
-                                   a transformed n_a is not a multiple of 4 */
+  /* Operand split of the tensor-core products (the "decompose and accumulate" of Section II-A).  Both use 3
+     products of 11-bit pieces with fp32 accumulation and meet the same error bound.  Default: fp16 pieces (KDFT:
+     when every transformed n_a % 4 == 0, TF32 pieces otherwise). */
+  DFT3D_SPLIT_FP16 = 4u,        /* insist on fp16 pieces (operands scaled by exact powers of two: KDFT from the largest
+                                   input magnitude, FFT per line; half the tensor-core instructions of TF32);
+                                   DFT3D_ERR_UNSUPPORTED for KDFT when a transformed n_a is not a multiple of 4 */
   DFT3D_SPLIT_TF32 = 8u         /* insist on TF32 pieces (no scaling; every element keeps ~22 significant bits
                                    whatever the dynamic range of the input) */
 };
@@ -139,7 +139,7 @@ size_t dft3d_plan_workspace_bytes(dft3d_plan_t plan);
  * that finds the largest input magnitude before the first axis pass. */
 int dft3d_plan_launches(dft3d_plan_t plan);
 
-/* DFT3D_SPLIT_FP16 or DFT3D_SPLIT_TF32: the operand split a KDFT plan uses; 0 for an FFT plan or NULL. */
+/* DFT3D_SPLIT_FP16 or DFT3D_SPLIT_TF32: the operand split the plan uses; 0 for NULL. */
 int dft3d_plan_split(dft3d_plan_t plan);
 
 /* Frees device and host memory of the plan.  NULL is accepted. */

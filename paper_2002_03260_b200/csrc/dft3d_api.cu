@@ -480,6 +480,9 @@ int fft_cols_for(const dft3d_plan_s* p, int axis, int layout) {
     // measured at 1024^3: natural layout, rows >= 1 MiB apart: 16; otherwise (close rows, or the blocked layout
     // where every stage is one contiguous block) 8-line stages, which leave room to load the next stage early
     cols = env ? atoi(env) : ((layout == FFT_NATURAL && C * 8 >= (1ll << 20)) ? 16 : 8);
+    // fp16 kernel, axis 0 into the blocked layout: 128-byte pieces of the far-apart input rows (half as many address
+    // translations per byte); the stage is free again as soon as it has been split
+    if (!env && p->f16 && layout == FFT_OUT_BLOCKED) cols = 16;
     if (cols != 8 && cols != 16) cols = 16;
   }
   return cols;
@@ -530,14 +533,14 @@ int fft_axis_pass(dft3d_plan_s* p, int axis, const float* in, float* out, cudaSt
     const unsigned long long strides[2] = {(unsigned long long)(C * 8), (unsigned long long)N * C * 8ull};
     const unsigned box[3] = {unsigned(2 * cols), 256u, 1u};
     if (layout == FFT_IN_BLOCKED) {
-      // `in` = T[tile][k0][colsA] written by the axis-0 pass; this stage is (k0 = batch, n2 tile) and its rows are n1
+      // `in` = T[n2 tile][i1][k0][colsA] written by the axis-0 pass; this stage is (k0 = batch, n2 tile) and its rows are i1
       const int colsA = fft_cols_for(p, 0, FFT_OUT_BLOCKED);
       const long long n0 = p->n[0], n1 = p->n[1], n2 = p->n[2];
       const unsigned long long bdims[4] = {(unsigned long long)(2 * colsA), (unsigned long long)n0,
-                                           (unsigned long long)(n2 / colsA), (unsigned long long)n1};
+                                           (unsigned long long)n1, (unsigned long long)(n2 / colsA)};
       const unsigned long long bstr[3] = {(unsigned long long)(colsA * 8), (unsigned long long)(n0 * colsA * 8),
-                                          (unsigned long long)(n2 * n0 * 8)};
-      const unsigned bbox[4] = {unsigned(2 * cols), 1u, 1u, 256u};
+                                          (unsigned long long)(n1 * n0 * colsA * 8)};
+      const unsigned bbox[4] = {unsigned(2 * cols), 1u, 256u, 1u};
       rc = encode_f32(&map_data, in, 4, bdims, bstr, bbox, cols * 8);
       fp.in_blocked = 1;
       fp.blk_ratio = colsA / cols;
@@ -550,7 +553,12 @@ int fft_axis_pass(dft3d_plan_s* p, int axis, const float* in, float* out, cudaSt
       const unsigned long long bstr[2] = {(unsigned long long)(cols * 8), (unsigned long long)N * cols * 8ull};
       if (rc == DFT3D_OK) rc = encode_f32(&map_out, out, 3, bdims, bstr, box, cols * 8);
       fp.out_blocked = 1;
-      stage_out = 1;
+      fp.blk_tiles = int(p->n[2] / cols);
+      fp.blk_rows = int(p->n[1]);
+      // TF32 kernel: the stage returns through shared memory and leaves as TMA stores; fp16 kernel: plain stores
+      // from registers (a block is one contiguous region), which frees the raw stage right after the split
+      const char* env = getenv("DFT3D_FFT_STAGE_OUT");
+      stage_out = env ? atoi(env) : (p->f16 ? 0 : 1);
     } else {
       if (rc == DFT3D_OK) rc = encode_f32(&map_out, out, 3, dims, strides, box, cols * 8);
       // rows MiBs apart: send the results out as full rows through TMA stores instead of 32-byte pieces
@@ -566,6 +574,12 @@ int fft_axis_pass(dft3d_plan_s* p, int axis, const float* in, float* out, cudaSt
     hp.out_mul = ax.out_mul;
     hp.base.raw_stages = dft3d::kFft16RawBytes / fp.stage_bytes;
     if (hp.base.raw_stages > 4) hp.base.raw_stages = 4;
+    // a worker group takes every fourth M-tile, i.e. every (4 / tiles per stage)-th stage: that step must divide the
+    // ring length so that the group meets each ring slot in consecutive phases
+    if (fp.mtiles_per_stage == 1 && hp.base.raw_stages != 4) return fail(DFT3D_ERR_UNSUPPORTED, "internal: raw ring of %d stages", hp.base.raw_stages);
+    if (fp.mtiles_per_stage == 2 && hp.base.raw_stages == 3) hp.base.raw_stages = 2;
+    if (fp.mtiles_per_stage != 1 && fp.mtiles_per_stage != 2 && fp.mtiles_per_stage != 4)
+      return fail(DFT3D_ERR_UNSUPPORTED, "internal: %d tiles per stage", fp.mtiles_per_stage);
     const int grid = int(fp.num_stages < p->sm_count ? fp.num_stages : p->sm_count);
     const size_t smem = dft3d::fft16_smem_bytes(R);
 #define DFT3D_FFT16_LAUNCH(MODE, R_, RX_, COLS_, SO_)                                         \
@@ -669,7 +683,8 @@ const char* dft3d_last_error(void) { return g_last_error; }
 #ifdef DFT3D_PROFILE_WAITS
 // diagnostic builds only: copies the MMA issuer's cycle counters [grid][4] = {total, wait acc, wait W, wait data}
 int dft3d_debug_read_profile(dft3d_plan_t p, long long* host, int ctas) {
-  return cudaMemcpy(host, p->d_profile, sizeof(long long) * ctas, cudaMemcpyDeviceToHost) == cudaSuccess ? 0 : 4;
+  if (cudaMemcpy(host, p->d_profile, sizeof(long long) * ctas, cudaMemcpyDeviceToHost) != cudaSuccess) return 4;
+  return cudaMemset(p->d_profile, 0, sizeof(long long) * ctas) == cudaSuccess ? 0 : 4;   // counters restart after a read
 }
 #endif
 
@@ -729,8 +744,8 @@ int dft3d_plan_create_ex(dft3d_plan_t* out, long long n0, long long n1, long lon
     return fail(DFT3D_ERR_INVALID_ARG, "unknown flag");
   if ((opt.flags & DFT3D_SPLIT_FP16) && (opt.flags & DFT3D_SPLIT_TF32))
     return fail(DFT3D_ERR_INVALID_ARG, "DFT3D_SPLIT_FP16 and DFT3D_SPLIT_TF32 exclude each other");
-  // default: fp16 pieces for KDFT where the sizes allow it; the FFT formulation uses them on request
-  bool f16 = mode == DFT3D_KDFT ? !(opt.flags & DFT3D_SPLIT_TF32) : (opt.flags & DFT3D_SPLIT_FP16) != 0;
+  // default: fp16 pieces (KDFT: where the sizes allow it, see below)
+  bool f16 = !(opt.flags & DFT3D_SPLIT_TF32);
   if (opt.axes > 7) return fail(DFT3D_ERR_INVALID_ARG, "axes must be a mask of bits 0..2");
   const unsigned axes = opt.axes ? opt.axes : 7u;
   for (int a = 0; a < 3; ++a) {

@@ -1,59 +1,65 @@
-// The fused FFT axis kernel of fft_kernel.cuh (paper Section III-B, Eq. 17-18: GEMM, phase adjustment, GEMM, all on
-// chip) with fp16 pieces instead of TF32 pieces: x = hi + lo and F_R = W_hi + W_lo with 11-bit significands as
-// before, multiplied by tcgen05.mma kind::f16 (K = 16 per instruction).  Compared with the TF32 kernel this halves
-// the tensor instructions, the tensor-memory stores of the stage-1 operand, the shared-memory bytes of the tables
-// and of the stage-2 operand, and so leaves room (tensor memory and shared memory) to double-buffer both
-// accumulators and the stage-2 operand at every size.
+// The fused FFT axis kernel (paper Section III-B, Eq. 17-18: GEMM, phase adjustment, GEMM, all on chip) with fp16
+// pieces and tile-parallel warp groups.
+//
+// Arithmetic: as in fft_kernel.cuh (n = R*l + beta, k = k1 + R*k2, complex-as-real 2R x 2R matrices, three products
+// hi*hi, lo*hi, hi*lo per K step, fp32 accumulation in tensor memory), but x = hi + lo and F_R = W_hi + W_lo use fp16
+// pieces (11-bit significands, as TF32 has) and tcgen05.mma kind::f16 (K = 16 per instruction): half the tensor
+// instructions, half the tensor-memory stores of the stage-1 operand, half the shared-memory bytes of the tables and
+// of the stage-2 operand.
 //
 // fp16's exponent range is handled with exact powers of two:
 //   * the tables hold 1024 * F_R (real form);
-//   * every line (after the radix-2 butterfly, if there is one) is multiplied by its own 2^(13 - e), e = ilogb(largest
-//     |component| of the line), so every stage-1 operand component lies below 2^14.  A split thread holds its R
-//     elements of the line in registers, so e costs a maximum and a shuffle reduction over the lanes of the line;
+//   * every line (after the radix-2 butterfly, if there is one) is multiplied by its own 2^(13 - e), e = the exponent
+//     of its largest |component|, so every stage-1 operand component lies below 2^14.  A thread holds its R elements
+//     of the line in registers, so e costs a maximum and one reduction over the lanes of the line;
 //   * a stage-1 result is at most R*sqrt(2) times the largest operand component; the twiddle factors carry
-//     2^-(10 + log2(R) - 1), which undoes the table's 1024 and brings the stage-2 operand below 2^15.5 again;
-//   * the store multiplies by 2^(log2(R) - 1 - 10) (times 1/n for a scaled inverse) and by the line's 2^(e - E), which
-//     the split warps leave in a small tagged ring in shared memory for the warps that drain stage 2.
+//     2^-(10 + log2(R) - 1), which undoes the table's 1024 and keeps the stage-2 operand below 2^15.5;
+//   * the store multiplies by 2^(log2(R) - 1 - 10) (times 1/n for a scaled inverse) and by the line's 2^(e - 13).
+// An element more than 2^18 below its line's largest keeps less than full relative precision (its lo piece becomes
+// subnormal: absolute error 2^-38 of the line's largest element), which is invisible in the norm-wise error.
 //
-// Geometry, warp roles, barriers and the radix-2 pre-pass are those of fft_kernel.cuh; the differences are the
-// operand formats and the second buffer of each accumulator:
-//   tensor memory columns: D1 buffers at 0 and 64, D2 buffers at 128 and 192, A1 buffers (hi R columns, lo R columns,
-//                          two K-adjacent fp16 values per column) at 256 and 320
-//   shared memory:         [W: 2 pieces x 2R rows x 128 B] [A2: 2 buffers x (hi, lo) x 128 rows x 128 B] [raw ring]
+// Organisation.  The per-tile chain  split -> MMA 1 -> drain 1 (+twiddle) -> MMA 2 -> drain 2 (+store)  is latency
+// bound when every link is one warp group (the TF32 kernel's design: each group sees one warp per scheduler).  Here
+// four identical worker groups each take every fourth M-tile through ALL the links, so each scheduler always has four
+// independent warps to pick from, and the two MMA issuer threads serve the groups in tile order:
+//   warp 0      TMA producer (raw stages, tables)
+//   warp 1, 2   MMA issuers, stage 1 (A from tensor memory) and stage 2 (A from shared memory)
+//   warp 3      STAGE_OUT only: sends finished stages out as TMA stores
+//   warps 4-19  worker groups g = 0..3 (tile t belongs to group t mod 4)
+// Tensor memory, per group g at column 128*g: D1 at +0 (2R columns), A1 at +64 (hi R columns, lo R columns, two
+// K-adjacent fp16 values per column); D2 reuses A1's columns (stage 1 has consumed them by then).
+// Shared memory: [W: 2 pieces x 2R rows x 128 B] [A2: 2 buffers x (hi, lo) x 128 rows x 128 B, used in tile order]
+// [twiddles R x R complex64] [raw ring 128 KB] [barriers].
+// A mbarrier wait tells phases apart by parity only, so nobody may wait on a barrier two phases ahead: every barrier
+// here is waited on in consecutive phases by construction (per-group barriers by that group and the issuers in tile
+// order; a2_empty[h] by group h^2 for every tile of group h; raw_full[s] needs (4 / tiles per stage) to divide the
+// ring length, which the host guarantees).
 #pragma once
 #include <cuda_fp16.h>
 #include "fft_kernel.cuh"
 
 namespace dft3d {
 
-constexpr int kF16TmemD1 = 0, kF16TmemD2 = 128, kF16TmemA1 = 256;
-
 struct FftF16Params {
   FftParams base;               // twiddle: T[k1][beta] * 2^-(10 + log2(R) - 1), unscaled otherwise
   float out_mul;                // 2^(log2(R) - 1 - 10), times 1/n for a scaled inverse
 };
 
-constexpr int kFft16ScaleRing = 16;   // M-tiles whose line scales can be pending between the split and the last drain
-
 struct FftF16Shared {
-  uint64_t raw_full[4], raw_empty[4];
-  uint64_t a1_full[2], a1_empty[2];
-  uint64_t d1_full[2], d1_empty[2];
-  uint64_t a2_full[2], a2_empty[2];
-  uint64_t d2_full[2], d2_empty[2];
+  uint64_t raw_full[4], raw_empty[4], out_ready[4];
+  uint64_t a1_full[4], d1_full[4], a2_full[4], a2_empty[4], d2_full[4], sc_full[4];
   uint64_t w_full;
-  uint64_t out_ready;
   uint32_t tmem_base;
   volatile int abort_flag;
-  // per M-tile and (sub-)line: (tile number + 1) << 32 | float bits of 2^(e - E); written by the split warps
-  volatile unsigned long long line_scale[kFft16ScaleRing][8];
+  float line_scale[4][8];      // STRIDED: per group, 2^(e - 13) of the tile's (sub-)lines, from the split to the store
 };
 
 __host__ __device__ constexpr int fft16_w_bytes(int R) { return 2 * 2 * R * 128; }
+__host__ __device__ constexpr int fft16_tw_bytes(int R) { return R * R * 8; }
 constexpr int kFft16A2Piece = 128 * 128;
 constexpr int kFft16RawBytes = 128 * 1024;
 __host__ __device__ constexpr size_t fft16_smem_bytes(int R) {
-  return size_t(fft16_w_bytes(R)) + 4 * size_t(kFft16A2Piece) + kFft16RawBytes + 1024 + 2048;
+  return size_t(fft16_w_bytes(R)) + 4 * size_t(kFft16A2Piece) + fft16_tw_bytes(R) + kFft16RawBytes + 1024 + 1024;
 }
 
 #define F16_WAIT(bar, parity, code)                                 \
@@ -77,11 +83,14 @@ __host__ __device__ constexpr size_t fft16_smem_bytes(int R) {
     FFT_PROF_END(code)                                                                    \
   }
 
-// (re, im) -> packed fp16 pairs: hi = round to nearest, lo = the remainder rounded to fp16
+// (re, im) -> packed fp16 pairs.  hi = the value rounded to an 11-bit significand with integer arithmetic on the fp32
+// word (exactly representable in fp16 unless it is below 2^-14, where the conversion rounds once more and the
+// remainder piece absorbs nothing: an absolute error below 2^-25), lo = the exact remainder rounded to fp16.
 __device__ __forceinline__ void split_half2(float re, float im, uint32_t& hi, uint32_t& lo) {
-  const __half2 h = __floats2half2_rn(re, im);
-  const float2 hf = __half22float2(h);
-  const __half2 l = __floats2half2_rn(re - hf.x, im - hf.y);
+  const float hr = __uint_as_float((__float_as_uint(re) + 0x1000u) & 0xffffe000u);
+  const float hi_ = __uint_as_float((__float_as_uint(im) + 0x1000u) & 0xffffe000u);
+  const __half2 h = __floats2half2_rn(hr, hi_);
+  const __half2 l = __floats2half2_rn(re - hr, im - hi_);
   hi = *reinterpret_cast<const uint32_t*>(&h);
   lo = *reinterpret_cast<const uint32_t*>(&l);
 }
@@ -100,7 +109,8 @@ fft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_c
   constexpr int a2_piece = kFft16A2Piece;
   uint8_t* smem_w = smem;
   uint8_t* smem_a2 = smem_w + fft16_w_bytes(R);            // buffer i = [hi piece][lo piece] at i * 2 * a2_piece
-  uint8_t* smem_rawring = smem_a2 + 4 * a2_piece;
+  float2* smem_tw = reinterpret_cast<float2*>(smem_a2 + 4 * a2_piece);
+  uint8_t* smem_rawring = reinterpret_cast<uint8_t*>(smem_tw) + fft16_tw_bytes(R);
   FftF16Shared& sh = *reinterpret_cast<FftF16Shared*>(smem_rawring + kFft16RawBytes);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 #ifdef DFT3D_PROFILE_WAITS
@@ -112,25 +122,24 @@ fft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_c
   constexpr int Lg = SL / RX;          // lines of the cube per M-tile
   constexpr int NL = R * R;            // length of a (sub-)line
   constexpr int kRowBytes = COLS * 8;  // STRIDED: bytes of one row of a raw stage
-  constexpr int kD1Warps = 4 * (K / 32);
 
   if (tid == 0) {
     for (int i = 0; i < 4; ++i) {
       ptx::mbar_init(&sh.raw_full[i], 1);
-      ptx::mbar_init(&sh.raw_empty[i], 4 * p.mtiles_per_stage + (STAGE_OUT ? 1 : 0));
-    }
-    ptx::mbar_init(&sh.out_ready, 4);
-    for (int i = 0; i < 2; ++i) {
-      ptx::mbar_init(&sh.a1_full[i], 4); ptx::mbar_init(&sh.a1_empty[i], 1);
-      ptx::mbar_init(&sh.d1_full[i], 1); ptx::mbar_init(&sh.d1_empty[i], kD1Warps);
-      ptx::mbar_init(&sh.a2_full[i], kD1Warps); ptx::mbar_init(&sh.a2_empty[i], 1);
-      ptx::mbar_init(&sh.d2_full[i], 1); ptx::mbar_init(&sh.d2_empty[i], 4);
+      ptx::mbar_init(&sh.raw_empty[i], STAGE_OUT ? 1 : 4 * p.mtiles_per_stage);   // the store warp / the split warps
+      ptx::mbar_init(&sh.sc_full[i], 4);
+      ptx::mbar_init(&sh.out_ready[i], 4 * p.mtiles_per_stage);
+      ptx::mbar_init(&sh.a1_full[i], 4);
+      ptx::mbar_init(&sh.d1_full[i], 1);
+      ptx::mbar_init(&sh.a2_full[i], 4);
+      ptx::mbar_init(&sh.a2_empty[i], 1);
+      ptx::mbar_init(&sh.d2_full[i], 1);
     }
     ptx::mbar_init(&sh.w_full, 1);
     sh.abort_flag = 0;
     ptx::fence_mbar_init();
   }
-  if (tid < kFft16ScaleRing * 8) sh.line_scale[tid >> 3][tid & 7] = 0ull;
+  for (int i = tid; i < R * R; i += kFftThreads) smem_tw[i] = __ldg(p.twiddle + i);
   if (warp == 1) {
     ptx::tmem_alloc(&sh.tmem_base, 512);
     ptx::tmem_relinquish();
@@ -148,139 +157,177 @@ fft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_c
   if ((long long)blockIdx.x < p.num_stages) my_stages = (p.num_stages - 1 - blockIdx.x) / gridDim.x + 1;
   const long long my_mtiles = my_stages * p.mtiles_per_stage;
 
-  // the split warps keep a whole line slice in registers: they take what the producer / issuer group can spare
-  // (setmaxnreg is a warp-group-wide instruction: one call site per group, executed by all four of its warps; an
-  // increase can only take what decreases of the same CTA released: 72 + 120 + 3 x 96 = 5 x 96)
+  // Registers: the workers keep a line slice in registers and take what the first group can spare.  setmaxnreg is a
+  // warp-group-wide instruction (one call site per group, executed by all four of its warps), and an increase can
+  // only take what decreases of the same CTA released: 64 + 4 x 104 = 5 x 96.
   if (warp < 4) {
-  ptx::setmaxnreg_dec<72>();
-  if (warp == 0) {
-    // ------------------------------------------------------------ TMA producer
-    if (lane == 0) {
-      ptx::mbar_arrive_expect_tx(&sh.w_full, uint32_t(fft16_w_bytes(R)));
-      for (int pc = 0; pc < 2; ++pc)                // [piece][2R rows][64 halves]
-        ptx::tma_load_2d(smem_w + pc * kWPiece, &map_w, &sh.w_full, 0, pc * NB);
-      long long i = 0;
-      for (long long sidx = blockIdx.x; sidx < p.num_stages; sidx += gridDim.x, ++i) {
-        const uint32_t s = uint32_t(i % p.raw_stages), ph = uint32_t(i / p.raw_stages) & 1;
-        F16_WAIT(&sh.raw_empty[s], ph ^ 1, 0x501);
-        ptx::mbar_arrive_expect_tx(&sh.raw_full[s], uint32_t(p.stage_bytes));
-        uint8_t* dst = smem_rawring + size_t(s) * p.stage_bytes;
-        if (MODE == FFT_CONTIG) {
-          ptx::tma_load_3d(dst, &map_data, &sh.raw_full[s], 0, 0, int(sidx * Lg));
-        } else {
+    ptx::setmaxnreg_dec<64>();
+    if (warp == 0) {
+      // ---------------------------------------------------------- TMA producer
+      if (lane == 0) {
+        ptx::mbar_arrive_expect_tx(&sh.w_full, uint32_t(fft16_w_bytes(R)));
+        for (int pc = 0; pc < 2; ++pc)                // [piece][2R rows][64 halves]
+          ptx::tma_load_2d(smem_w + pc * kWPiece, &map_w, &sh.w_full, 0, pc * NB);
+        long long i = 0;
+        for (long long sidx = blockIdx.x; sidx < p.num_stages; sidx += gridDim.x, ++i) {
+          const uint32_t s = uint32_t(i % p.raw_stages), ph = uint32_t(i / p.raw_stages) & 1;
+          F16_WAIT(&sh.raw_empty[s], ph ^ 1, 0x501);
+          ptx::mbar_arrive_expect_tx(&sh.raw_full[s], uint32_t(p.stage_bytes));
+          uint8_t* dst = smem_rawring + size_t(s) * p.stage_bytes;
+          if (MODE == FFT_CONTIG) {
+            ptx::tma_load_3d(dst, &map_data, &sh.raw_full[s], 0, 0, int(sidx * Lg));
+          } else {
+            const long long ct = sidx % p.c_tiles, bt = sidx / p.c_tiles;
+            for (int r0 = 0; r0 < p.N; r0 += 256) {
+              if (p.in_blocked)
+                ptx::tma_load_4d(dst + size_t(r0) * kRowBytes, &map_data, &sh.raw_full[s],
+                                 int(ct % p.blk_ratio) * 2 * COLS, int(bt), r0, int(ct / p.blk_ratio));
+              else
+                ptx::tma_load_3d(dst + size_t(r0) * kRowBytes, &map_data, &sh.raw_full[s], int(ct * 2 * COLS), r0, int(bt));
+            }
+            const long long nidx = sidx + gridDim.x;
+            if (p.l2_prefetch && nidx < p.num_stages) {
+              const long long nct = nidx % p.c_tiles, nbt = nidx / p.c_tiles;
+              for (int r0 = 0; r0 < p.N; r0 += 256)
+                ptx::tma_prefetch_l2_3d(&map_data, int(nct * 2 * COLS), r0, int(nbt));
+            }
+          }
+        }
+      }
+    } else if (warp == 1) {
+      // ---------------------------------------------------------- MMA issuer, stage 1: D1[g] = A1[g] (tensor memory) x W
+      if (lane == 0) {
+        const uint32_t idesc = ptx::make_idesc_f16(128, NB);
+        const uint32_t w_addr = ptx::smem_u32(smem_w);
+        // operand descriptors: a K = 16 step advances the start address by 32 bytes = 2 descriptor units
+        const uint64_t wh = ptx::make_kmajor_sw128_desc(w_addr);
+        const uint64_t wl = ptx::make_kmajor_sw128_desc(w_addr + kWPiece);
+        F16_WAIT(&sh.w_full, 0, 0x601);
+        for (long long t = 0; t < my_mtiles; ++t) {
+          const uint32_t g = uint32_t(t) & 3, pk = uint32_t(t >> 2) & 1;
+          F16_WAIT(&sh.a1_full[g], pk, 0x602);
+          ptx::tc_fence_after();
+          const uint32_t d = tmem + g * 128;
+          const uint32_t a_hi = d + 64, a_lo = a_hi + R;
+#pragma unroll
+          for (int k = 0; k < KS; ++k) {
+            ptx::mma_f16_ts(d, a_hi + k * 8, wh + 2 * k, idesc, k != 0);
+            ptx::mma_f16_ts(d, a_lo + k * 8, wh + 2 * k, idesc, 1);
+            ptx::mma_f16_ts(d, a_hi + k * 8, wl + 2 * k, idesc, 1);
+          }
+          ptx::tc_commit(&sh.d1_full[g]);
+        }
+      }
+    } else if (warp == 2) {
+      // ---------------------------------------------------------- MMA issuer, stage 2: D2[g] = A2[t & 1] (shared memory) x W
+      if (lane == 0) {
+        const uint32_t idesc = ptx::make_idesc_f16(128, NB);
+        const uint32_t w_addr = ptx::smem_u32(smem_w);
+        const uint32_t a2_addr = ptx::smem_u32(smem_a2);
+        const uint64_t wh = ptx::make_kmajor_sw128_desc(w_addr);
+        const uint64_t wl = ptx::make_kmajor_sw128_desc(w_addr + kWPiece);
+        const uint64_t ah0 = ptx::make_kmajor_sw128_desc(a2_addr);
+        const uint64_t al0 = ptx::make_kmajor_sw128_desc(a2_addr + a2_piece);
+        constexpr uint64_t kBufStep = uint64_t(2 * a2_piece) >> 4;   // second A2 buffer, in descriptor address units
+        F16_WAIT(&sh.w_full, 0, 0x611);
+        for (long long t = 0; t < my_mtiles; ++t) {
+          const uint32_t g = uint32_t(t) & 3, pk = uint32_t(t >> 2) & 1;
+          F16_WAIT(&sh.a2_full[g], pk, 0x604);
+          ptx::tc_fence_after();
+          const uint64_t ah = ah0 + ((t & 1) ? kBufStep : 0), al = al0 + ((t & 1) ? kBufStep : 0);
+          const uint32_t d = tmem + g * 128 + 64;
+#pragma unroll
+          for (int k = 0; k < KS; ++k) {
+            ptx::mma_f16_ss(d, ah + 2 * k, wh + 2 * k, idesc, k != 0);
+            ptx::mma_f16_ss(d, al + 2 * k, wh + 2 * k, idesc, 1);
+            ptx::mma_f16_ss(d, ah + 2 * k, wl + 2 * k, idesc, 1);
+          }
+          ptx::tc_commit(&sh.a2_empty[g]);
+          ptx::tc_commit(&sh.d2_full[g]);
+        }
+      }
+    } else if (STAGE_OUT) {
+      // ---------------------------------------------------------- warp 3: finished stages leave as TMA stores
+      long long istage = 0;
+      for (long long sidx = blockIdx.x; sidx < p.num_stages; sidx += gridDim.x, ++istage) {
+        const uint32_t s = uint32_t(istage % p.raw_stages), ph = uint32_t(istage / p.raw_stages) & 1;
+        F16_WAIT_WARP(&sh.out_ready[s], ph, 0x902);
+        if (lane == 0) {
+          const uint8_t* stage = smem_rawring + size_t(s) * p.stage_bytes;
           const long long ct = sidx % p.c_tiles, bt = sidx / p.c_tiles;
           for (int r0 = 0; r0 < p.N; r0 += 256) {
-            if (p.in_blocked)
-              ptx::tma_load_4d(dst + size_t(r0) * kRowBytes, &map_data, &sh.raw_full[s],
-                               int(ct % p.blk_ratio) * 2 * COLS, int(bt), int(ct / p.blk_ratio), r0);
+            if (p.out_blocked)
+              ptx::tma_store_3d(&map_out, stage + size_t(r0) * kRowBytes, 0, r0,
+                                int((ct % p.blk_tiles) * p.blk_rows + ct / p.blk_tiles));
             else
-              ptx::tma_load_3d(dst + size_t(r0) * kRowBytes, &map_data, &sh.raw_full[s], int(ct * 2 * COLS), r0, int(bt));
+              ptx::tma_store_3d(&map_out, stage + size_t(r0) * kRowBytes, int(ct * 2 * COLS), r0, int(bt));
           }
-          const long long nidx = sidx + gridDim.x;
-          if (p.l2_prefetch && nidx < p.num_stages) {
-            const long long nct = nidx % p.c_tiles, nbt = nidx / p.c_tiles;
-            for (int r0 = 0; r0 < p.N; r0 += 256)
-              ptx::tma_prefetch_l2_3d(&map_data, int(nct * 2 * COLS), r0, int(nbt));
-          }
+          ptx::tma_store_commit();
+          ptx::tma_store_wait_read();
+          ptx::mbar_arrive(&sh.raw_empty[s]);
         }
+        __syncwarp();
       }
+      if (lane == 0) ptx::tma_store_wait_all();
     }
-  } else if (warp == 1) {
-    // ------------------------------------------------------------ MMA issuer, stage 1 (A from tensor memory)
-    if (lane == 0) {
-      const uint32_t idesc = ptx::make_idesc_f16(128, NB);
-      const uint32_t w_addr = ptx::smem_u32(smem_w);
-      // operand descriptors: a K = 16 step advances the start address by 32 bytes = 2 descriptor units
-      const uint64_t wh = ptx::make_kmajor_sw128_desc(w_addr);
-      const uint64_t wl = ptx::make_kmajor_sw128_desc(w_addr + kWPiece);
-      F16_WAIT(&sh.w_full, 0, 0x601);
-      for (long long t = 0; t < my_mtiles; t += 2) {
-#pragma unroll
-        for (int b = 0; b < 2; ++b) {
-          if (t + b < my_mtiles) {
-            const uint32_t phb = uint32_t(t >> 1) & 1;
-            F16_WAIT(&sh.a1_full[b], phb, 0x602);
-            F16_WAIT(&sh.d1_empty[b], phb ^ 1, 0x603);
-            ptx::tc_fence_after();
-            const uint32_t a_hi = tmem + kF16TmemA1 + b * 64, a_lo = a_hi + R;
-            const uint32_t d = tmem + kF16TmemD1 + b * 64;
-#pragma unroll
-            for (int k = 0; k < KS; ++k) {
-              ptx::mma_f16_ts(d, a_hi + k * 8, wh + 2 * k, idesc, k != 0);
-              ptx::mma_f16_ts(d, a_lo + k * 8, wh + 2 * k, idesc, 1);
-              ptx::mma_f16_ts(d, a_hi + k * 8, wl + 2 * k, idesc, 1);
-            }
-            ptx::tc_commit(&sh.a1_empty[b]);
-            ptx::tc_commit(&sh.d1_full[b]);
-          }
-        }
-      }
-    }
-  } else if (warp == 2) {
-    // ------------------------------------------------------------ MMA issuer, stage 2 (A from shared memory)
-    if (lane == 0) {
-      const uint32_t idesc = ptx::make_idesc_f16(128, NB);
-      const uint32_t w_addr = ptx::smem_u32(smem_w);
-      const uint32_t a2_addr = ptx::smem_u32(smem_a2);
-      const uint64_t wh = ptx::make_kmajor_sw128_desc(w_addr);
-      const uint64_t wl = ptx::make_kmajor_sw128_desc(w_addr + kWPiece);
-      const uint64_t ah = ptx::make_kmajor_sw128_desc(a2_addr);
-      const uint64_t al = ptx::make_kmajor_sw128_desc(a2_addr + a2_piece);
-      constexpr uint64_t kBufStep = uint64_t(2 * a2_piece) >> 4;   // second A2 buffer, in descriptor address units
-      F16_WAIT(&sh.w_full, 0, 0x611);
-      for (long long t = 0; t < my_mtiles; t += 2) {
-#pragma unroll
-        for (int b = 0; b < 2; ++b) {
-          if (t + b < my_mtiles) {
-            const uint32_t phb = uint32_t(t >> 1) & 1;
-            F16_WAIT(&sh.a2_full[b], phb, 0x604);
-            F16_WAIT(&sh.d2_empty[b], phb ^ 1, 0x605);
-            ptx::tc_fence_after();
-            const uint64_t bstep = b ? kBufStep : 0;
-            const uint32_t d = tmem + kF16TmemD2 + b * 64;
-#pragma unroll
-            for (int k = 0; k < KS; ++k) {
-              ptx::mma_f16_ss(d, ah + bstep + 2 * k, wh + 2 * k, idesc, k != 0);
-              ptx::mma_f16_ss(d, al + bstep + 2 * k, wh + 2 * k, idesc, 1);
-              ptx::mma_f16_ss(d, ah + bstep + 2 * k, wl + 2 * k, idesc, 1);
-            }
-            ptx::tc_commit(&sh.a2_empty[b]);
-            ptx::tc_commit(&sh.d2_full[b]);
-          }
-        }
-      }
-    }
-  }
-  } else if (warp < 8) {
-    // ------------------------------------------------------------ split: raw lines -> scaled (hi, lo) fp16 pairs -> A1
-    ptx::setmaxnreg_inc<120>();
-    const int q = warp & 3;
+  } else {
+    // ------------------------------------------------------------ worker groups: every fourth M-tile, start to end
+    ptx::setmaxnreg_inc<104>();
+    const int g = (warp - 4) >> 2;              // group = tile number mod 4
+    const int q = warp & 3;                     // lane quarter of tensor memory this warp may touch
     const int m = q * 32 + lane;
-    const int sl = m / R, beta = m % R;           // stage-1 lane = (sub-line sl, beta), beta fastest
-    const int g = sl / RX, bsel = sl % RX;        // line of the cube within the M-tile; which butterfly output
-    const uint32_t lane_addr = tmem + (uint32_t(q * 32) << 16);
-    long long t = 0;
-    for (long long i = 0; i < my_stages; ++i) {
-      const uint32_t s = uint32_t(i % p.raw_stages), phs = uint32_t(i / p.raw_stages) & 1;
+    // stage-1 lane = (sub-line sl1, beta), beta fastest; stage-2 lane = (sub-line sl2, k1)
+    const int sl1 = m / R, beta = m % R;
+    const int g1 = sl1 / RX, bsel1 = sl1 % RX;  // line of the cube within the M-tile; which butterfly output
+    const int sl2 = (MODE == FFT_CONTIG) ? m / R : m % SL;
+    const int k1 = (MODE == FFT_CONTIG) ? m % R : m / SL;
+    const int g2 = sl2 / RX, bsel2 = sl2 % RX;
+    const uint32_t tm_d1 = tmem + (uint32_t(q * 32) << 16) + g * 128;
+    const uint32_t tm_a1 = tm_d1 + 64;          // A1 (hi | lo), later D2
+    // A2 row of (sl, k1): CONTIG sl*R + k1 ; STRIDED k1*SL + sl (so that stage-2 stores of one k2 touch neighbouring lines).
+    // K position (beta, re/im) = halves 2*beta, 2*beta+1 of the row: 16-byte chunk beta/4 (XORed with row % 8 by the
+    // 128-byte swizzle), word beta%4.  row % 8 takes kSwzPer different values as k1 runs: offsets for each of them.
+    constexpr int row_mul_k1 = (MODE == FFT_CONTIG) ? 1 : SL;
+    constexpr int kSwzPer = (MODE == FFT_CONTIG) ? 8 : (SL >= 8 ? 1 : 8 / SL);
+    uint32_t a2_off[kSwzPer];                   // byte offset of (row of k1 = v, this beta) minus v * row_mul_k1 * 128
+    {
+      const int row_base = (MODE == FFT_CONTIG) ? sl1 * R : sl1;
+      const uint32_t a2_chunk = uint32_t(beta) >> 2;
+      const uint32_t a2_word = uint32_t(beta & 3) * 4u;
+#pragma unroll
+      for (int v = 0; v < kSwzPer; ++v) {
+        const uint32_t r = uint32_t(row_base + v * row_mul_k1) & 7u;
+        a2_off[v] = uint32_t(row_base) * 128u + ((a2_chunk ^ r) << 4) + a2_word;
+      }
+    }
+    const float om1 = pp.out_mul;
+
+    for (long long t = g; t < my_mtiles; t += 4) {
+      const long long istage = t / p.mtiles_per_stage;
+      const int mt = int(t % p.mtiles_per_stage);
+      const long long sidx = (long long)blockIdx.x + istage * gridDim.x;
+      const uint32_t s = uint32_t(istage % p.raw_stages), phs = uint32_t(istage / p.raw_stages) & 1;
+      const uint32_t pk = uint32_t(t >> 2) & 1;
+      uint8_t* stage = smem_rawring + size_t(s) * p.stage_bytes;
+
+      // ---- split: this lane's R elements (after the butterfly when RX == 2) -> scaled fp16 pieces -> A1
       F16_WAIT_WARP(&sh.raw_full[s], phs, 0x701);
-      const uint8_t* stage = smem_rawring + size_t(s) * p.stage_bytes;
-      for (int mt = 0; mt < p.mtiles_per_stage; ++mt, ++t) {
+      float inv_scale;
+      {
         uint32_t base, stride, half;
         if (MODE == FFT_CONTIG) {
-          base = uint32_t(g * p.N + beta) * 8u;
+          base = uint32_t(g1 * p.N + beta) * 8u;
           stride = uint32_t(R) * 8u;
           half = uint32_t(NL) * 8u;
         } else {
-          const int c = mt * Lg + g;                // column within the stage
+          const int c = mt * Lg + g1;               // column within the stage
           const uint32_t swz = (COLS == 16) ? uint32_t(beta & 7) : uint32_t((beta >> 1) & 3);   // TMA swizzle of the row
           base = uint32_t(beta) * kRowBytes + ((uint32_t(c >> 1) ^ swz) << 4) + uint32_t(c & 1) * 8u;
           stride = uint32_t(R) * kRowBytes;
           half = uint32_t(NL) * kRowBytes;
         }
-        // this lane's R elements (after the butterfly when RX == 2), kept in registers: the line's scale comes from
-        // their largest magnitude, reduced over the R lanes (all beta) of the (sub-)line
         float xr[R], xi[R];
-        float mx = 0.0f;
+        float mxf = 0.0f;                           // largest magnitude of this lane's elements
 #pragma unroll
         for (int l = 0; l < R; ++l) {
           const uint2 v = *reinterpret_cast<const uint2*>(stage + base + uint32_t(l) * stride);
@@ -290,7 +337,7 @@ fft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_c
             const uint2 w = *reinterpret_cast<const uint2*>(stage + base + half + uint32_t(l) * stride);
             const float ur = __uint_as_float(v.x), ui = __uint_as_float(v.y);
             const float vr = __uint_as_float(w.x), vi = __uint_as_float(w.y);
-            if (bsel == 0) {
+            if (bsel1 == 0) {
               xr[l] = ur + vr; xi[l] = ui + vi;
             } else {
               const float2 tw = __ldg(p.twiddle2 + l * R + beta);
@@ -298,213 +345,167 @@ fft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_c
               xr[l] = dr * tw.x - di * tw.y; xi[l] = dr * tw.y + di * tw.x;
             }
           }
-          mx = fmaxf(mx, fmaxf(fabsf(xr[l]), fabsf(xi[l])));
+          mxf = fmaxf(mxf, fmaxf(fabsf(xr[l]), fabsf(xi[l])));
         }
-        // the raw stage is refilled by TMA (async proxy): order this thread's reads before that write
-        ptx::fence_proxy_async_smem();
-#pragma unroll
-        for (int o = R / 2; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-        if (lane == 0) ptx::mbar_arrive(&sh.raw_empty[s]);
-        float in_scale = 1.0f;
-        {
-          float inv = 1.0f;
-          if (mx > 0.0f && mx < 3.0e38f) {
-            const int e = max(ilogbf(mx), 13 - 126);    // the scale stops growing at 2^126 (subnormal-sized data)
-            in_scale = ldexpf(1.0f, 13 - e);
-            inv = ldexpf(1.0f, e - 13);
-          }
-          if (beta == 0)
-            sh.line_scale[t % kFft16ScaleRing][sl] = ((unsigned long long)(t + 1) << 32) | __float_as_uint(inv);
+        if (!STAGE_OUT) {
+          // the raw stage is refilled by TMA (async proxy): order this thread's reads before that write
+          ptx::fence_proxy_async_smem();
+          __syncwarp();
+          if (lane == 0) ptx::mbar_arrive(&sh.raw_empty[s]);
         }
-        const uint32_t b = uint32_t(t & 1), phb = uint32_t(t >> 1) & 1;
-        F16_WAIT_WARP(&sh.a1_empty[b], phb ^ 1, 0x702);
-        ptx::tc_fence_after();
-        const uint32_t a_hi = lane_addr + kF16TmemA1 + b * 64, a_lo = a_hi + R;
+        // the line's largest magnitude over its R lanes (all beta), then 2^(13 - e) and 2^(e - 13) from the exponent
+        // field f = e + 127, clamped so that both are normal floats (lines of subnormal-sized data lose nothing:
+        // after the largest safe scaling, 2^126, they are multiples of 2^-23)
+        // (as bits: non-negative floats order like integers)
+        const uint32_t mx = __reduce_max_sync(R == 32 ? 0xffffffffu : (0xffffu << (lane & 16)), __float_as_uint(mxf));
+        const uint32_t f = max(mx >> 23, 14u);
+        const float in_scale = __uint_as_float((267u - f) << 23);
+        inv_scale = __uint_as_float((f - 13u) << 23);
+        if (MODE == FFT_STRIDED) {
+          // the stage-2 lanes of this thread belong to another (sub-)line: exchange through shared memory
+          // (a bounded mbarrier rather than a named barrier: a warp that gave up a wait must not strand the others)
+          if (beta == 0) sh.line_scale[g][sl1] = inv_scale;
+          __syncwarp();
+          if (lane == 0) ptx::mbar_arrive(&sh.sc_full[g]);
+          F16_WAIT_WARP(&sh.sc_full[g], pk, 0x703);
+          inv_scale = sh.line_scale[g][sl2];
+        }
 #pragma unroll
-        for (int l0 = 0; l0 < R; l0 += 16) {      // 16 complex = 16 packed columns per tensor-memory store
+        for (int l0 = 0; l0 < R; l0 += 16) {        // 16 complex = 16 packed columns per tensor-memory store
           uint32_t hw[16], lw[16];
 #pragma unroll
           for (int j = 0; j < 16; ++j) split_half2(xr[l0 + j] * in_scale, xi[l0 + j] * in_scale, hw[j], lw[j]);
-          ptx::tmem_st_32x16(a_hi + l0, hw);
-          ptx::tmem_st_32x16(a_lo + l0, lw);
+          ptx::tmem_st_32x16(tm_a1 + l0, hw);
+          ptx::tmem_st_32x16(tm_a1 + R + l0, lw);
         }
         ptx::tc_wait_st();
         ptx::tc_fence_before();
         __syncwarp();
-        if (lane == 0) ptx::mbar_arrive(&sh.a1_full[b]);
+        if (lane == 0) ptx::mbar_arrive(&sh.a1_full[g]);
       }
-    }
-  } else if (warp >= 8 && warp < 16) {
-    // ------------------------------------------------------------ drain stage 1: twiddle, split, write A2
-    // Two warp groups share the work by k1: group c takes the 16 values k1 = 16c .. 16c+15 (one 32-column chunk of
-    // the accumulator).  For R = 16 there is one chunk and the second group has nothing to do.
-    const int grp = (warp - 8) >> 2;
-    if (grp < K / 32) {
-      const int q = warp & 3;
-      const int m = q * 32 + lane;
-      const int sl = m / R, beta = m % R;
-      const uint32_t lane_addr = tmem + (uint32_t(q * 32) << 16) + kF16TmemD1 + grp * 32;
-      // A2 row of (sl, k1): CONTIG sl*R + k1 ; STRIDED k1*SL + sl (so that stage-2 stores of one k2 touch neighbouring lines)
-      const int row_mul_k1 = (MODE == FFT_CONTIG) ? 1 : SL;
-      const int row_base = ((MODE == FFT_CONTIG) ? sl * R : sl) + grp * 16 * row_mul_k1;
-      // K position (beta, re/im) = halves 2*beta, 2*beta+1 of the row: 16-byte chunk beta/4, word beta%4
-      const uint32_t a2_chunk = uint32_t(beta) >> 2;
-      const uint32_t a2_word = uint32_t(beta & 3) * 4u;
-      float twr[16], twi[16];                        // scaled T[16*grp + j][beta], kept for the whole kernel
+
+      // ---- drain stage 1: twiddle, split, write the stage-2 operand (buffer t & 1)
+      F16_WAIT_WARP(&sh.d1_full[g], pk, 0x801);
+      ptx::tc_fence_after();
+      {
+        uint8_t* a2buf = smem_a2 + size_t(t & 1) * 2 * a2_piece;
 #pragma unroll
-      for (int j = 0; j < 16; ++j) {
-        const float2 w = __ldg(p.twiddle + (grp * 16 + j) * R + beta);
-        twr[j] = w.x; twi[j] = w.y;
-      }
-      for (long long t = 0; t < my_mtiles; ++t) {
-        const uint32_t b = uint32_t(t & 1), phb = uint32_t(t >> 1) & 1;
-        F16_WAIT_WARP(&sh.d1_full[b], phb, 0x801);
-        ptx::tc_fence_after();
-        uint32_t v0[32];
-        ptx::tmem_ld_32x32(lane_addr + b * 64, v0);
-        ptx::tc_wait_ld();
+        for (int c = 0; c < K / 32; ++c) {          // 16 values of k1 per chunk of 32 accumulator columns
+          uint32_t v0[32];
+          ptx::tmem_ld_32x32(tm_d1 + c * 32, v0);
+          ptx::tc_wait_ld();
+          uint32_t ch[16], cl[16];                  // C[k1] for this lane's beta, as packed fp16 pieces
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            const float2 tw = smem_tw[(c * 16 + j) * R + beta];
+            const float br = __uint_as_float(v0[2 * j]);
+            const float bi = __uint_as_float(v0[2 * j + 1]);
+            split_half2(br * tw.x - bi * tw.y, br * tw.y + bi * tw.x, ch[j], cl[j]);
+          }
+          if (c == 0 && t >= 2) {
+            // stage 2 of tile t - 2 (group g ^ 2) must be done reading this buffer
+            F16_WAIT_WARP(&sh.a2_empty[g ^ 2], uint32_t((t - 2) >> 2) & 1, 0x802);
+          }
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            const int k1i = c * 16 + j;
+            uint8_t* dst2 = a2buf + a2_off[k1i % kSwzPer] + k1i * row_mul_k1 * 128;
+            *reinterpret_cast<uint32_t*>(dst2) = ch[j];
+            *reinterpret_cast<uint32_t*>(dst2 + a2_piece) = cl[j];
+          }
+        }
         ptx::tc_fence_before();
-        __syncwarp();
-        if (lane == 0) ptx::mbar_arrive(&sh.d1_empty[b]);
-        uint32_t ch[16], cl[16];                      // C[k1] for this lane's beta, as packed fp16 pieces
-#pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          const float br = __uint_as_float(v0[2 * j]);
-          const float bi = __uint_as_float(v0[2 * j + 1]);
-          split_half2(br * twr[j] - bi * twi[j], br * twi[j] + bi * twr[j], ch[j], cl[j]);
-        }
-        // stage 2 of the M-tile two back must be done reading this A2 buffer
-        F16_WAIT_WARP(&sh.a2_empty[b], phb ^ 1, 0x802);
-        uint8_t* a2buf = smem_a2 + size_t(b) * 2 * a2_piece;
-        int rb = row_base;
-        asm volatile("" : "+r"(rb));                  // recompute the 16 store addresses per tile instead of keeping them live
-#pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          const int row = rb + j * row_mul_k1;
-          const uint32_t off = uint32_t(row) * 128u + ((a2_chunk ^ uint32_t(row & 7)) << 4) + a2_word;
-          *reinterpret_cast<uint32_t*>(a2buf + off) = ch[j];
-          *reinterpret_cast<uint32_t*>(a2buf + a2_piece + off) = cl[j];
-        }
         ptx::fence_proxy_async_smem();                // generic writes -> visible to the MMA's shared-memory reads
         __syncwarp();
-        if (lane == 0) ptx::mbar_arrive(&sh.a2_full[b]);
+        if (lane == 0) ptx::mbar_arrive(&sh.a2_full[g]);
       }
-    }
-  } else if (warp >= 16) {
-    // ------------------------------------------------------------ drain stage 2: undo the scales, store in natural order
-    const int q = warp & 3;
-    const int m = q * 32 + lane;
-    const int sl = (MODE == FFT_CONTIG) ? m / R : m % SL;
-    const int k1 = (MODE == FFT_CONTIG) ? m % R : m / SL;
-    const int g = sl / RX, bsel = sl % RX;
-    const uint32_t lane_addr = tmem + (uint32_t(q * 32) << 16) + kF16TmemD2;
-    const float om1 = pp.out_mul;
-    long long t = 0, istage = 0;
-    for (long long sidx = blockIdx.x; sidx < p.num_stages; sidx += gridDim.x, ++istage) {
-      uint8_t* stage = smem_rawring + size_t(istage % p.raw_stages) * p.stage_bytes;   // STAGE_OUT: results return here
-      for (int mt = 0; mt < p.mtiles_per_stage; ++mt, ++t) {
+
+      // ---- drain stage 2: undo the scales, store in natural order
+      {
         float2* dst;              // &out[line][RX*k1 + bsel]; output k = RX*(k1 + R*k2) + bsel is k2*k2_stride further
         long long k2_stride;
         bool ok;
         if (MODE == FFT_CONTIG) {
-          const long long line = sidx * Lg + g;
+          const long long line = sidx * Lg + g2;
           ok = line < p.rows;
-          dst = reinterpret_cast<float2*>(p.out) + line * p.N + (RX * k1 + bsel);
+          dst = reinterpret_cast<float2*>(p.out) + line * p.N + (RX * k1 + bsel2);
           k2_stride = RX * R;
         } else {
           const long long ct = sidx % p.c_tiles, bt = sidx / p.c_tiles;
-          const long long col = ct * COLS + mt * Lg + g;
+          const long long col = ct * COLS + mt * Lg + g2;
           ok = col < p.C;
-          dst = reinterpret_cast<float2*>(p.out) + (bt * p.N + (RX * k1 + bsel)) * p.C + col;
-          k2_stride = (long long)(RX * R) * p.C;
+          if (p.out_blocked) {
+            // block [k][COLS] number n2tile*blk_rows + i1 of the blocked intermediate: pieces of one block are close
+            // together, so plain stores from registers do (the L2 merges them into full lines)
+            const long long blk = (ct % p.blk_tiles) * p.blk_rows + ct / p.blk_tiles;
+            dst = reinterpret_cast<float2*>(p.out) + (blk * p.N + (RX * k1 + bsel2)) * COLS + (mt * Lg + g2);
+            k2_stride = (long long)(RX * R) * COLS;
+          } else {
+            dst = reinterpret_cast<float2*>(p.out) + (bt * p.N + (RX * k1 + bsel2)) * p.C + col;
+            k2_stride = (long long)(RX * R) * p.C;
+          }
         }
-        const uint32_t b = uint32_t(t & 1), phb = uint32_t(t >> 1) & 1;
-        F16_WAIT_WARP(&sh.d2_full[b], phb, 0x901);
+        // one factor when the product of the two is a normal float (always, except for subnormal-sized data)
+        float om = om1 * inv_scale, om_b = 1.0f;
+        if (!(om >= 1.1754944e-38f)) { om = om1; om_b = inv_scale; }
+        F16_WAIT_WARP(&sh.d2_full[g], pk, 0x901);
         ptx::tc_fence_after();
-        // this line's scale; the split warps wrote it long ago (the tag guards against reading a slot too early)
-        float out_mul2;
-        {
-          unsigned long long sv;
-          bool seen;
-          const long long t0 = clock64();
-          for (;;) {
-            sv = sh.line_scale[t % kFft16ScaleRing][sl];
-            seen = (sv >> 32) == (unsigned long long)(t + 1);
-            if (seen || sh.abort_flag || clock64() - t0 > 4000000000LL) break;
-          }
-          if (!__all_sync(0xffffffffu, seen ? 1 : 0)) {
-            sh.abort_flag = 1;
-            atomicCAS(p.status, 0u, 0x903u);
-            goto role_done;
-          }
-          out_mul2 = __uint_as_float(uint32_t(sv));
-        }
 #pragma unroll
         for (int ch = 0; ch < K / 32; ++ch) {
           uint32_t v0[32];
-          ptx::tmem_ld_32x32(lane_addr + b * 64 + ch * 32, v0);
+          ptx::tmem_ld_32x32(tm_a1 + ch * 32, v0);
           ptx::tc_wait_ld();
-          if (ch == K / 32 - 1) {
-            ptx::tc_fence_before();
-            __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(&sh.d2_empty[b]);
-          }
           float f[32];
 #pragma unroll
-          for (int j = 0; j < 32; ++j) f[j] = (__uint_as_float(v0[j]) * om1) * out_mul2;
+          for (int j = 0; j < 32; ++j) f[j] = __uint_as_float(v0[j]) * om;
+          if (om_b != 1.0f) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) f[j] *= om_b;
+          }
           if (STAGE_OUT) {
             // element (row k, column c) of the stage, in the layout TMA wrote the input in (same swizzle)
-            const int c = mt * Lg + g;
+            const int c = mt * Lg + g2;
 #pragma unroll
             for (int j = 0; j < 16; ++j) {
-              const int k = RX * (k1 + R * (ch * 16 + j)) + bsel;
+              const int k = RX * (k1 + R * (ch * 16 + j)) + bsel2;
               const uint32_t swz = (COLS == 16) ? uint32_t(k & 7) : uint32_t((k >> 1) & 3);
               const uint32_t off = uint32_t(k) * kRowBytes + ((uint32_t(c >> 1) ^ swz) << 4) + uint32_t(c & 1) * 8u;
               *reinterpret_cast<float2*>(stage + off) = make_float2(f[2 * j], f[2 * j + 1]);
             }
           } else if (ok) {
-            float2* pd = dst + (long long)(ch * 16) * k2_stride;
+            if (MODE == FFT_CONTIG) {
+              float2* pd = dst + ch * 16 * (RX * R);  // compile-time stride: immediate offsets
 #pragma unroll
-            for (int j = 0; j < 16; ++j) {
-              *pd = make_float2(f[2 * j], f[2 * j + 1]);
-              pd += k2_stride;
-              asm volatile("" : "+l"(pd));            // one running pointer, not sixteen precomputed ones
+              for (int j = 0; j < 16; ++j) pd[j * (RX * R)] = make_float2(f[2 * j], f[2 * j + 1]);
+            } else {
+              float2* pd = dst + (long long)(ch * 16) * k2_stride;
+#pragma unroll
+              for (int j = 0; j < 16; ++j) {
+                *pd = make_float2(f[2 * j], f[2 * j + 1]);
+                pd += k2_stride;
+                asm volatile("" : "+l"(pd));          // one running pointer, not sixteen precomputed ones
+              }
             }
           }
         }
-      }
-      if (STAGE_OUT) {
-        ptx::fence_proxy_async_smem();
-        __syncwarp();
-        if (lane == 0) ptx::mbar_arrive(&sh.out_ready);
-        if (warp == 16) {
-          F16_WAIT_WARP(&sh.out_ready, uint32_t(istage) & 1, 0x902);
-          if (lane == 0) {
-            const long long ct = sidx % p.c_tiles, bt = sidx / p.c_tiles;
-            for (int r0 = 0; r0 < p.N; r0 += 256) {
-              if (p.out_blocked)
-                ptx::tma_store_3d(&map_out, stage + size_t(r0) * kRowBytes, 0, r0, int(ct));
-              else
-                ptx::tma_store_3d(&map_out, stage + size_t(r0) * kRowBytes, int(ct * 2 * COLS), r0, int(bt));
-            }
-            ptx::tma_store_commit();
-            ptx::tma_store_wait_read();
-            ptx::mbar_arrive(&sh.raw_empty[istage % p.raw_stages]);
-          }
+        ptx::tc_fence_before();                       // the next tile's split overwrites these columns
+        if (STAGE_OUT) {
+          ptx::fence_proxy_async_smem();              // generic writes -> visible to the TMA store
           __syncwarp();
+          if (lane == 0) ptx::mbar_arrive(&sh.out_ready[s]);
         }
       }
     }
-    if (STAGE_OUT && warp == 16 && lane == 0) ptx::tma_store_wait_all();
   }
 
 role_done:
 #ifdef DFT3D_PROFILE_WAITS
-  if (p.profile && lane == 0 && (warp <= 2 || (warp & 3) == 0)) {
+  if (p.profile && lane == 0 && (warp <= 3 || (warp & 3) == 0)) {
+    // one reporter per role / group: rows 5..9 by wait code, column by code & 7; workers add up over the groups
     long long* dst = p.profile + size_t(blockIdx.x) * 128;
     for (int i = 5; i < 10; ++i)
       for (int j = 0; j < 8; ++j)
-        if (prof_wait[i][j]) dst[i * 8 + j] = prof_wait[i][j];
+        if (prof_wait[i][j]) atomicAdd(reinterpret_cast<unsigned long long*>(dst + i * 8 + j), (unsigned long long)prof_wait[i][j]);
     if (warp == 0) dst[0] = clock64() - prof_start;
   }
 #endif

@@ -61,11 +61,14 @@ struct FftParams {
   long long C;
   long long c_tiles;     // C / COLS
   int l2_prefetch;       // STRIDED: prefetch the next stage's rows into L2
-  // Blocked intermediate layout T[column tile][row][COLS] (one contiguous block per stage), used between the axis-0
-  // and the axis-1 pass of a 3D transform so that the far-apart rows of axis 0 are only ever READ piecewise:
-  int out_blocked;       // STAGE_OUT: store the stage as block number `column tile` of T (map_out is T's 3D map)
+  // Blocked intermediate layout T[n2 tile][i1][k0][COLS] (one contiguous block [k0][COLS] per axis-0 stage), used
+  // between the axis-0 and the axis-1 pass of a 3D transform so that the far-apart rows of axis 0 are only ever READ
+  // piecewise, and so that the n1 rows an axis-1 stage gathers lie close together (one block apart, not a plane apart):
+  int out_blocked;       // the stage of column tile ct = i1*blk_tiles + n2tile goes to block n2tile*blk_rows + i1 of T
+  int blk_tiles;         // out_blocked: n2 / COLS
+  int blk_rows;          // out_blocked: n1
   int blk_ratio;         // in_blocked: columns of a block of T / COLS of this pass
-  int in_blocked;        // load rows from T through a 4D map {COLS, row-in-block, tile, block row}; batch = row-in-block
+  int in_blocked;        // load rows from T through a 4D map {COLS, k0, i1, n2 tile}; batch = k0
   const float2* twiddle; // [R][R] complex64, T[k1][beta] (times 1/RX for a scaled inverse)
   const float2* twiddle2;// RX == 2: [R*R] complex64, exp(s*2*pi*i*m/N)
   float* out;
@@ -202,7 +205,7 @@ fft_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_const
           for (int r0 = 0; r0 < p.N; r0 += 256) {
             if (p.in_blocked)
               ptx::tma_load_4d(dst + size_t(r0) * kRowBytes, &map_data, &sh.raw_full[s],
-                               int(ct % p.blk_ratio) * 2 * COLS, int(bt), int(ct / p.blk_ratio), r0);
+                               int(ct % p.blk_ratio) * 2 * COLS, int(bt), r0, int(ct / p.blk_ratio));
             else
               ptx::tma_load_3d(dst + size_t(r0) * kRowBytes, &map_data, &sh.raw_full[s], int(ct * 2 * COLS), r0, int(bt));
           }
@@ -489,7 +492,8 @@ fft_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_const
             const long long ct = sidx % p.c_tiles, bt = sidx / p.c_tiles;
             for (int r0 = 0; r0 < p.N; r0 += 256) {
               if (p.out_blocked)
-                ptx::tma_store_3d(&map_out, stage + size_t(r0) * kRowBytes, 0, r0, int(ct));
+                ptx::tma_store_3d(&map_out, stage + size_t(r0) * kRowBytes, 0, r0,
+                                  int((ct % p.blk_tiles) * p.blk_rows + ct / p.blk_tiles));
               else
                 ptx::tma_store_3d(&map_out, stage + size_t(r0) * kRowBytes, int(ct * 2 * COLS), r0, int(bt));
             }

@@ -208,7 +208,7 @@ class Plan:
 
     @property
     def split(self):
-        """DFT3D_SPLIT_FP16 or DFT3D_SPLIT_TF32 for a KDFT plan, 0 for an FFT plan."""
+        """DFT3D_SPLIT_FP16 or DFT3D_SPLIT_TF32: the operand split of the plan's tensor-core products."""
         return int(_lib.dft3d_plan_split(self._h))
 
     def destroy(self):

@@ -43,9 +43,10 @@ def _split_flag(lib, split):
     return lib.DFT3D_SPLIT_FP16 if split == "fp16" else lib.DFT3D_SPLIT_TF32
 
 
-def _pre(lib, plan):
-    """Launches before the axis passes: the fp16 split first reduces the input to its largest magnitude."""
-    return 1 if plan.split == lib.DFT3D_SPLIT_FP16 else 0
+def _pre(lib, plan, kdft=True):
+    """Launches before the axis passes: the fp16 split of the KDFT kernels first reduces the input to its largest
+    magnitude (the FFT kernels scale line by line inside the pass)."""
+    return 1 if (kdft and plan.split == lib.DFT3D_SPLIT_FP16) else 0
 
 
 # ------------------------------------------------------------------ single axes (each kernel variant alone)
@@ -203,9 +204,11 @@ def test_execute_host(lib, oracle):
 
 @pytest.mark.parametrize("shape,axis", [((256, 256, 256), 0), ((256, 256, 256), 1), ((256, 256, 256), 2),
                                         ((256, 256, 1024), 2), ((256, 1024, 256), 1), ((1024, 256, 256), 0)])
-def test_fft_single_axis(lib, oracle, shape, axis):
+@pytest.mark.parametrize("split", SPLITS)
+def test_fft_single_axis(lib, oracle, shape, axis, split):
     x = _inputs().cube(shape, "normal", 61 + axis, device="cuda")
-    plan = lib.Plan(*shape, mode=lib.DFT3D_FFT)
+    plan = lib.Plan(*shape, mode=lib.DFT3D_FFT, flags=_split_flag(lib, split))
+    assert plan.split == _split_flag(lib, split)
     y = plan.execute_axis(axis, x)
     _finish(plan)
     ref = oracle.dft_axis(x.cpu().numpy().astype(np.complex128), axis)
@@ -214,11 +217,13 @@ def test_fft_single_axis(lib, oracle, shape, axis):
     plan.destroy()
 
 
-def test_fft_256_forward_inverse_and_kdft_agreement(lib, oracle):
+@pytest.mark.parametrize("split", SPLITS)
+def test_fft_256_forward_inverse_and_kdft_agreement(lib, oracle, split):
     shape = (256, 256, 256)
+    sf = _split_flag(lib, split)
     x = _inputs().cube(shape, "uniform", 62, device="cuda")
-    fft = lib.Plan(*shape, mode=lib.DFT3D_FFT)
-    kdft = lib.Plan(*shape, mode=lib.DFT3D_KDFT)
+    fft = lib.Plan(*shape, mode=lib.DFT3D_FFT, flags=sf)
+    kdft = lib.Plan(*shape, mode=lib.DFT3D_KDFT, flags=sf)
     y = fft(x)
     z = kdft(x)
     _finish(fft)
@@ -227,11 +232,11 @@ def test_fft_256_forward_inverse_and_kdft_agreement(lib, oracle):
     assert oracle.rel_l2(y.cpu().numpy(), ref) < SANITY
     assert oracle.rel_l2(y.cpu().numpy(), z.cpu().numpy()) < TOL      # the two formulations agree
     assert torch.equal(x, _inputs().cube(shape, "uniform", 62, device="cuda"))  # input untouched
-    inv = lib.Plan(*shape, mode=lib.DFT3D_FFT, sign=lib.DFT3D_INVERSE)
+    inv = lib.Plan(*shape, mode=lib.DFT3D_FFT, sign=lib.DFT3D_INVERSE, flags=sf)
     back = inv(y)
     _finish(inv)
     assert oracle.rel_l2(back.cpu().numpy(), x.cpu().numpy()) < SANITY
-    raw = lib.Plan(*shape, mode=lib.DFT3D_FFT, sign=lib.DFT3D_INVERSE, flags=lib.DFT3D_UNSCALED_INVERSE)
+    raw = lib.Plan(*shape, mode=lib.DFT3D_FFT, sign=lib.DFT3D_INVERSE, flags=lib.DFT3D_UNSCALED_INVERSE | sf)
     w = raw(y)
     _finish(raw)
     assert oracle.rel_l2(w.cpu().numpy() / np.prod(shape), x.cpu().numpy()) < SANITY
@@ -239,15 +244,32 @@ def test_fft_256_forward_inverse_and_kdft_agreement(lib, oracle):
         p.destroy()
 
 
-def test_fft_schedules_agree(lib, oracle):
+@pytest.mark.parametrize("split", SPLITS)
+@pytest.mark.parametrize("shape", [(256, 512, 256), (1024, 256, 256), (512, 1024, 256)])
+def test_fft_schedules_agree(lib, oracle, split, shape):
     """With a cube of workspace the 3D FFT goes in -> out (blocked order) -> workspace -> out; without it the
-    three passes run in place on out.  Both against the oracle."""
-    shape = (256, 512, 256)
+    three passes run in place on out.  The small shape: both against the oracle.  The longer ones (1024-point strided
+    axes, the blocked layout with 16-line and 8-line stages): against each other and against the KDFT kernels, whose
+    single axes are checked against the oracle above."""
+    sf = _split_flag(lib, split)
     x = _inputs().cube(shape, "normal", 66, device="cuda")
+    with_ws = lib.Plan(*shape, mode=lib.DFT3D_FFT, flags=sf)
+    in_place = lib.Plan(*shape, mode=lib.DFT3D_FFT, workspace_limit=1 << 20, flags=sf)
+    assert in_place.workspace_bytes == 0
+    if shape != (256, 512, 256):
+        # (a plan skips the workspace when the stage widths of its axis-0 and axis-1 passes do not nest)
+        a, b = with_ws(x), in_place(x)
+        _finish(with_ws)
+        in_place.status()
+        kd = lib.Plan(*shape, mode=lib.DFT3D_KDFT)
+        c = kd(x)
+        _finish(kd)
+        assert _rel_l2_gpu(a, b) < SANITY and _rel_l2_gpu(a, c) < TOL
+        for plan in (with_ws, in_place, kd):
+            plan.destroy()
+        return
     ref = oracle.dft3d(x.cpu().numpy())
-    with_ws = lib.Plan(*shape, mode=lib.DFT3D_FFT)
-    in_place = lib.Plan(*shape, mode=lib.DFT3D_FFT, workspace_limit=1 << 20)
-    assert with_ws.workspace_bytes == x.numel() * 8 and in_place.workspace_bytes == 0
+    assert with_ws.workspace_bytes == x.numel() * 8
     for plan in (with_ws, in_place):
         y = plan(x)
         _finish(plan)
@@ -255,10 +277,11 @@ def test_fft_schedules_agree(lib, oracle):
         plan.destroy()
 
 
-def test_fft_mixed_axis_lengths(lib, oracle):
+@pytest.mark.parametrize("split", SPLITS)
+def test_fft_mixed_axis_lengths(lib, oracle, split):
     shape = (256, 1024, 256)
     x = _inputs().cube(shape, "normal", 63, device="cuda")
-    plan = lib.Plan(*shape, mode=lib.DFT3D_FFT, fft_split=((16, 16), (32, 32), None))
+    plan = lib.Plan(*shape, mode=lib.DFT3D_FFT, fft_split=((16, 16), (32, 32), None), flags=_split_flag(lib, split))
     y = plan(x)
     _finish(plan)
     assert oracle.rel_l2(y.cpu().numpy(), oracle.dft3d(x.cpu().numpy())) < SANITY
@@ -273,11 +296,12 @@ def test_fft_mixed_axis_lengths(lib, oracle):
 
 @pytest.mark.parametrize("shape,axis", [((256, 256, 512), 2), ((256, 512, 256), 1), ((512, 256, 256), 0),
                                         ((256, 256, 2048), 2), ((256, 2048, 256), 1), ((2048, 256, 256), 0)])
-def test_fft_radix2_lengths_single_axis(lib, oracle, shape, axis):
+@pytest.mark.parametrize("split", SPLITS)
+def test_fft_radix2_lengths_single_axis(lib, oracle, shape, axis, split):
     """N = 2*R*R (512 = 2*16*16, 2048 = 2*32*32): butterfly + two GEMM stages.  The oracle transforms a slab of
     8 lines-worth along an untransformed axis (lines are independent), which keeps the 2048 cases short."""
     x = _inputs().cube(shape, "normal", 64 + axis, device="cuda")
-    plan = lib.Plan(*shape, mode=lib.DFT3D_FFT)
+    plan = lib.Plan(*shape, mode=lib.DFT3D_FFT, flags=_split_flag(lib, split))
     y = plan.execute_axis(axis, x)
     _finish(plan)
     plan.destroy()
@@ -461,7 +485,7 @@ def test_batched_2d(lib, oracle, mode_name, shape):
     plan = lib.Plan(*shape, mode=mode, axes=(1, 2))
     y = plan(x)
     _finish(plan)
-    assert plan.launches == _pre(lib, plan) + 2
+    assert plan.launches == _pre(lib, plan, mode_name == "kdft") + 2
     plan.destroy()
     err = oracle.rel_l2(y.cpu().numpy(), _oracle_axes(oracle, x.cpu().numpy(), (1, 2)))
     assert err < SANITY, (mode_name, shape, err)
@@ -581,3 +605,26 @@ def test_splits_agree_512(lib, oracle):
         plan.destroy()
     diff = torch.linalg.vector_norm((res["fp16"] - res["tf32"]).flatten()) / torch.linalg.vector_norm(res["tf32"].flatten())
     assert diff.item() < SANITY
+
+
+@pytest.mark.parametrize("axis", [1, 2])
+def test_fft_fp16_scales_every_line_on_its_own(lib, oracle, axis):
+    """The fp16 split of the FFT kernel scales each line by a power of two taken from that line's largest element.
+    Lines that differ by up to 2^120 in magnitude must each come out with fp32-level error relative to their OWN norm
+    (a single scale for the whole array would flush the small lines to zero)."""
+    shape = (64, 256, 256)
+    x = _inputs().cube(shape, "normal", 96, device="cuda")
+    g = torch.Generator(device="cuda").manual_seed(97)
+    other = [d for d in range(3) if d != axis]
+    expo = torch.randint(-60, 61, [shape[d] for d in other], generator=g, device="cuda").to(torch.float32)
+    scale = torch.exp2(expo).unsqueeze(axis)
+    xs = (x * scale).contiguous()
+    plan = lib.Plan(*shape, mode=lib.DFT3D_FFT, flags=lib.DFT3D_SPLIT_FP16, axes=(axis,))
+    ys = plan(xs)
+    _finish(plan)
+    plan.destroy()
+    assert bool(torch.isfinite(torch.view_as_real(ys)).all())
+    ref = oracle.dft_axis(x.cpu().numpy().astype(np.complex128), axis)     # unscaled lines: scaling by 2^k is exact
+    got = (ys / scale).cpu().numpy().astype(np.complex128)
+    err = np.sqrt((np.abs(got - ref) ** 2).sum(axis=axis) / (np.abs(ref) ** 2).sum(axis=axis))
+    assert err.max() < SANITY_AXIS, err.max()
