@@ -40,6 +40,9 @@ def parse_args():
     ap.add_argument("--no-kdft", action="store_true", help="FFT mode only: skip the KDFT timing of the same cube")
     ap.add_argument("--split", choices=["default", "fp16", "tf32"], default="default",
                     help="operand split of the tensor-core products (default: the library's choice per formulation)")
+    ap.add_argument("--destroy-input", action="store_true",
+                    help="plans use the input cube as their workspace (DFT3D_DESTROY_INPUT): for sizes where input + "
+                         "output leave no room for one, e.g. 2048^3; the input is not regenerated between steps")
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing leg")
@@ -200,6 +203,8 @@ def main():
     def time_mode(mode_name, steps, warmup, sample_clocks):
         """W warm-up steps, then K timed steps between barriers; CUDA events on the launching stream; max over ranks."""
         flags = {"default": 0, "fp16": dft.DFT3D_SPLIT_FP16, "tf32": dft.DFT3D_SPLIT_TF32}[args.split]
+        if args.destroy_input:
+            flags |= dft.DFT3D_DESTROY_INPUT
         plan_ = dft.Plan(*shape, mode=dft.DFT3D_KDFT if mode_name == "kdft" else dft.DFT3D_FFT, sign=dft.DFT3D_FORWARD,
                          flags=flags)
         for _ in range(warmup):
@@ -306,7 +311,8 @@ def main():
                 "config": {"workload": "%s forward 3D complex64 DFT %s, re/im iid U(-1,1), seed 1003+rank" % (mode.upper(), wl),
                            "mode": mode, "shape": list(shape),
                            "l2": "input and output (%.2f GiB each) are larger than L2" % (P * 8 / 2**30),
-                           "per_rank": "one independent cube per GPU"},
+                           "per_rank": "one independent cube per GPU",
+                           "destroy_input": bool(args.destroy_input)},
                 "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches * args.steps,
                 "clocks": clocks, "kdft": kdft_info}
         print(json.dumps(line))

@@ -55,13 +55,16 @@ enum {
   DFT3D_SPLIT_FP16 = 4u,        /* insist on fp16 pieces (operands scaled by exact powers of two: KDFT from the largest
                                    input magnitude, FFT per line; half the tensor-core instructions of TF32);
                                    DFT3D_ERR_UNSUPPORTED for KDFT when a transformed n_a is not a multiple of 4 */
-  DFT3D_SPLIT_TF32 = 8u         /* insist on TF32 pieces (no scaling; every element keeps ~22 significant bits
+  DFT3D_SPLIT_TF32 = 8u,        /* insist on TF32 pieces (no scaling; every element keeps ~22 significant bits
                                    whatever the dynamic range of the input) */
+  DFT3D_DESTROY_INPUT = 16u     /* dft3d_execute may overwrite `in`: a plan over all three axes then uses the input
+                                   cube as its workspace and allocates none, which keeps the fast schedules available
+                                   when input + output fill the memory (2048^3).  Ignored by plans over fewer axes. */
 };
 
 typedef struct dft3d_options_s {
   size_t struct_size;     /* sizeof(dft3d_options_t), for forward compatibility */
-  unsigned flags;         /* DFT3D_NODES_ON_OUTPUT | DFT3D_UNSCALED_INVERSE | DFT3D_SPLIT_* */
+  unsigned flags;         /* DFT3D_NODES_ON_OUTPUT | DFT3D_UNSCALED_INVERSE | DFT3D_SPLIT_* | DFT3D_DESTROY_INPUT */
   int fft_split[3][2];    /* FFT mode: {N1, N2} per axis with N1*N2 = n_a; {0,0} = default split */
   size_t workspace_limit; /* upper bound in bytes for the plan-owned workspace; 0 = default (16 GiB).  KDFT needs a
                              workspace and shrinks it to groups of n0-planes; FFT uses one cube of workspace when it
@@ -106,7 +109,7 @@ int dft3d_plan_create_ex(dft3d_plan_t* out, long long n0, long long n1, long lon
  * Run the transform (all three axes; Eq. 12 for KDFT, Eq. 17 per axis for FFT).
  *
  *   in, out      DEVICE pointers, 16-byte aligned, n0*n1*n2*8 bytes each, not overlapping.
- *                `in` is only read.
+ *                `in` is only read, unless the plan was created with DFT3D_DESTROY_INPUT.
  *   cuda_stream  a cudaStream_t (NULL = default stream).
  *
  * Asynchronous: kernels are enqueued on the stream and the call returns without

@@ -115,7 +115,8 @@ struct dft3d_plan_s {
   long long n[3] = {0, 0, 0};
   int mode = 0, sign = 0;
   unsigned flags = 0;
-  bool f16 = false;       // KDFT with fp16 pieces (else TF32 pieces)
+  bool f16 = false;       // fp16 pieces (else TF32 pieces)
+  bool in_is_ws = false;  // DFT3D_DESTROY_INPUT: the caller's input buffer serves as the workspace
   unsigned axes = 7;            // bit a: axis a is transformed
   int device = 0;
   int sm_count = 0;
@@ -740,7 +741,7 @@ int dft3d_plan_create_ex(dft3d_plan_t* out, long long n0, long long n1, long lon
       return fail(DFT3D_ERR_INVALID_ARG, "options->struct_size is not a known size");
     memcpy(&opt, options, options->struct_size);
   }
-  if (opt.flags & ~(DFT3D_NODES_ON_OUTPUT | DFT3D_UNSCALED_INVERSE | DFT3D_SPLIT_FP16 | DFT3D_SPLIT_TF32))
+  if (opt.flags & ~(DFT3D_NODES_ON_OUTPUT | DFT3D_UNSCALED_INVERSE | DFT3D_SPLIT_FP16 | DFT3D_SPLIT_TF32 | DFT3D_DESTROY_INPUT))
     return fail(DFT3D_ERR_INVALID_ARG, "unknown flag");
   if ((opt.flags & DFT3D_SPLIT_FP16) && (opt.flags & DFT3D_SPLIT_TF32))
     return fail(DFT3D_ERR_INVALID_ARG, "DFT3D_SPLIT_FP16 and DFT3D_SPLIT_TF32 exclude each other");
@@ -812,6 +813,9 @@ int dft3d_plan_create_ex(dft3d_plan_t* out, long long n0, long long n1, long lon
       const size_t plane_bytes = size_t(n1) * n2 * 8;
       size_t limit = opt.workspace_limit ? opt.workspace_limit : (size_t(16) << 30);
       long long g = n0;
+      // with DFT3D_DESTROY_INPUT the input cube is the workspace once the first pass has read it
+      p->in_is_ws = (opt.flags & DFT3D_DESTROY_INPUT) && axes == 7u;
+      if (p->in_is_ws) limit = ~size_t(0);
       if (size_t(g) * plane_bytes > limit) {
         g = (long long)(limit / plane_bytes);
         if (g < 1) g = 1;
@@ -824,8 +828,8 @@ int dft3d_plan_create_ex(dft3d_plan_t* out, long long n0, long long n1, long lon
       }
       if (axes == 1u || axes == 2u || axes == 4u) g = 0;   // a single axis goes straight from in to out
       p->group_planes = g ? g : n0;
-      p->workspace_bytes = size_t(g) * plane_bytes;
-      if (g != 0) {
+      p->workspace_bytes = p->in_is_ws ? 0 : size_t(g) * plane_bytes;
+      if (g != 0 && !p->in_is_ws) {
         e = cudaMalloc(&p->workspace, p->workspace_bytes);
         if (e != cudaSuccess) { rc = fail(DFT3D_ERR_ALLOC, "cudaMalloc(workspace %zu bytes): %s", p->workspace_bytes, cudaGetErrorString(e)); break; }
       }
@@ -837,7 +841,10 @@ int dft3d_plan_create_ex(dft3d_plan_t* out, long long n0, long long n1, long lon
       // without it the three passes run in place on `out`
       const size_t cube_bytes = size_t(n0) * n1 * n2 * 8;
       const size_t limit = opt.workspace_limit ? opt.workspace_limit : (size_t(16) << 30);
-      if (axes == 7u && cube_bytes <= limit && fft_cols_for(p, 0, FFT_OUT_BLOCKED) % fft_cols_for(p, 1, FFT_IN_BLOCKED) == 0) {
+      const bool nests = fft_cols_for(p, 0, FFT_OUT_BLOCKED) % fft_cols_for(p, 1, FFT_IN_BLOCKED) == 0;
+      if (axes == 7u && nests && (opt.flags & DFT3D_DESTROY_INPUT)) {
+        p->in_is_ws = true;   // in -> out (blocked) -> in (natural) -> out
+      } else if (axes == 7u && cube_bytes <= limit && nests) {
         e = cudaMalloc(&p->workspace, cube_bytes);
         if (e == cudaSuccess) p->workspace_bytes = cube_bytes;
         else { p->workspace = nullptr; (void)cudaGetLastError(); }   // fall back to the in-place schedule
@@ -883,7 +890,7 @@ int dft3d_execute(dft3d_plan_t p, const void* in, void* out, void* cuda_stream) 
   if (p->mode == DFT3D_KDFT) {
     const long long g = p->group_planes;
     const long long plane_floats = p->n[1] * p->n[2] * 2;
-    float* ws = static_cast<float*>(p->workspace);
+    float* ws = p->in_is_ws ? const_cast<float*>(fin) : static_cast<float*>(p->workspace);
     if ((rc = prepare_scales(p, fin, stream)) != DFT3D_OK) return rc;
     // the last argument is the pass's position in the chain (fp16 pieces: every pass reads the largest magnitude its
     // predecessor recorded; a later group of planes may read a value that earlier groups already raised, which is
@@ -914,10 +921,18 @@ int dft3d_execute(dft3d_plan_t p, const void* in, void* out, void* cuda_stream) 
   }
   // FFT: the first transformed axis (last axis first) in -> out, the others in place on out (a CTA loads a group of
   // lines completely into shared memory before it stores any of their results, and groups are disjoint)
-  if (axes == 7u && p->workspace && !getenv("DFT3D_FFT_INPLACE")) {
+  if (axes == 7u && (p->workspace || p->in_is_ws) && !getenv("DFT3D_FFT_INPLACE")) {
     // with a cube of workspace: axis 0 in -> out (blocked order: its far-apart rows are only read, never written
     // piecewise), axis 1 out -> workspace (natural order), axis 2 workspace -> out
-    float* ws = static_cast<float*>(p->workspace);
+    float* ws = p->in_is_ws ? const_cast<float*>(fin) : static_cast<float*>(p->workspace);
+#ifdef DFT3D_PROFILE_WAITS
+    if (const char* only = getenv("DFT3D_DEBUG_ONLY_PASS")) {   // diagnostic builds: one pass of the schedule alone
+      const int k = atoi(only);
+      if (k == 0) return fft_axis_pass(p, 0, fin, fout, stream, 0, FFT_OUT_BLOCKED);
+      if (k == 1) return fft_axis_pass(p, 1, fout, ws, stream, 1, FFT_IN_BLOCKED);
+      return fft_axis_pass(p, 2, ws, fout, stream, 2);
+    }
+#endif
     if ((rc = fft_axis_pass(p, 0, fin, fout, stream, 0, FFT_OUT_BLOCKED)) != DFT3D_OK) return rc;
     if ((rc = fft_axis_pass(p, 1, fout, ws, stream, 1, FFT_IN_BLOCKED)) != DFT3D_OK) return rc;
     return fft_axis_pass(p, 2, ws, fout, stream, 2);

@@ -83,14 +83,37 @@ __host__ __device__ constexpr size_t fft16_smem_bytes(int R) {
     FFT_PROF_END(code)                                                                    \
   }
 
+// Two fp32 values in one 64-bit register for the packed fp32 instructions of sm_100 (one issue slot for two results).
+__device__ __forceinline__ uint64_t pack2(float a, float b) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+  return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& a, float& b) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v));
+}
+__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
+  uint64_t r;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+__device__ __forceinline__ uint64_t sub2(uint64_t a, uint64_t b) {
+  uint64_t r;
+  asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+
 // (re, im) -> packed fp16 pairs.  hi = the value rounded to an 11-bit significand with integer arithmetic on the fp32
 // word (exactly representable in fp16 unless it is below 2^-14, where the conversion rounds once more and the
 // remainder piece absorbs nothing: an absolute error below 2^-25), lo = the exact remainder rounded to fp16.
-__device__ __forceinline__ void split_half2(float re, float im, uint32_t& hi, uint32_t& lo) {
+__device__ __forceinline__ void split_half2(uint64_t x, uint32_t& hi, uint32_t& lo) {
+  float re, im, lr, li;
+  unpack2(x, re, im);
   const float hr = __uint_as_float((__float_as_uint(re) + 0x1000u) & 0xffffe000u);
   const float hi_ = __uint_as_float((__float_as_uint(im) + 0x1000u) & 0xffffe000u);
+  unpack2(sub2(x, pack2(hr, hi_)), lr, li);
   const __half2 h = __floats2half2_rn(hr, hi_);
-  const __half2 l = __floats2half2_rn(re - hr, im - hi_);
+  const __half2 l = __floats2half2_rn(lr, li);
   hi = *reinterpret_cast<const uint32_t*>(&h);
   lo = *reinterpret_cast<const uint32_t*>(&l);
 }
@@ -360,6 +383,7 @@ fft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_c
         const uint32_t mx = __reduce_max_sync(R == 32 ? 0xffffffffu : (0xffffu << (lane & 16)), __float_as_uint(mxf));
         const uint32_t f = max(mx >> 23, 14u);
         const float in_scale = __uint_as_float((267u - f) << 23);
+        const uint64_t scale2 = pack2(in_scale, in_scale);
         inv_scale = __uint_as_float((f - 13u) << 23);
         if (MODE == FFT_STRIDED) {
           // the stage-2 lanes of this thread belong to another (sub-)line: exchange through shared memory
@@ -374,7 +398,7 @@ fft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_c
         for (int l0 = 0; l0 < R; l0 += 16) {        // 16 complex = 16 packed columns per tensor-memory store
           uint32_t hw[16], lw[16];
 #pragma unroll
-          for (int j = 0; j < 16; ++j) split_half2(xr[l0 + j] * in_scale, xi[l0 + j] * in_scale, hw[j], lw[j]);
+          for (int j = 0; j < 16; ++j) split_half2(mul2(pack2(xr[l0 + j], xi[l0 + j]), scale2), hw[j], lw[j]);
           ptx::tmem_st_32x16(tm_a1 + l0, hw);
           ptx::tmem_st_32x16(tm_a1 + R + l0, lw);
         }
@@ -400,7 +424,7 @@ fft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_c
             const float2 tw = smem_tw[(c * 16 + j) * R + beta];
             const float br = __uint_as_float(v0[2 * j]);
             const float bi = __uint_as_float(v0[2 * j + 1]);
-            split_half2(br * tw.x - bi * tw.y, br * tw.y + bi * tw.x, ch[j], cl[j]);
+            split_half2(pack2(br * tw.x - bi * tw.y, br * tw.y + bi * tw.x), ch[j], cl[j]);
           }
           if (c == 0 && t >= 2) {
             // stage 2 of tile t - 2 (group g ^ 2) must be done reading this buffer
@@ -450,14 +474,17 @@ fft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_c
         if (!(om >= 1.1754944e-38f)) { om = om1; om_b = inv_scale; }
         F16_WAIT_WARP(&sh.d2_full[g], pk, 0x901);
         ptx::tc_fence_after();
+        uint32_t v0[K / 32][32];                      // all chunks in flight before the one wait
+#pragma unroll
+        for (int ch = 0; ch < K / 32; ++ch) ptx::tmem_ld_32x32(tm_a1 + ch * 32, v0[ch]);
+        ptx::tc_wait_ld();
+        const uint64_t om2 = pack2(om, om);
 #pragma unroll
         for (int ch = 0; ch < K / 32; ++ch) {
-          uint32_t v0[32];
-          ptx::tmem_ld_32x32(tm_a1 + ch * 32, v0);
-          ptx::tc_wait_ld();
           float f[32];
 #pragma unroll
-          for (int j = 0; j < 32; ++j) f[j] = __uint_as_float(v0[j]) * om;
+          for (int j = 0; j < 16; ++j)
+            unpack2(mul2(pack2(__uint_as_float(v0[ch][2 * j]), __uint_as_float(v0[ch][2 * j + 1])), om2), f[2 * j], f[2 * j + 1]);
           if (om_b != 1.0f) {
 #pragma unroll
             for (int j = 0; j < 32; ++j) f[j] *= om_b;

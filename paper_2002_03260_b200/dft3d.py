@@ -15,7 +15,7 @@ _LIB_PATH = os.environ.get("DFT3D_LIBRARY") or os.path.join(_HERE, "libdft3d.so"
 
 DFT3D_KDFT, DFT3D_FFT = 0, 1
 DFT3D_FORWARD, DFT3D_INVERSE = -1, +1
-DFT3D_NODES_ON_OUTPUT, DFT3D_UNSCALED_INVERSE, DFT3D_SPLIT_FP16, DFT3D_SPLIT_TF32 = 1, 2, 4, 8
+DFT3D_NODES_ON_OUTPUT, DFT3D_UNSCALED_INVERSE, DFT3D_SPLIT_FP16, DFT3D_SPLIT_TF32, DFT3D_DESTROY_INPUT = 1, 2, 4, 8, 16
 
 EXPORTS = [
     "dft3d_plan_create", "dft3d_plan_create_ex", "dft3d_execute", "dft3d_execute_host", "dft3d_execute_axis",

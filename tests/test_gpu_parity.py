@@ -628,3 +628,24 @@ def test_fft_fp16_scales_every_line_on_its_own(lib, oracle, axis):
     got = (ys / scale).cpu().numpy().astype(np.complex128)
     err = np.sqrt((np.abs(got - ref) ** 2).sum(axis=axis) / (np.abs(ref) ** 2).sum(axis=axis))
     assert err.max() < SANITY_AXIS, err.max()
+
+
+@pytest.mark.parametrize("mode_name,shape", [("kdft", (64, 128, 192)), ("fft", (256, 512, 256)), ("fft", (1024, 256, 256))])
+def test_destroy_input_uses_the_input_as_workspace(lib, oracle, mode_name, shape):
+    """DFT3D_DESTROY_INPUT: no workspace is allocated, the input cube is overwritten, the result is the same."""
+    mode = lib.DFT3D_KDFT if mode_name == "kdft" else lib.DFT3D_FFT
+    x = _inputs().cube(shape, "normal", 98, device="cuda")
+    keep = lib.Plan(*shape, mode=mode)
+    want = keep(x)
+    _finish(keep)
+    keep.destroy()
+    plan = lib.Plan(*shape, mode=mode, flags=lib.DFT3D_DESTROY_INPUT)
+    assert plan.workspace_bytes == 0
+    scratch = x.clone()
+    got = plan(scratch)
+    _finish(plan)
+    plan.destroy()
+    assert _rel_l2_gpu(got, want) < SANITY
+    if shape[0] <= 256:
+        assert oracle.rel_l2(got.cpu().numpy(), oracle.dft3d(x.cpu().numpy())) < SANITY
+    assert not torch.equal(scratch, x)      # the input really served as scratch
