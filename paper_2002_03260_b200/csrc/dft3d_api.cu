@@ -558,7 +558,7 @@ int fft_axis_pass(dft3d_plan_s* p, int axis, const float* in, float* out, cudaSt
       fp.blk_rows = int(p->n[1]);
       // TF32 kernel: the stage returns through shared memory and leaves as TMA stores; fp16 kernel: plain stores
       // from registers (a block is one contiguous region), which frees the raw stage right after the split
-      const char* env = getenv("DFT3D_FFT_STAGE_OUT");
+      const char* env = getenv("DFT3D_FFT_STAGE_OUT_BLOCKED");
       stage_out = env ? atoi(env) : (p->f16 ? 0 : 1);
     } else {
       if (rc == DFT3D_OK) rc = encode_f32(&map_out, out, 3, dims, strides, box, cols * 8);

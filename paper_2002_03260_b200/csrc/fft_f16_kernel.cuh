@@ -103,16 +103,13 @@ __device__ __forceinline__ uint64_t sub2(uint64_t a, uint64_t b) {
   return r;
 }
 
-// (re, im) -> packed fp16 pairs.  hi = the value rounded to an 11-bit significand with integer arithmetic on the fp32
-// word (exactly representable in fp16 unless it is below 2^-14, where the conversion rounds once more and the
-// remainder piece absorbs nothing: an absolute error below 2^-25), lo = the exact remainder rounded to fp16.
+// (re, im) -> packed fp16 pairs: hi = the value rounded to fp16, lo = the exact remainder x - hi rounded to fp16.
 __device__ __forceinline__ void split_half2(uint64_t x, uint32_t& hi, uint32_t& lo) {
   float re, im, lr, li;
   unpack2(x, re, im);
-  const float hr = __uint_as_float((__float_as_uint(re) + 0x1000u) & 0xffffe000u);
-  const float hi_ = __uint_as_float((__float_as_uint(im) + 0x1000u) & 0xffffe000u);
-  unpack2(sub2(x, pack2(hr, hi_)), lr, li);
-  const __half2 h = __floats2half2_rn(hr, hi_);
+  const __half2 h = __floats2half2_rn(re, im);
+  const float2 hf = __half22float2(h);
+  unpack2(sub2(x, pack2(hf.x, hf.y)), lr, li);
   const __half2 l = __floats2half2_rn(lr, li);
   hi = *reinterpret_cast<const uint32_t*>(&h);
   lo = *reinterpret_cast<const uint32_t*>(&l);
