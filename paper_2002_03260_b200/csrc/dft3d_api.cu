@@ -16,6 +16,7 @@
 #include "kdft_kernel.cuh"
 #include "kdft_f16_kernel.cuh"
 #include "fft_f16_kernel.cuh"
+#include "kdft_f16x2_kernel.cuh"
 #include "fft_kernel.cuh"
 
 namespace {
@@ -94,6 +95,8 @@ struct KdftAxis {
   long long n = 0;
   float* d_w = nullptr;   // [2 pieces][2n][2n] floats (TF32 pieces), or halves holding 1024*W (fp16 pieces)
   CUtensorMap map_w;
+  CUtensorMap map_w_pair; // fp16 pieces, paired CTAs: boxes of 128 table rows (half an N-tile)
+  bool pair = false;      // the paired-CTA kernel applies (fp16 pieces, 2n >= 256)
   int bn = 0;
   float out_mul = 1.0f;   // fp16 pieces: 2^-10, times 1/n for a scaled inverse
 };
@@ -151,6 +154,10 @@ int set_kernel_attributes(int device) {
                                   cudaFuncAttributeMaxDynamicSharedMemorySize, int(dft3d::kKdftF16SmemBytes)));
   DFT3D_CUDA(cudaFuncSetAttribute(dft3d::kdft_f16_axis_kernel<dft3d::KDFT_STRIDED>,
                                   cudaFuncAttributeMaxDynamicSharedMemorySize, int(dft3d::kKdftF16SmemBytes)));
+  DFT3D_CUDA(cudaFuncSetAttribute(dft3d::kdft_f16x2_axis_kernel<dft3d::KDFT_CONTIG>,
+                                  cudaFuncAttributeMaxDynamicSharedMemorySize, int(dft3d::kKdftX2SmemBytes)));
+  DFT3D_CUDA(cudaFuncSetAttribute(dft3d::kdft_f16x2_axis_kernel<dft3d::KDFT_STRIDED>,
+                                  cudaFuncAttributeMaxDynamicSharedMemorySize, int(dft3d::kKdftX2SmemBytes)));
 #define DFT3D_FFT_ATTR(MODE, R, RX, COLS, NB2, SO)                                                            \
   DFT3D_CUDA(cudaFuncSetAttribute(dft3d::fft_axis_kernel<MODE, R, RX, COLS, NB2, SO>,                          \
                                   cudaFuncAttributeMaxDynamicSharedMemorySize, int(dft3d::fft_smem_bytes(R, NB2))))
@@ -237,6 +244,16 @@ int build_kdft_axis(dft3d_plan_s* p, int a, const double* nodes) {
     const unsigned long long hdims[3] = {(unsigned long long)(2 * n), (unsigned long long)(2 * n), 2ull};
     const unsigned long long hstrides[2] = {(unsigned long long)(2 * n * 2), (unsigned long long)(4 * n * n * 2)};
     const unsigned hbox[3] = {unsigned(dft3d::kF16BlockK), unsigned(ax.bn), 2u};
+    {
+      // pairs of CTAs (cta_group::2) share a 256-column table tile, each loading 128 of its rows
+      const char* env = getenv("DFT3D_KDFT_PAIR");
+      ax.pair = ax.bn == 256 && (p->sm_count % 2 == 0) && (env ? atoi(env) != 0 : true);
+      if (ax.pair) {
+        const unsigned pbox[3] = {unsigned(dft3d::kF16BlockK), 128u, 2u};
+        int rc = encode_map(&ax.map_w_pair, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, ax.d_w, 3, hdims, hstrides, pbox, 128);
+        if (rc != DFT3D_OK) return rc;
+      }
+    }
     return encode_map(&ax.map_w, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, ax.d_w, 3, hdims, hstrides, hbox, 128);
   }
   dft3d::gen::axis_matrix(n, p->sign, scale, nodes, (p->flags & DFT3D_NODES_ON_OUTPUT) != 0, M.data());
@@ -291,7 +308,14 @@ int launch_kdft_strided(dft3d_plan_s* p, int a, const float* in, float* out, lon
   if (rc != DFT3D_OK) return rc;
   const long long total = kp.m_tiles * kp.n_tiles;
   const int grid = int(total < p->sm_count ? total : p->sm_count);
-  if (f16) {
+  if (f16 && ax.pair) {
+    dft3d::KdftF16Params fp;
+    fill_f16_params(fp, kp, ax, p, chain_pos);
+    const long long pairs = ((kp.m_tiles + 1) / 2) * kp.n_tiles;
+    const int pgrid = 2 * int(pairs < p->sm_count / 2 ? pairs : p->sm_count / 2);
+    dft3d::kdft_f16x2_axis_kernel<dft3d::KDFT_STRIDED>
+        <<<pgrid, dft3d::kKdftThreads, dft3d::kKdftX2SmemBytes, stream>>>(map_data, ax.map_w_pair, fp);
+  } else if (f16) {
     dft3d::KdftF16Params fp;
     fill_f16_params(fp, kp, ax, p, chain_pos);
     dft3d::kdft_f16_axis_kernel<dft3d::KDFT_STRIDED>
@@ -329,7 +353,14 @@ int launch_kdft_contig(dft3d_plan_s* p, int a, const float* in, float* out, long
   if (rc != DFT3D_OK) return rc;
   const long long total = kp.m_tiles * kp.n_tiles;
   const int grid = int(total < p->sm_count ? total : p->sm_count);
-  if (p->f16) {
+  if (p->f16 && ax.pair) {
+    dft3d::KdftF16Params fp;
+    fill_f16_params(fp, kp, ax, p, chain_pos);
+    const long long pairs = ((kp.m_tiles + 1) / 2) * kp.n_tiles;
+    const int pgrid = 2 * int(pairs < p->sm_count / 2 ? pairs : p->sm_count / 2);
+    dft3d::kdft_f16x2_axis_kernel<dft3d::KDFT_CONTIG>
+        <<<pgrid, dft3d::kKdftThreads, dft3d::kKdftX2SmemBytes, stream>>>(map_data, ax.map_w_pair, fp);
+  } else if (p->f16) {
     dft3d::KdftF16Params fp;
     fill_f16_params(fp, kp, ax, p, chain_pos);
     dft3d::kdft_f16_axis_kernel<dft3d::KDFT_CONTIG>
