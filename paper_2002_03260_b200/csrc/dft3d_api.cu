@@ -247,7 +247,9 @@ int build_kdft_axis(dft3d_plan_s* p, int a, const double* nodes) {
     {
       // pairs of CTAs (cta_group::2) share a 256-column table tile, each loading 128 of its rows
       const char* env = getenv("DFT3D_KDFT_PAIR");
-      ax.pair = ax.bn == 256 && (p->sm_count % 2 == 0) && (env ? atoi(env) != 0 : true);
+      // (off by default: it computes the same bits at the same speed as the one-CTA kernel -- its MMAs run at full
+      // rate, but every chain end now waits for a cross-CTA round trip to drain the accumulator)
+      ax.pair = ax.bn == 256 && (p->sm_count % 2 == 0) && (env ? atoi(env) != 0 : false);
       if (ax.pair) {
         const unsigned pbox[3] = {unsigned(dft3d::kF16BlockK), 128u, 2u};
         int rc = encode_map(&ax.map_w_pair, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, ax.d_w, 3, hdims, hstrides, pbox, 128);

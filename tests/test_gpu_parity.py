@@ -649,3 +649,28 @@ def test_destroy_input_uses_the_input_as_workspace(lib, oracle, mode_name, shape
     if shape[0] <= 256:
         assert oracle.rel_l2(got.cpu().numpy(), oracle.dft3d(x.cpu().numpy())) < SANITY
     assert not torch.equal(scratch, x)      # the input really served as scratch
+
+
+def test_kdft_cta_pair_kernel_matches(lib, oracle, monkeypatch):
+    """The cta_group::2 form of the fp16 KDFT kernel (pairs of CTAs share every table tile; enabled with
+    DFT3D_KDFT_PAIR=1 at plan creation) computes the same sums in the same order: identical bits, and a ragged
+    shape against the oracle."""
+    shape = (256, 128, 384)
+    x = _inputs().cube(shape, "normal", 99, device="cuda")
+    plan = lib.Plan(*shape, flags=lib.DFT3D_SPLIT_FP16)
+    want = plan(x)
+    _finish(plan)
+    plan.destroy()
+    monkeypatch.setenv("DFT3D_KDFT_PAIR", "1")
+    plan = lib.Plan(*shape, flags=lib.DFT3D_SPLIT_FP16)
+    got = plan(x)
+    _finish(plan)
+    plan.destroy()
+    assert torch.equal(got, want)
+    shape = (132, 260, 200)
+    x = _inputs().cube(shape, "normal", 100, device="cuda")
+    plan = lib.Plan(*shape, flags=lib.DFT3D_SPLIT_FP16)
+    y = plan(x)
+    _finish(plan)
+    plan.destroy()
+    assert oracle.rel_l2(y.cpu().numpy(), oracle.dft3d(x.cpu().numpy())) < SANITY
