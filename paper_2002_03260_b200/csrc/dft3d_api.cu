@@ -180,7 +180,7 @@ int set_kernel_attributes(int device) {
 #undef DFT3D_FFT_ATTR
 #define DFT3D_FFT16_ATTR(MODE, R, RX, COLS, SO)                                                   \
   DFT3D_CUDA(cudaFuncSetAttribute(dft3d::fft_f16_axis_kernel<MODE, R, RX, COLS, SO>,              \
-                                  cudaFuncAttributeMaxDynamicSharedMemorySize, int(dft3d::fft16_smem_bytes(R))))
+                                  cudaFuncAttributeMaxDynamicSharedMemorySize, int(dft3d::fft16_smem_bytes(R, RX))))
   DFT3D_FFT16_ATTR(dft3d::FFT_CONTIG, 32, 1, 16, 0);
   DFT3D_FFT16_ATTR(dft3d::FFT_CONTIG, 16, 1, 16, 0);
   DFT3D_FFT16_ATTR(dft3d::FFT_CONTIG, 32, 2, 16, 0);
@@ -615,7 +615,7 @@ int fft_axis_pass(dft3d_plan_s* p, int axis, const float* in, float* out, cudaSt
     if (fp.mtiles_per_stage != 1 && fp.mtiles_per_stage != 2 && fp.mtiles_per_stage != 4)
       return fail(DFT3D_ERR_UNSUPPORTED, "internal: %d tiles per stage", fp.mtiles_per_stage);
     const int grid = int(fp.num_stages < p->sm_count ? fp.num_stages : p->sm_count);
-    const size_t smem = dft3d::fft16_smem_bytes(R);
+    const size_t smem = dft3d::fft16_smem_bytes(R, RX);
 #define DFT3D_FFT16_LAUNCH(MODE, R_, RX_, COLS_, SO_)                                         \
   dft3d::fft_f16_axis_kernel<MODE, R_, RX_, COLS_, SO_>                                        \
       <<<grid, dft3d::kFftThreads, smem, stream>>>(map_data, ax.map_w, map_out, hp)

@@ -29,7 +29,7 @@
 // Tensor memory, per group g at column 128*g: D1 at +0 (2R columns), A1 at +64 (hi R columns, lo R columns, two
 // K-adjacent fp16 values per column); D2 reuses A1's columns (stage 1 has consumed them by then).
 // Shared memory: [W: 2 pieces x 2R rows x 128 B] [A2: 2 buffers x (hi, lo) x 128 rows x 128 B, used in tile order]
-// [twiddles R x R complex64] [raw ring 128 KB] [barriers].
+// [twiddles R x R complex64 (and those of the radix-2 step)] [raw ring 128 KB] [barriers].
 // A mbarrier wait tells phases apart by parity only, so nobody may wait on a barrier two phases ahead: every barrier
 // here is waited on in consecutive phases by construction (per-group barriers by that group and the issuers in tile
 // order; a2_empty[h] by group h^2 for every tile of group h; raw_full[s] needs (4 / tiles per stage) to divide the
@@ -58,8 +58,8 @@ __host__ __device__ constexpr int fft16_w_bytes(int R) { return 2 * 2 * R * 128;
 __host__ __device__ constexpr int fft16_tw_bytes(int R) { return R * R * 8; }
 constexpr int kFft16A2Piece = 128 * 128;
 constexpr int kFft16RawBytes = 128 * 1024;
-__host__ __device__ constexpr size_t fft16_smem_bytes(int R) {
-  return size_t(fft16_w_bytes(R)) + 4 * size_t(kFft16A2Piece) + fft16_tw_bytes(R) + kFft16RawBytes + 1024 + 1024;
+__host__ __device__ constexpr size_t fft16_smem_bytes(int R, int RX) {   // RX == 2: a second twiddle table (radix-2 step)
+  return size_t(fft16_w_bytes(R)) + 4 * size_t(kFft16A2Piece) + size_t(RX) * fft16_tw_bytes(R) + kFft16RawBytes + 1024 + 1024;
 }
 
 #define F16_WAIT(bar, parity, code)                                 \
@@ -130,7 +130,8 @@ fft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_c
   uint8_t* smem_w = smem;
   uint8_t* smem_a2 = smem_w + fft16_w_bytes(R);            // buffer i = [hi piece][lo piece] at i * 2 * a2_piece
   float2* smem_tw = reinterpret_cast<float2*>(smem_a2 + 4 * a2_piece);
-  uint8_t* smem_rawring = reinterpret_cast<uint8_t*>(smem_tw) + fft16_tw_bytes(R);
+  float2* smem_tw2 = smem_tw + R * R;                      // RX == 2 only: exp(s*2*pi*i*m/N), m < R*R
+  uint8_t* smem_rawring = reinterpret_cast<uint8_t*>(smem_tw) + RX * fft16_tw_bytes(R);
   FftF16Shared& sh = *reinterpret_cast<FftF16Shared*>(smem_rawring + kFft16RawBytes);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 #ifdef DFT3D_PROFILE_WAITS
@@ -160,6 +161,8 @@ fft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_c
     ptx::fence_mbar_init();
   }
   for (int i = tid; i < R * R; i += kFftThreads) smem_tw[i] = __ldg(p.twiddle + i);
+  if (RX == 2)
+    for (int i = tid; i < R * R; i += kFftThreads) smem_tw2[i] = __ldg(p.twiddle2 + i);
   if (warp == 1) {
     ptx::tmem_alloc(&sh.tmem_base, 512);
     ptx::tmem_relinquish();
@@ -298,10 +301,17 @@ fft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_c
     const int m = q * 32 + lane;
     // stage-1 lane = (sub-line sl1, beta), beta fastest; stage-2 lane = (sub-line sl2, k1)
     const int sl1 = m / R, beta = m % R;
-    const int g1 = sl1 / RX, bsel1 = sl1 % RX;  // line of the cube within the M-tile; which butterfly output
+    // Which line of the stage and which butterfly output a sub-line is.  CONTIG: the RX sub-lines of a line sit in one
+    // M-tile.  STRIDED with RX == 2: an M-tile holds the SAME butterfly output of SL neighbouring lines (tiles 2u and
+    // 2u+1 are the a and b halves of lines u*SL ...), so that a stage-2 store still covers SL neighbouring columns of
+    // one output row (32 bytes) instead of SL/2.
+    constexpr bool kPairTiles = (MODE == FFT_STRIDED) && (RX == 2);
+    const int g1 = kPairTiles ? sl1 : sl1 / RX;         // line within the tile (kPairTiles: within the pair of tiles)
+    const int bsel1_fixed = sl1 % RX;
     const int sl2 = (MODE == FFT_CONTIG) ? m / R : m % SL;
     const int k1 = (MODE == FFT_CONTIG) ? m % R : m / SL;
-    const int g2 = sl2 / RX, bsel2 = sl2 % RX;
+    const int g2 = kPairTiles ? sl2 : sl2 / RX;
+    const int bsel2_fixed = sl2 % RX;
     const uint32_t tm_d1 = tmem + (uint32_t(q * 32) << 16) + g * 128;
     const uint32_t tm_a1 = tm_d1 + 64;          // A1 (hi | lo), later D2
     // A2 row of (sl, k1): CONTIG sl*R + k1 ; STRIDED k1*SL + sl (so that stage-2 stores of one k2 touch neighbouring lines).
@@ -329,6 +339,8 @@ fft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_c
       const uint32_t s = uint32_t(istage % p.raw_stages), phs = uint32_t(istage / p.raw_stages) & 1;
       const uint32_t pk = uint32_t(t >> 2) & 1;
       uint8_t* stage = smem_rawring + size_t(s) * p.stage_bytes;
+      const int bsel1 = kPairTiles ? (mt & 1) : bsel1_fixed, bsel2 = kPairTiles ? (mt & 1) : bsel2_fixed;
+      const int col0 = kPairTiles ? (mt >> 1) * SL : mt * Lg;     // first column of the stage this tile's lines occupy
 
       // ---- split: this lane's R elements (after the butterfly when RX == 2) -> scaled fp16 pieces -> A1
       F16_WAIT_WARP(&sh.raw_full[s], phs, 0x701);
@@ -340,7 +352,7 @@ fft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_c
           stride = uint32_t(R) * 8u;
           half = uint32_t(NL) * 8u;
         } else {
-          const int c = mt * Lg + g1;               // column within the stage
+          const int c = col0 + g1;                  // column within the stage
           const uint32_t swz = (COLS == 16) ? uint32_t(beta & 7) : uint32_t((beta >> 1) & 3);   // TMA swizzle of the row
           base = uint32_t(beta) * kRowBytes + ((uint32_t(c >> 1) ^ swz) << 4) + uint32_t(c & 1) * 8u;
           stride = uint32_t(R) * kRowBytes;
@@ -360,7 +372,7 @@ fft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_c
             if (bsel1 == 0) {
               xr[l] = ur + vr; xi[l] = ui + vi;
             } else {
-              const float2 tw = __ldg(p.twiddle2 + l * R + beta);
+              const float2 tw = smem_tw2[l * R + beta];
               const float dr = ur - vr, di = ui - vi;
               xr[l] = dr * tw.x - di * tw.y; xi[l] = dr * tw.y + di * tw.x;
             }
@@ -453,13 +465,13 @@ fft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_c
           k2_stride = RX * R;
         } else {
           const long long ct = sidx % p.c_tiles, bt = sidx / p.c_tiles;
-          const long long col = ct * COLS + mt * Lg + g2;
+          const long long col = ct * COLS + col0 + g2;
           ok = col < p.C;
           if (p.out_blocked) {
             // block [k][COLS] number n2tile*blk_rows + i1 of the blocked intermediate: pieces of one block are close
             // together, so plain stores from registers do (the L2 merges them into full lines)
             const long long blk = (ct % p.blk_tiles) * p.blk_rows + ct / p.blk_tiles;
-            dst = reinterpret_cast<float2*>(p.out) + (blk * p.N + (RX * k1 + bsel2)) * COLS + (mt * Lg + g2);
+            dst = reinterpret_cast<float2*>(p.out) + (blk * p.N + (RX * k1 + bsel2)) * COLS + (col0 + g2);
             k2_stride = (long long)(RX * R) * COLS;
           } else {
             dst = reinterpret_cast<float2*>(p.out) + (bt * p.N + (RX * k1 + bsel2)) * p.C + col;
@@ -488,7 +500,7 @@ fft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_c
           }
           if (STAGE_OUT) {
             // element (row k, column c) of the stage, in the layout TMA wrote the input in (same swizzle)
-            const int c = mt * Lg + g2;
+            const int c = col0 + g2;
 #pragma unroll
             for (int j = 0; j < 16; ++j) {
               const int k = RX * (k1 + R * (ch * 16 + j)) + bsel2;
