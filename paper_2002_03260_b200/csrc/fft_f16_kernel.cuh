@@ -51,7 +51,8 @@ struct FftF16Shared {
   uint64_t w_full;
   uint32_t tmem_base;
   volatile int abort_flag;
-  float line_scale[4][8];      // STRIDED: per group, 2^(e - 13) of the tile's (sub-)lines, from the split to the store
+  float line_scale[4][8];      // per group, 2^(e - 13) of the tile's (sub-)lines, from the split to the store (where a
+                               // thread's stage-2 lane belongs to another sub-line than its stage-1 lane)
 };
 
 __host__ __device__ constexpr int fft16_w_bytes(int R) { return 2 * 2 * R * 128; }
@@ -308,20 +309,22 @@ fft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_c
     constexpr bool kPairTiles = (MODE == FFT_STRIDED) && (RX == 2);
     const int g1 = kPairTiles ? sl1 : sl1 / RX;         // line within the tile (kPairTiles: within the pair of tiles)
     const int bsel1_fixed = sl1 % RX;
-    const int sl2 = (MODE == FFT_CONTIG) ? m / R : m % SL;
-    const int k1 = (MODE == FFT_CONTIG) ? m % R : m / SL;
+    // stage-2 lanes.  CONTIG: (line, k1, butterfly output), output fastest, so that the lanes of a warp store
+    // consecutive outputs X[RX*k1 + b] of one line; STRIDED: (k1, sub-line), sub-line fastest (neighbouring columns).
+    const int sl2 = (MODE == FFT_CONTIG) ? (m / (RX * R)) * RX + (m % RX) : m % SL;
+    const int k1 = (MODE == FFT_CONTIG) ? (m % (RX * R)) / RX : m / SL;
     const int g2 = kPairTiles ? sl2 : sl2 / RX;
     const int bsel2_fixed = sl2 % RX;
     const uint32_t tm_d1 = tmem + (uint32_t(q * 32) << 16) + g * 128;
     const uint32_t tm_a1 = tm_d1 + 64;          // A1 (hi | lo), later D2
-    // A2 row of (sl, k1): CONTIG sl*R + k1 ; STRIDED k1*SL + sl (so that stage-2 stores of one k2 touch neighbouring lines).
+    // A2 row (= stage-2 lane) of (sub-line, k1): CONTIG line*RX*R + RX*k1 + b ; STRIDED k1*SL + sl.
     // K position (beta, re/im) = halves 2*beta, 2*beta+1 of the row: 16-byte chunk beta/4 (XORed with row % 8 by the
     // 128-byte swizzle), word beta%4.  row % 8 takes kSwzPer different values as k1 runs: offsets for each of them.
-    constexpr int row_mul_k1 = (MODE == FFT_CONTIG) ? 1 : SL;
-    constexpr int kSwzPer = (MODE == FFT_CONTIG) ? 8 : (SL >= 8 ? 1 : 8 / SL);
+    constexpr int row_mul_k1 = (MODE == FFT_CONTIG) ? RX : SL;
+    constexpr int kSwzPer = (row_mul_k1 >= 8) ? 1 : 8 / row_mul_k1;
     uint32_t a2_off[kSwzPer];                   // byte offset of (row of k1 = v, this beta) minus v * row_mul_k1 * 128
     {
-      const int row_base = (MODE == FFT_CONTIG) ? sl1 * R : sl1;
+      const int row_base = (MODE == FFT_CONTIG) ? (sl1 / RX) * RX * R + (sl1 % RX) : sl1;
       const uint32_t a2_chunk = uint32_t(beta) >> 2;
       const uint32_t a2_word = uint32_t(beta & 3) * 4u;
 #pragma unroll
@@ -394,7 +397,7 @@ fft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_c
         const float in_scale = __uint_as_float((267u - f) << 23);
         const uint64_t scale2 = pack2(in_scale, in_scale);
         inv_scale = __uint_as_float((f - 13u) << 23);
-        if (MODE == FFT_STRIDED) {
+        if (MODE == FFT_STRIDED || RX == 2) {
           // the stage-2 lanes of this thread belong to another (sub-)line: exchange through shared memory
           // (a bounded mbarrier rather than a named barrier: a warp that gave up a wait must not strand the others)
           if (beta == 0) sh.line_scale[g][sl1] = inv_scale;

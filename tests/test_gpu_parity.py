@@ -608,11 +608,11 @@ def test_splits_agree_512(lib, oracle):
 
 
 @pytest.mark.parametrize("axis", [1, 2])
-def test_fft_fp16_scales_every_line_on_its_own(lib, oracle, axis):
+@pytest.mark.parametrize("shape", [(64, 256, 256), (64, 512, 512)])     # 256 = 16*16; 512 = 2*16*16 (radix-2 step first)
+def test_fft_fp16_scales_every_line_on_its_own(lib, oracle, axis, shape):
     """The fp16 split of the FFT kernel scales each line by a power of two taken from that line's largest element.
     Lines that differ by up to 2^120 in magnitude must each come out with fp32-level error relative to their OWN norm
     (a single scale for the whole array would flush the small lines to zero)."""
-    shape = (64, 256, 256)
     x = _inputs().cube(shape, "normal", 96, device="cuda")
     g = torch.Generator(device="cuda").manual_seed(97)
     other = [d for d in range(3) if d != axis]
