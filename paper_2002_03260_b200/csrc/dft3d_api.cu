@@ -247,9 +247,11 @@ int build_kdft_axis(dft3d_plan_s* p, int a, const double* nodes) {
     {
       // pairs of CTAs (cta_group::2) share a 256-column table tile, each loading 128 of its rows
       const char* env = getenv("DFT3D_KDFT_PAIR");
-      // (off by default: it computes the same bits at the same speed as the one-CTA kernel -- its MMAs run at full
-      // rate, but every chain end now waits for a cross-CTA round trip to drain the accumulator)
-      ax.pair = ax.bn == 256 && (p->sm_count % 2 == 0) && (env ? atoi(env) != 0 : false);
+      // Same bits as the one-CTA kernel.  Its MMAs run at full rate but every chain end waits for a cross-CTA round
+      // trip, which cancels out at n = 1024 (77.6 vs 78.5 ms); at n = 2048, where the 64 MiB table no longer sits in
+      // L2 beside the data and the part runs at its 1 kW cap, fetching every table tile once per CTA pair wins
+      // (1365 -> 1235 ms, 1305 -> 1522 MHz).  Default: pairs from n = 2048 on.
+      ax.pair = ax.bn == 256 && (p->sm_count % 2 == 0) && (env ? atoi(env) != 0 : n >= 2048);
       if (ax.pair) {
         const unsigned pbox[3] = {unsigned(dft3d::kF16BlockK), 128u, 2u};
         int rc = encode_map(&ax.map_w_pair, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, ax.d_w, 3, hdims, hstrides, pbox, 128);
