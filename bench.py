@@ -40,6 +40,8 @@ def parse_args():
     ap.add_argument("--no-kdft", action="store_true", help="FFT mode only: skip the KDFT timing of the same cube")
     ap.add_argument("--split", choices=["default", "fp16", "tf32"], default="default",
                     help="operand split of the tensor-core products (default: the library's choice per formulation)")
+    ap.add_argument("--axes", type=str, default=None,
+                    help="transform only these axes, e.g. 1,2 with --shape 1,8192,8192 for the paper's 2D workload")
     ap.add_argument("--destroy-input", action="store_true",
                     help="plans use the input cube as their workspace (DFT3D_DESTROY_INPUT): for sizes where input + "
                          "output leave no room for one, e.g. 2048^3; the input is not regenerated between steps")
@@ -205,8 +207,9 @@ def main():
         flags = {"default": 0, "fp16": dft.DFT3D_SPLIT_FP16, "tf32": dft.DFT3D_SPLIT_TF32}[args.split]
         if args.destroy_input:
             flags |= dft.DFT3D_DESTROY_INPUT
+        axes = tuple(int(v) for v in args.axes.split(",")) if args.axes else None
         plan_ = dft.Plan(*shape, mode=dft.DFT3D_KDFT if mode_name == "kdft" else dft.DFT3D_FFT, sign=dft.DFT3D_FORWARD,
-                         flags=flags)
+                         flags=flags, axes=axes)
         for _ in range(warmup):
             plan_.execute(x, y)
         barrier()
@@ -258,7 +261,8 @@ def main():
     if rank == 0:
         peaks, peak_kind = measured_peaks()
         P = float(shape[0]) * shape[1] * shape[2]
-        nsum = float(sum(shape))
+        taxes = tuple(int(v) for v in args.axes.split(",")) if args.axes else (0, 1, 2)
+        nsum = float(sum(shape[a] for a in taxes))   # lengths of the transformed axes
 
         def kdft_roofline(ms, nlaunch, split):
             # dominant kernel: the KDFT axis kernel (the fp16 split adds one small reduction over the input).
@@ -286,7 +290,7 @@ def main():
             roofline = kdft_roofline(ms_step, launches, plan.split)
         else:
             # only kernel: fft_axis_kernel, one launch per axis; algorithmic traffic 16 B per point per axis
-            algo_bytes = 3 * 16.0 * P
+            algo_bytes = len(taxes) * 16.0 * P
             achieved = algo_bytes / (ms_step * 1e-3) * 1e-9
             fkernel = "fft_f16_axis_kernel" if plan.split == dft.DFT3D_SPLIT_FP16 else "fft_axis_kernel"
             roofline = {"bound": "hbm", "kernel": fkernel, "achieved": achieved, "peak": peaks["hbm_gbs"],
@@ -309,7 +313,7 @@ def main():
                 "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": "fp16x3" if plan.split == dft.DFT3D_SPLIT_FP16 else "tf32x3", "data": "synthetic",
                 "config": {"workload": "%s forward 3D complex64 DFT %s, re/im iid U(-1,1), seed 1003+rank" % (mode.upper(), wl),
-                           "mode": mode, "shape": list(shape),
+                           "mode": mode, "shape": list(shape), "axes": list(taxes),
                            "l2": "input and output (%.2f GiB each) are larger than L2" % (P * 8 / 2**30),
                            "per_rank": "one independent cube per GPU",
                            "destroy_input": bool(args.destroy_input)},
