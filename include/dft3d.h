@@ -57,9 +57,16 @@ enum {
                                    DFT3D_ERR_UNSUPPORTED for KDFT when a transformed n_a is not a multiple of 4 */
   DFT3D_SPLIT_TF32 = 8u,        /* insist on TF32 pieces (no scaling; every element keeps ~22 significant bits
                                    whatever the dynamic range of the input) */
-  DFT3D_DESTROY_INPUT = 16u     /* dft3d_execute may overwrite `in`: a plan over all three axes then uses the input
+  DFT3D_DESTROY_INPUT = 16u,    /* dft3d_execute may overwrite `in`: a plan over all three axes then uses the input
                                    cube as its workspace and allocates none, which keeps the fast schedules available
                                    when input + output fill the memory (2048^3).  Ignored by plans over fewer axes. */
+  DFT3D_INVERSE_SOLVE = 32u     /* KDFT, sign = +1, axes with nodes: the true inverse of the nonuniform transform
+                                   (Section III-A: for points that are not roots of unity the inverse "amounts to
+                                   solving the linear system").  The n_a x n_a forward matrix of the nodes is inverted
+                                   once at plan creation (float64, on the host; n_a <= 2048) and the solve becomes
+                                   one more matrix product, so inverse(forward(x)) = x for distinct nodes.  Axes
+                                   without nodes use the usual scaled inverse, which is that inverse.  Singular or
+                                   hopelessly ill-conditioned node sets are refused. */
 };
 
 typedef struct dft3d_options_s {
@@ -85,7 +92,7 @@ typedef struct dft3d_options_s {
  *            as solving Eq. 2; on a uniform grid that solve is this product).
  *   nodesA   HOST pointer to n_a doubles, or NULL for the uniform grid t_j = j/n_a.
  *            Any finite value is accepted and used modulo 1.  Copied during the call.
- *            With nodes and sign=+1 the result is the conjugate-kernel product, not an
+ *            With nodes and sign=+1 the result is the conjugate-kernel product (see DFT3D_INVERSE_SOLVE), not an
  *            inverse of the nonuniform transform.  FFT mode takes no nodes.
  *
  * The DFT / Vandermonde matrices and twiddles are evaluated in float64 with exactly
@@ -168,6 +175,9 @@ const char* dft3d_last_error(void);
 int dft3d_generate_axis_matrix(long long n, int sign, double scale, const double* nodes, int nodes_on_output,
                                double* matrix);
 int dft3d_generate_twiddle(long long N1, long long N2, int sign, double* twiddle);
+/* dft3d_generate_inverse_matrix: the inverse of the forward matrix of `nodes` (what DFT3D_INVERSE_SOLVE multiplies
+ *   by), n*n complex doubles; *growth (may be NULL) receives max|M| * max|M^-1|. */
+int dft3d_generate_inverse_matrix(long long n, const double* nodes, int nodes_on_output, double* matrix, double* growth);
 int dft3d_generate_real_table(long long n, int sign, double scale, const double* nodes, int nodes_on_output,
                               float* hi, float* lo);
 

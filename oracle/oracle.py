@@ -122,6 +122,33 @@ def dft3d(x, sign=-1, scaled_inverse=False, nodes=None, nodes_on_output=False):
     return out
 
 
+def solve_axis(X, axis, nodes, nodes_on_output=False):
+    """Inverse nonuniform transform of one axis (Section III-A, below Eq. 3: for sample points that are not the roots
+    of unity the inverse "amounts to solving the linear system"): x with V x = X along `axis`, V the forward matrix
+    of Eq. 3 for these nodes.  numpy.linalg.solve (LAPACK, float64) is the library step."""
+    X = np.ascontiguousarray(X, dtype=np.complex128)
+    assert X.ndim == 3
+    n = X.shape[axis]
+    V = axis_matrix(n, -1, 1.0, nodes, nodes_on_output)
+    moved = np.moveaxis(X, axis, 0).reshape(n, -1)
+    sol = np.linalg.solve(V, moved)
+    shape = (n,) + tuple(np.delete(np.array(X.shape), axis))
+    return np.ascontiguousarray(np.moveaxis(sol.reshape(shape), 0, axis))
+
+
+def solve3d(X, nodes, nodes_on_output=False):
+    """Inverse of dft3d(., sign=-1, nodes=nodes): axes with nodes are solved, axes without use the scaled inverse
+    kernel (which is the inverse of the uniform matrix)."""
+    X = np.ascontiguousarray(X, dtype=np.complex128)
+    for a in range(3):
+        nd = None if nodes is None else nodes[a]
+        if nd is None:
+            X = dft_axis(X, a, sign=+1, scale=1.0 / X.shape[a])
+        else:
+            X = solve_axis(X, a, nd, nodes_on_output)
+    return X
+
+
 def coeff_triple(x, k, sign=-1, scaled_inverse=False, nodes=None, nodes_on_output=False):
     """One output coefficient X[k0,k1,k2] by the literal triple sum (complex64 input)."""
     x = np.ascontiguousarray(x, dtype=np.complex64)

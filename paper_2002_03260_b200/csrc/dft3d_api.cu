@@ -215,9 +215,28 @@ int build_kdft_axis(dft3d_plan_s* p, int a, const double* nodes) {
   } catch (const std::bad_alloc&) {
     return fail(DFT3D_ERR_ALLOC, "host allocation of the axis-%d table failed", a);
   }
+  // DFT3D_INVERSE_SOLVE on an axis with nodes: the table is the inverse of the forward matrix of those nodes
+  const bool solve = (p->flags & DFT3D_INVERSE_SOLVE) && nodes;
+  if (solve) {
+    dft3d::gen::axis_matrix(n, DFT3D_FORWARD, 1.0, nodes, (p->flags & DFT3D_NODES_ON_OUTPUT) != 0, M.data());
+    double growth = 0.0;
+    if (!dft3d::gen::invert_matrix(n, M.data(), &growth))
+      return fail(DFT3D_ERR_INVALID_ARG, "axis %d: the matrix of these nodes is singular (nodes must be distinct modulo 1)", a);
+    if (growth > 1e6)
+      return fail(DFT3D_ERR_UNSUPPORTED, "axis %d: the nodes make the system too ill-conditioned for fp32 data "
+                  "(|V| |V^-1| = %.3g)", a, growth);
+  }
   if (p->f16) {
-    // fp16 pieces of 1024*W; the 1/n of a scaled inverse goes into the epilogue multiplier instead of the table
-    dft3d::gen::axis_matrix(n, p->sign, 1.0, nodes, (p->flags & DFT3D_NODES_ON_OUTPUT) != 0, M.data());
+    // fp16 pieces of 2^s*W (s = 10 for entries of modulus one); the 1/n of a scaled inverse goes into the epilogue
+    // multiplier instead of the table
+    if (!solve) dft3d::gen::axis_matrix(n, p->sign, 1.0, nodes, (p->flags & DFT3D_NODES_ON_OUTPUT) != 0, M.data());
+    int s2 = 10;
+    if (solve) {
+      double mx = 0.0;
+      for (size_t i = 0; i < M.size(); ++i) mx = std::fmax(mx, std::fabs(M[i]));
+      s2 = 9 - std::ilogb(mx);           // largest table entry in [512, 1024)
+    }
+    const double tscale = std::ldexp(1.0, s2);
     std::vector<__half> H;
     try {
       H.resize(size_t(2) * 4 * n * n);
@@ -227,7 +246,7 @@ int build_kdft_axis(dft3d_plan_s* p, int a, const double* nodes) {
     const size_t piece = size_t(4) * n * n, ld = size_t(2) * n;
     for (long long k = 0; k < n; ++k)
       for (long long j = 0; j < n; ++j) {
-        const double re = 1024.0 * M[2 * (k * n + j)], im = 1024.0 * M[2 * (k * n + j) + 1];
+        const double re = tscale * M[2 * (k * n + j)], im = tscale * M[2 * (k * n + j) + 1];
         const double vals[4] = {re, -im, im, re};                  // W[2k][2j], W[2k][2j+1], W[2k+1][2j], W[2k+1][2j+1]
         const size_t idx[4] = {(2 * k) * ld + 2 * j, (2 * k) * ld + 2 * j + 1, (2 * k + 1) * ld + 2 * j,
                                (2 * k + 1) * ld + 2 * j + 1};
@@ -238,7 +257,7 @@ int build_kdft_axis(dft3d_plan_s* p, int a, const double* nodes) {
           H[piece + idx[q]] = __float2half_rn(float(lo));
         }
       }
-    ax.out_mul = float(scale / 1024.0);
+    ax.out_mul = float((solve ? 1.0 : scale) / tscale);
     DFT3D_CUDA(cudaMalloc(&ax.d_w, H.size() * sizeof(__half)));
     DFT3D_CUDA(cudaMemcpy(ax.d_w, H.data(), H.size() * sizeof(__half), cudaMemcpyHostToDevice));
     const unsigned long long hdims[3] = {(unsigned long long)(2 * n), (unsigned long long)(2 * n), 2ull};
@@ -260,7 +279,7 @@ int build_kdft_axis(dft3d_plan_s* p, int a, const double* nodes) {
     }
     return encode_map(&ax.map_w, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, ax.d_w, 3, hdims, hstrides, hbox, 128);
   }
-  dft3d::gen::axis_matrix(n, p->sign, scale, nodes, (p->flags & DFT3D_NODES_ON_OUTPUT) != 0, M.data());
+  if (!solve) dft3d::gen::axis_matrix(n, p->sign, scale, nodes, (p->flags & DFT3D_NODES_ON_OUTPUT) != 0, M.data());
   dft3d::gen::real_table_from_matrix(n, M.data(), W.data(), W.data() + size_t(4) * n * n);
   DFT3D_CUDA(cudaMalloc(&ax.d_w, W.size() * sizeof(float)));
   DFT3D_CUDA(cudaMemcpy(ax.d_w, W.data(), W.size() * sizeof(float), cudaMemcpyHostToDevice));
@@ -734,6 +753,16 @@ int dft3d_generate_axis_matrix(long long n, int sign, double scale, const double
   return DFT3D_OK;
 }
 
+int dft3d_generate_inverse_matrix(long long n, const double* nodes, int nodes_on_output, double* matrix, double* growth) {
+  if (n < 1 || !matrix || !nodes) return fail(DFT3D_ERR_INVALID_ARG, "bad argument");
+  for (long long i = 0; i < n; ++i)
+    if (!std::isfinite(nodes[i])) return fail(DFT3D_ERR_INVALID_ARG, "node %lld is not finite", i);
+  dft3d::gen::axis_matrix(n, DFT3D_FORWARD, 1.0, nodes, nodes_on_output != 0, matrix);
+  if (!dft3d::gen::invert_matrix(n, matrix, growth))
+    return fail(DFT3D_ERR_INVALID_ARG, "the matrix of these nodes is singular (nodes must be distinct modulo 1)");
+  return DFT3D_OK;
+}
+
 int dft3d_generate_twiddle(long long N1, long long N2, int sign, double* twiddle) {
   if (N1 < 1 || N2 < 1 || !twiddle || (sign != -1 && sign != 1)) return fail(DFT3D_ERR_INVALID_ARG, "bad argument");
   dft3d::gen::twiddle(N1, N2, sign, twiddle);
@@ -776,8 +805,16 @@ int dft3d_plan_create_ex(dft3d_plan_t* out, long long n0, long long n1, long lon
       return fail(DFT3D_ERR_INVALID_ARG, "options->struct_size is not a known size");
     memcpy(&opt, options, options->struct_size);
   }
-  if (opt.flags & ~(DFT3D_NODES_ON_OUTPUT | DFT3D_UNSCALED_INVERSE | DFT3D_SPLIT_FP16 | DFT3D_SPLIT_TF32 | DFT3D_DESTROY_INPUT))
+  if (opt.flags & ~(DFT3D_NODES_ON_OUTPUT | DFT3D_UNSCALED_INVERSE | DFT3D_SPLIT_FP16 | DFT3D_SPLIT_TF32 | DFT3D_DESTROY_INPUT |
+                    DFT3D_INVERSE_SOLVE))
     return fail(DFT3D_ERR_INVALID_ARG, "unknown flag");
+  if (opt.flags & DFT3D_INVERSE_SOLVE) {
+    if (mode != DFT3D_KDFT || sign != DFT3D_INVERSE || (opt.flags & DFT3D_UNSCALED_INVERSE))
+      return fail(DFT3D_ERR_INVALID_ARG, "DFT3D_INVERSE_SOLVE needs mode KDFT, sign +1 and the scaled inverse");
+    for (int a = 0; a < 3; ++a)
+      if (nodes[a] && nn[a] > 2048)
+        return fail(DFT3D_ERR_UNSUPPORTED, "DFT3D_INVERSE_SOLVE inverts the n x n matrix on the host: n%d = %lld exceeds 2048", a, nn[a]);
+  }
   if ((opt.flags & DFT3D_SPLIT_FP16) && (opt.flags & DFT3D_SPLIT_TF32))
     return fail(DFT3D_ERR_INVALID_ARG, "DFT3D_SPLIT_FP16 and DFT3D_SPLIT_TF32 exclude each other");
   // default: fp16 pieces (KDFT: where the sizes allow it, see below)

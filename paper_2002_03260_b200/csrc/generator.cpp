@@ -1,6 +1,10 @@
 #include "generator.h"
 
+#include <atomic>
 #include <cmath>
+#include <complex>
+#include <thread>
+#include <vector>
 
 namespace dft3d {
 namespace gen {
@@ -80,6 +84,88 @@ void axis_matrix(int64_t n, int sign, double scale, const double* nodes, bool no
       M[2 * (k * n + j) + 1] = scale * im;
     }
   }
+}
+
+namespace {
+
+// all threads of a team meet here; sense-reversing spin barrier (the waits are microseconds long)
+struct SpinBarrier {
+  explicit SpinBarrier(int n) : count(n), waiting(0), sense(0) {}
+  void wait() {
+    const int my = sense.load(std::memory_order_acquire);
+    if (waiting.fetch_add(1, std::memory_order_acq_rel) + 1 == count) {
+      waiting.store(0, std::memory_order_relaxed);
+      sense.store(my ^ 1, std::memory_order_release);
+    } else {
+      while (sense.load(std::memory_order_acquire) == my) std::this_thread::yield();
+    }
+  }
+  const int count;
+  std::atomic<int> waiting, sense;
+};
+
+}  // namespace
+
+bool invert_matrix(int64_t n, double* Mraw, double* growth) {
+  using cd = std::complex<double>;
+  cd* A = reinterpret_cast<cd*>(Mraw);
+  double amax = 0.0;
+  for (int64_t i = 0; i < n * n; ++i) amax = std::fmax(amax, std::abs(A[i]));
+  std::vector<int64_t> perm(n);
+  int threads = int(std::thread::hardware_concurrency());
+  if (threads < 1) threads = 1;
+  if (threads > 16) threads = 16;
+  if (n < 128) threads = 1;
+  SpinBarrier barrier(threads);
+  std::atomic<int> singular(0);
+  // Gauss-Jordan in place: after step k column k holds column k of the inverse of the row-permuted matrix
+  auto worker = [&](int tid) {
+    for (int64_t k = 0; k < n; ++k) {
+      if (tid == 0) {
+        int64_t piv = k;
+        double best = std::abs(A[k * n + k]);
+        for (int64_t i = k + 1; i < n; ++i) {
+          const double v = std::abs(A[i * n + k]);
+          if (v > best) { best = v; piv = i; }
+        }
+        perm[k] = piv;
+        if (!(best > 0.0) || !std::isfinite(best)) {
+          singular.store(1);
+        } else {
+          if (piv != k)
+            for (int64_t j = 0; j < n; ++j) std::swap(A[k * n + j], A[piv * n + j]);
+          const cd inv = 1.0 / A[k * n + k];
+          A[k * n + k] = 1.0;
+          for (int64_t j = 0; j < n; ++j) A[k * n + j] *= inv;
+        }
+      }
+      barrier.wait();
+      if (singular.load()) return;
+      const cd* rk = A + k * n;
+      for (int64_t i = tid; i < n; i += threads) {
+        if (i == k) continue;
+        cd* ri = A + i * n;
+        const cd f = ri[k];
+        ri[k] = 0.0;
+        for (int64_t j = 0; j < n; ++j) ri[j] -= f * rk[j];
+      }
+      barrier.wait();
+    }
+  };
+  std::vector<std::thread> team;
+  for (int t = 1; t < threads; ++t) team.emplace_back(worker, t);
+  worker(0);
+  for (auto& t : team) t.join();
+  if (singular.load()) return false;
+  // undo the row exchanges: they become column exchanges of the inverse, in reverse order
+  for (int64_t k = n - 1; k >= 0; --k)
+    if (perm[k] != k)
+      for (int64_t i = 0; i < n; ++i) std::swap(A[i * n + k], A[i * n + perm[k]]);
+  double imax = 0.0;
+  for (int64_t i = 0; i < n * n; ++i) imax = std::fmax(imax, std::abs(A[i]));
+  if (!std::isfinite(imax)) return false;
+  if (growth) *growth = imax * amax;
+  return true;
 }
 
 void twiddle(int64_t N1, int64_t N2, int sign, double* T) {

@@ -16,6 +16,14 @@ void root_of_unity(int64_t num, int64_t den, int sign, double* re, double* im);
 //   nodes, on output : exp(sign*2*pi*i*nodes[k]*j)                  (Eq. 1 read literally)
 void axis_matrix(int64_t n, int sign, double scale, const double* nodes, bool nodes_on_output, double* M);
 
+// In-place inverse of a complex n x n matrix (interleaved, row-major) by Gauss-Jordan elimination with partial
+// pivoting in float64, rows shared among up to 16 host threads.  This is the inverse nonuniform transform of
+// Section III-A: for sample points that are not the roots of unity the matrix of Eq. 3 is not unitary and the inverse
+// "amounts to solving the linear system"; with the inverse as a table the solve is one more matrix product per axis.
+// Returns false if a pivot vanishes (the nodes are not distinct modulo 1); *growth receives max|inverse entry| *
+// max|matrix entry|, a cheap indication of how much accuracy the solve costs.
+bool invert_matrix(int64_t n, double* M, double* growth);
+
 // T[k1][beta] = exp(sign*2*pi*i*k1*beta/(N1*N2))  (phase adjustment of Eq. 17), N1*N2 complex entries
 void twiddle(int64_t N1, int64_t N2, int sign, double* T);
 

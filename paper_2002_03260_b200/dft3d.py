@@ -16,11 +16,12 @@ _LIB_PATH = os.environ.get("DFT3D_LIBRARY") or os.path.join(_HERE, "libdft3d.so"
 DFT3D_KDFT, DFT3D_FFT = 0, 1
 DFT3D_FORWARD, DFT3D_INVERSE = -1, +1
 DFT3D_NODES_ON_OUTPUT, DFT3D_UNSCALED_INVERSE, DFT3D_SPLIT_FP16, DFT3D_SPLIT_TF32, DFT3D_DESTROY_INPUT = 1, 2, 4, 8, 16
+DFT3D_INVERSE_SOLVE = 32
 
 EXPORTS = [
     "dft3d_plan_create", "dft3d_plan_create_ex", "dft3d_execute", "dft3d_execute_host", "dft3d_execute_axis",
     "dft3d_plan_status", "dft3d_plan_workspace_bytes", "dft3d_plan_launches", "dft3d_plan_split", "dft3d_plan_destroy",
-    "dft3d_status_string", "dft3d_last_error", "dft3d_generate_axis_matrix", "dft3d_generate_twiddle",
+    "dft3d_status_string", "dft3d_last_error", "dft3d_generate_axis_matrix", "dft3d_generate_twiddle", "dft3d_generate_inverse_matrix",
     "dft3d_generate_real_table", "dft3d_kdft_execute_static",
 ]
 
@@ -64,6 +65,7 @@ def _load():
     lib.dft3d_last_error.restype = ctypes.c_char_p
     lib.dft3d_generate_axis_matrix.argtypes = [ll, ci, cd, vp, ci, vp]
     lib.dft3d_generate_twiddle.argtypes = [ll, ll, ci, vp]
+    lib.dft3d_generate_inverse_matrix.argtypes = [ll, vp, ci, vp, vp]
     lib.dft3d_generate_real_table.argtypes = [ll, ci, cd, vp, ci, vp, vp]
     lib.dft3d_kdft_execute_static.argtypes = [ll, ll, ll, vp, vp, vp, vp, vp, vp, ctypes.c_char_p, ctypes.c_size_t]
     return lib
@@ -100,6 +102,16 @@ def generate_twiddle(N1, N2, sign=-1):
     T = np.empty((N1, N2), dtype=np.complex128)
     _check(_lib.dft3d_generate_twiddle(N1, N2, sign, T.ctypes.data))
     return T
+
+
+def generate_inverse_matrix(n, nodes, nodes_on_output=False):
+    """dft3d_generate_inverse_matrix: inverse of the forward matrix of `nodes` as complex128, and the growth figure
+    max|M| * max|M^-1| (host only)."""
+    M = np.empty((n, n), dtype=np.complex128)
+    growth = ctypes.c_double(0.0)
+    keep, ptr = _nodes_arg(nodes, n)
+    _check(_lib.dft3d_generate_inverse_matrix(n, ptr, int(nodes_on_output), M.ctypes.data, ctypes.byref(growth)))
+    return M, growth.value
 
 
 def generate_real_table(n, sign=-1, scale=1.0, nodes=None, nodes_on_output=False):

@@ -154,3 +154,24 @@ def test_generator_rejects_bad_arguments(dft):
     assert b._lib.dft3d_generate_twiddle(2, 2, -1, None) == 1
     bad = np.array([0.0, np.inf])
     assert b._lib.dft3d_generate_axis_matrix(2, -1, 1.0, bad.ctypes.data, 0, buf.ctypes.data) == 1
+
+
+def test_inverse_matrix_matches_the_solve(dft, oracle):
+    """The host-side inversion behind DFT3D_INVERSE_SOLVE (threaded Gauss-Jordan, no library) against the oracle's
+    LAPACK solve and the defining identity; singular node sets are refused."""
+    rng = np.random.default_rng(7)
+    for n in (2, 16, 100, 300):
+        nodes = (np.arange(n) + 0.3 * rng.uniform(-1, 1, n)) / n
+        Minv, growth = dft.generate_inverse_matrix(n, nodes)
+        V = oracle.axis_matrix(n, -1, 1.0, nodes)
+        assert np.abs(Minv @ V - np.eye(n)).max() < 1e-11 and growth > 0
+        X = rng.standard_normal((1, n, 3)) + 1j * rng.standard_normal((1, n, 3))
+        want = oracle.solve_axis(X, 1, nodes)
+        got = np.einsum("kj,ajc->akc", Minv, X)
+        assert np.abs(got - want).max() < 1e-11 * max(1.0, growth * n)
+    with pytest.raises(dft.Dft3dError) as e:
+        dft.generate_inverse_matrix(4, np.array([0.25, 0.5, 0.25, 0.75]))   # two equal nodes: two equal columns
+    assert e.value.status == 1
+    # nodes that coincide up to rounding (1.1 is not 0.1 + 1 in binary): no zero pivot, but the growth figure says it
+    _, growth = dft.generate_inverse_matrix(4, np.array([0.1, 0.3, 1.1, 0.7]))
+    assert growth > 1e12

@@ -719,3 +719,42 @@ def test_2d_kdft_8192_squared_separable_input(lib, oracle):
     got = y.cpu().numpy().reshape(n, n).astype(np.complex128)
     err = np.linalg.norm(got - ref) / np.linalg.norm(ref)
     assert err < SANITY, err
+
+
+# ------------------------------------------------------------------ inverse nonuniform transform
+
+@pytest.mark.parametrize("split", SPLITS)
+def test_inverse_solve_undoes_the_nonuniform_forward_transform(lib, oracle, split):
+    """DFT3D_INVERSE_SOLVE: nodes jittered around the uniform grid on two axes, a uniform third axis.  The solve
+    plan returns the input of the forward plan, and agrees with the oracle's LAPACK solve of the same system."""
+    shape = (64, 128, 192)
+    rng = np.random.default_rng(103)
+    nodes = [(np.arange(n) + 0.3 * rng.uniform(-1, 1, n)) / n for n in shape]
+    nodes[1] = None
+    x = _inputs().cube(shape, "normal", 104, device="cuda")
+    sf = _split_flag(lib, split)
+    fwd = lib.Plan(*shape, nodes=nodes, flags=sf)
+    X = fwd(x)
+    _finish(fwd)
+    fwd.destroy()
+    inv = lib.Plan(*shape, sign=lib.DFT3D_INVERSE, nodes=nodes, flags=sf | lib.DFT3D_INVERSE_SOLVE)
+    back = inv(X)
+    _finish(inv)
+    inv.destroy()
+    assert oracle.rel_l2(back.cpu().numpy(), x.cpu().numpy()) < TOL                     # two transforms in a row
+    want = oracle.solve3d(X.cpu().numpy().astype(np.complex128), nodes)
+    assert oracle.rel_l2(back.cpu().numpy(), want) < SANITY
+    # the conjugate-kernel product (no flag) is NOT the inverse for these nodes
+    plain = lib.Plan(*shape, sign=lib.DFT3D_INVERSE, nodes=nodes, flags=sf)
+    y = plain(X)
+    _finish(plain)
+    plain.destroy()
+    assert oracle.rel_l2(y.cpu().numpy(), x.cpu().numpy()) > 1e-2
+    # hopeless node sets and misuse are refused
+    bad = [np.sort(rng.uniform(0, 1, n)) for n in shape]
+    with pytest.raises(lib.Dft3dError) as e:
+        lib.Plan(*shape, sign=lib.DFT3D_INVERSE, nodes=bad, flags=lib.DFT3D_INVERSE_SOLVE)
+    assert e.value.status == 2
+    with pytest.raises(lib.Dft3dError) as e:
+        lib.Plan(*shape, sign=lib.DFT3D_FORWARD, nodes=nodes, flags=lib.DFT3D_INVERSE_SOLVE)
+    assert e.value.status == 1

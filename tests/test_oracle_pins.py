@@ -283,3 +283,43 @@ def test_two_stage_refactoring_equals_definition(oracle, N1, N2):
     for sign in (-1, +1):
         want = oracle.dft3d(x, sign=sign)[0, 0]
         assert oracle.rel_l2(two_stage_dft_1d(x[0, 0], N1, N2, sign), want) < 1e-12
+
+
+# ------------------------------------------------------------------ inverse nonuniform transform (the linear solve)
+
+def test_solve_axis_uniform_nodes_is_the_inverse_dft(oracle):
+    """Nodes j/n: the system matrix is the DFT matrix, whose inverse is known in closed form; numpy's ifft is the
+    independent opinion."""
+    rng = np.random.default_rng(5)
+    n = 24
+    X = rng.standard_normal((3, n, 2)) + 1j * rng.standard_normal((3, n, 2))
+    got = oracle.solve_axis(X, 1, np.arange(n) / n)
+    assert np.abs(got - np.fft.ifft(X, axis=1)).max() < 1e-12
+
+
+def test_solve_axis_two_points_closed_form(oracle):
+    """n = 2, nodes (t0, t1): V = [[1, 1], [w0, w1]], w = exp(-2 pi i t); x = V^-1 X written out by hand."""
+    t0, t1 = 0.1, 0.65
+    w0, w1 = np.exp(-2j * np.pi * t0), np.exp(-2j * np.pi * t1)
+    X = np.array([2.0 - 1.0j, 0.5 + 3.0j])
+    det = w1 - w0
+    want = np.array([(w1 * X[0] - X[1]) / det, (-w0 * X[0] + X[1]) / det])
+    got = oracle.solve_axis(X.reshape(1, 1, 2), 2, np.array([t0, t1])).reshape(2)
+    assert np.abs(got - want).max() < 1e-14
+
+
+def test_solve_undoes_the_forward_nonuniform_transform(oracle):
+    """solve3d(dft3d(x)) = x for jittered nodes on two axes and a uniform third axis; and V x = X holds with V typed
+    here from Eq. 3."""
+    rng = np.random.default_rng(6)
+    shape = (6, 10, 8)
+    nodes = [(np.arange(n) + 0.3 * rng.uniform(-1, 1, n)) / n for n in shape]
+    nodes[2] = None
+    x = rng.standard_normal(shape) + 1j * rng.standard_normal(shape)
+    X = oracle.dft3d(x, nodes=nodes)
+    assert np.abs(oracle.solve3d(X, nodes) - x).max() < 1e-11
+    n = shape[1]
+    V = np.exp(-2j * np.pi * np.outer(np.arange(n), nodes[1]))
+    y = rng.standard_normal((1, n, 1)) + 1j * rng.standard_normal((1, n, 1))
+    sol = oracle.solve_axis(y, 1, nodes[1]).reshape(n)
+    assert np.abs(V @ sol - y.reshape(n)).max() < 1e-11
