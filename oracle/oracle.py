@@ -5,7 +5,10 @@ import this module.  The product package never does, and this module imports
 nothing from the product package.
 
 The functions mirror oracle_dft.c one to one; see that file for the passages
-of the paper each of them follows (Eq. 11-14, Eq. 3, Eq. 5).
+of the paper each of them follows (Eq. 11-14, Eq. 3, Eq. 5).  solve_axis /
+solve3d (the inverse nonuniform transform of Section III-A as a linear solve)
+are written here, with numpy.linalg.solve as the library step.  Every function
+is pinned in tests/test_oracle_pins.py; none is "parity unpinned".
 """
 import ctypes
 import os
