@@ -59,10 +59,11 @@ def conv_flops(n):
 
 # DRAM bytes per point per launch (dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture divided by the
 # points of that launch; smaller cases than the bench workload, traffic grows in proportion to the points):
-#   profiles/fft_axis_kernel_256x1024x1024.md : (2.148 + 2.094) GB / 268.4 M points
-#   profiles/kdft_axis_kernel_512.md          : (1.084 + 1.035) GB / 134.2 M points
-NCU_DRAM_BYTES_PER_POINT = {"fft_axis_kernel": 15.80, "fft_f16_axis_kernel": 15.82, "kdft_axis_kernel": 15.79,
-                            "kdft_f16_axis_kernel": 15.79}
+#   profiles/fft_f16_axis_kernel_256x1024x1024.md : mean of the three launches, (2.187 + 2.100) GB / 268.4 M points
+#   profiles/kdft_f16_axis_kernel_512.md          : mean of the three launches, (1.081 + 1.031) GB / 134.2 M points
+#   (the TF32-piece kernels, captured before: 15.80 and 15.79)
+NCU_DRAM_BYTES_PER_POINT = {"fft_axis_kernel": 15.80, "fft_f16_axis_kernel": 15.97, "kdft_axis_kernel": 15.79,
+                            "kdft_f16_axis_kernel": 15.73}
 
 
 def measured_peaks():
