@@ -101,7 +101,8 @@ typedef struct dft3d_options_s {
  *
  * Supported sizes: KDFT: every n_a even, n_a <= 8192 (tiles that are not full are zero-filled on load
  * and masked on store, the way the paper's compiler pads to its hardware's preferred shapes).  FFT: every
- * transformed n_a in {256, 512, 1024, 2048} (N = R*R or 2*R*R with R = 16 or 32), the others multiples of 64.
+ * transformed n_a in {256, 512, 1024, 2048, 4096} (N = R*R, 2*R*R or 4*R*R with R = 16 or 32; 4096 with fp16
+ * pieces only), the others multiples of 64.
  * Other sizes return DFT3D_ERR_UNSUPPORTED.
  */
 int dft3d_plan_create(dft3d_plan_t* out, long long n0, long long n1, long long n2, int mode, int sign,

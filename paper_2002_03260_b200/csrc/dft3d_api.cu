@@ -195,6 +195,9 @@ int set_kernel_attributes(int device) {
   DFT3D_FFT16_ATTR(dft3d::FFT_STRIDED, 16, 1, 16, 1);
   DFT3D_FFT16_ATTR(dft3d::FFT_STRIDED, 32, 2, 8, 1);
   DFT3D_FFT16_ATTR(dft3d::FFT_STRIDED, 16, 2, 16, 1);
+  DFT3D_FFT16_ATTR(dft3d::FFT_CONTIG, 32, 4, 16, 0);
+  DFT3D_FFT16_ATTR(dft3d::FFT_STRIDED, 32, 4, 4, 0);
+  DFT3D_FFT16_ATTR(dft3d::FFT_STRIDED, 32, 4, 4, 1);
 #undef DFT3D_FFT16_ATTR
   done = true;
   return DFT3D_OK;
@@ -426,15 +429,18 @@ int build_fft_axis(dft3d_plan_s* p, int a, const int split[2]) {
   if (n == 512) { R = 16; RX = 2; }
   if (n == 1024) { R = 32; }
   if (n == 2048) { R = 32; RX = 2; }
+  if (n == 4096 && p->f16) { R = 32; RX = 4; }   // three factors: 4 * 32 * 32 (fp16-piece kernel only)
   if (!R)
-    return fail(DFT3D_ERR_UNSUPPORTED, "FFT mode supports axis lengths 256, 512, 1024 and 2048; n%d = %lld", a, n);
+    return fail(DFT3D_ERR_UNSUPPORTED, "FFT mode supports axis lengths 256, 512, 1024, 2048 and (fp16 pieces) 4096; "
+                "n%d = %lld", a, n);
   if ((split[0] || split[1]) && (split[0] != RX * R || split[1] != R))
     return fail(DFT3D_ERR_UNSUPPORTED, "FFT split %dx%d for n%d = %lld is not supported (only %dx%d)", split[0],
                 split[1], a, n, RX * R, R);
   ax.n = n;
   ax.R = R;
   ax.RX = RX;
-  ax.cols = (R == 32 && RX == 2) ? 8 : 16;   // default; fft_axis_pass may pick 8 for R = 32, RX = 1 (see there)
+  ax.cols = (R == 32 && RX == 4) ? 4 : ((R == 32 && RX == 2) ? 8 : 16);   // a 128 KB stage holds all n rows of `cols` lines
+                                                                           // (fft_axis_pass may pick 8 for R = 32, RX = 1)
   const bool scaled = (p->sign > 0) && !(p->flags & DFT3D_UNSCALED_INVERSE);
   const int K = 2 * R, NB = 2 * R, panels = K / 32;
   if (p->f16) {
@@ -466,16 +472,18 @@ int build_fft_axis(dft3d_plan_s* p, int a, const int split[2]) {
     DFT3D_CUDA(cudaMemcpy(ax.d_w, W.data(), W.size() * sizeof(__half), cudaMemcpyHostToDevice));
     DFT3D_CUDA(cudaMalloc(&ax.d_tw, tw.size() * sizeof(float)));
     DFT3D_CUDA(cudaMemcpy(ax.d_tw, tw.data(), tw.size() * sizeof(float), cudaMemcpyHostToDevice));
-    if (RX == 2) {
-      std::vector<float> tw2(size_t(2) * R * R);
-      for (long long m = 0; m < (long long)R * R; ++m) {
-        double re, im;
-        dft3d::gen::root_of_unity(m, n, p->sign, &re, &im);
-        tw2[2 * m] = float(re);
-        tw2[2 * m + 1] = float(im);
-      }
+    if (RX >= 2) {
+      // exp(s*2*pi*i*b*m/n) for b = 1 .. RX-1, m < R*R: the twiddles between the radix-RX step and the R*R-point parts
+      std::vector<float> tw2(size_t(2) * (RX - 1) * R * R);
+      for (int b = 1; b < RX; ++b)
+        for (long long m = 0; m < (long long)R * R; ++m) {
+          double re, im;
+          dft3d::gen::root_of_unity((b * m) % n, n, p->sign, &re, &im);
+          tw2[2 * ((b - 1) * (size_t)R * R + m)] = float(re);
+          tw2[2 * ((b - 1) * (size_t)R * R + m) + 1] = float(im);
+        }
       DFT3D_CUDA(cudaMalloc(&ax.d_tw2, tw2.size() * sizeof(float)));
-      DFT3D_CUDA(cudaMemcpy(ax.d_tw2, tw2.data(), tw2.size() * sizeof(float), cudaMemcpyHostToDevice));
+      DFT3D_CUDA(cudaMemcpy(ax.d_tw2, tw2.size() ? tw2.data() : nullptr, tw2.size() * sizeof(float), cudaMemcpyHostToDevice));
     }
     const unsigned long long dims[2] = {64ull, (unsigned long long)(2 * NB)};
     const unsigned long long strides[1] = {128ull};
@@ -627,6 +635,7 @@ int fft_axis_pass(dft3d_plan_s* p, int axis, const float* in, float* out, cudaSt
     dft3d::FftF16Params hp;
     hp.base = fp;
     hp.out_mul = ax.out_mul;
+    hp.quarter_turn = float(p->sign);
     hp.base.raw_stages = dft3d::kFft16RawBytes / fp.stage_bytes;
     if (hp.base.raw_stages > 4) hp.base.raw_stages = 4;
     // a worker group takes every fourth M-tile, i.e. every (4 / tiles per stage)-th stage: that step must divide the
@@ -643,18 +652,21 @@ int fft_axis_pass(dft3d_plan_s* p, int axis, const float* in, float* out, cudaSt
     if (axis == 2) {
       if (R == 32 && RX == 1) DFT3D_FFT16_LAUNCH(dft3d::FFT_CONTIG, 32, 1, 16, 0);
       else if (R == 16 && RX == 1) DFT3D_FFT16_LAUNCH(dft3d::FFT_CONTIG, 16, 1, 16, 0);
+      else if (R == 32 && RX == 4) DFT3D_FFT16_LAUNCH(dft3d::FFT_CONTIG, 32, 4, 16, 0);
       else if (R == 32) DFT3D_FFT16_LAUNCH(dft3d::FFT_CONTIG, 32, 2, 16, 0);
       else DFT3D_FFT16_LAUNCH(dft3d::FFT_CONTIG, 16, 2, 16, 0);
     } else if (!stage_out) {
       if (R == 32 && RX == 1 && cols == 16) DFT3D_FFT16_LAUNCH(dft3d::FFT_STRIDED, 32, 1, 16, 0);
       else if (R == 32 && RX == 1) DFT3D_FFT16_LAUNCH(dft3d::FFT_STRIDED, 32, 1, 8, 0);
       else if (R == 16 && RX == 1) DFT3D_FFT16_LAUNCH(dft3d::FFT_STRIDED, 16, 1, 16, 0);
+      else if (R == 32 && RX == 4) DFT3D_FFT16_LAUNCH(dft3d::FFT_STRIDED, 32, 4, 4, 0);
       else if (R == 32) DFT3D_FFT16_LAUNCH(dft3d::FFT_STRIDED, 32, 2, 8, 0);
       else DFT3D_FFT16_LAUNCH(dft3d::FFT_STRIDED, 16, 2, 16, 0);
     } else {
       if (R == 32 && RX == 1 && cols == 16) DFT3D_FFT16_LAUNCH(dft3d::FFT_STRIDED, 32, 1, 16, 1);
       else if (R == 32 && RX == 1) DFT3D_FFT16_LAUNCH(dft3d::FFT_STRIDED, 32, 1, 8, 1);
       else if (R == 16 && RX == 1) DFT3D_FFT16_LAUNCH(dft3d::FFT_STRIDED, 16, 1, 16, 1);
+      else if (R == 32 && RX == 4) DFT3D_FFT16_LAUNCH(dft3d::FFT_STRIDED, 32, 4, 4, 1);
       else if (R == 32) DFT3D_FFT16_LAUNCH(dft3d::FFT_STRIDED, 32, 2, 8, 1);
       else DFT3D_FFT16_LAUNCH(dft3d::FFT_STRIDED, 16, 2, 16, 1);
     }

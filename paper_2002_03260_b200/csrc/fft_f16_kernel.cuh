@@ -18,6 +18,11 @@
 // An element more than 2^18 below its line's largest keeps less than full relative precision (its lo piece becomes
 // subnormal: absolute error 2^-38 of the line's largest element), which is invisible in the norm-wise error.
 //
+// Lengths N = RX*R*R.  RX = 2 (512, 2048) and RX = 4 (4096 = 4*32*32, a three-factor split) apply Eq. 17 once more with
+// P = N/RX before the two GEMM stages: the thread of sub-line b forms  y_b[m] = (sum_q x[m + q*N/RX] * w_RX^(b*q)) *
+// exp(s*2*pi*i*b*m/N)  for m < R*R (a radix-RX butterfly on the CUDA cores: additions, swaps and one complex
+// multiplication), and X[RX*k + b] is entry k of the R*R-point transform of y_b.
+//
 // Organisation.  The per-tile chain  split -> MMA 1 -> drain 1 (+twiddle) -> MMA 2 -> drain 2 (+store)  is latency
 // bound when every link is one warp group (the TF32 kernel's design: each group sees one warp per scheduler).  Here
 // four identical worker groups each take every fourth M-tile through ALL the links, so each scheduler always has four
@@ -43,6 +48,7 @@ namespace dft3d {
 struct FftF16Params {
   FftParams base;               // twiddle: T[k1][beta] * 2^-(10 + log2(R) - 1), unscaled otherwise
   float out_mul;                // 2^(log2(R) - 1 - 10), times 1/n for a scaled inverse
+  float quarter_turn;           // RX == 4: the sign s of the exponent (exp(s*2*pi*i/4) = s*i)
 };
 
 struct FftF16Shared {
@@ -60,7 +66,8 @@ __host__ __device__ constexpr int fft16_tw_bytes(int R) { return R * R * 8; }
 constexpr int kFft16A2Piece = 128 * 128;
 constexpr int kFft16RawBytes = 128 * 1024;
 __host__ __device__ constexpr size_t fft16_smem_bytes(int R, int RX) {   // RX == 2: a second twiddle table (radix-2 step)
-  return size_t(fft16_w_bytes(R)) + 4 * size_t(kFft16A2Piece) + size_t(RX) * fft16_tw_bytes(R) + kFft16RawBytes + 1024 + 1024;
+  return size_t(fft16_w_bytes(R)) + 4 * size_t(kFft16A2Piece) + size_t(RX == 2 ? 2 : 1) * fft16_tw_bytes(R) +
+         kFft16RawBytes + 1024 + 1024;
 }
 
 #define F16_WAIT(bar, parity, code)                                 \
@@ -132,7 +139,7 @@ fft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_c
   uint8_t* smem_a2 = smem_w + fft16_w_bytes(R);            // buffer i = [hi piece][lo piece] at i * 2 * a2_piece
   float2* smem_tw = reinterpret_cast<float2*>(smem_a2 + 4 * a2_piece);
   float2* smem_tw2 = smem_tw + R * R;                      // RX == 2 only: exp(s*2*pi*i*m/N), m < R*R
-  uint8_t* smem_rawring = reinterpret_cast<uint8_t*>(smem_tw) + RX * fft16_tw_bytes(R);
+  uint8_t* smem_rawring = reinterpret_cast<uint8_t*>(smem_tw) + (RX == 2 ? 2 : 1) * fft16_tw_bytes(R);
   FftF16Shared& sh = *reinterpret_cast<FftF16Shared*>(smem_rawring + kFft16RawBytes);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 #ifdef DFT3D_PROFILE_WAITS
@@ -303,10 +310,10 @@ fft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_c
     // stage-1 lane = (sub-line sl1, beta), beta fastest; stage-2 lane = (sub-line sl2, k1)
     const int sl1 = m / R, beta = m % R;
     // Which line of the stage and which butterfly output a sub-line is.  CONTIG: the RX sub-lines of a line sit in one
-    // M-tile.  STRIDED with RX == 2: an M-tile holds the SAME butterfly output of SL neighbouring lines (tiles 2u and
-    // 2u+1 are the a and b halves of lines u*SL ...), so that a stage-2 store still covers SL neighbouring columns of
+    // M-tile.  STRIDED with RX >= 2: an M-tile holds the SAME butterfly output of SL neighbouring lines (tiles RX*u ..
+    // RX*u + RX-1 are the RX outputs of lines u*SL ...), so that a stage-2 store still covers SL neighbouring columns of
     // one output row (32 bytes) instead of SL/2.
-    constexpr bool kPairTiles = (MODE == FFT_STRIDED) && (RX == 2);
+    constexpr bool kPairTiles = (MODE == FFT_STRIDED) && (RX >= 2);
     const int g1 = kPairTiles ? sl1 : sl1 / RX;         // line within the tile (kPairTiles: within the pair of tiles)
     const int bsel1_fixed = sl1 % RX;
     // stage-2 lanes.  CONTIG: (line, k1, butterfly output), output fastest, so that the lanes of a warp store
@@ -342,8 +349,8 @@ fft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_c
       const uint32_t s = uint32_t(istage % p.raw_stages), phs = uint32_t(istage / p.raw_stages) & 1;
       const uint32_t pk = uint32_t(t >> 2) & 1;
       uint8_t* stage = smem_rawring + size_t(s) * p.stage_bytes;
-      const int bsel1 = kPairTiles ? (mt & 1) : bsel1_fixed, bsel2 = kPairTiles ? (mt & 1) : bsel2_fixed;
-      const int col0 = kPairTiles ? (mt >> 1) * SL : mt * Lg;     // first column of the stage this tile's lines occupy
+      const int bsel1 = kPairTiles ? (mt % RX) : bsel1_fixed, bsel2 = kPairTiles ? (mt % RX) : bsel2_fixed;
+      const int col0 = kPairTiles ? (mt / RX) * SL : mt * Lg;     // first column of the stage this tile's lines occupy
 
       // ---- split: this lane's R elements (after the butterfly when RX == 2) -> scaled fp16 pieces -> A1
       F16_WAIT_WARP(&sh.raw_full[s], phs, 0x701);
@@ -356,7 +363,7 @@ fft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_c
           half = uint32_t(NL) * 8u;
         } else {
           const int c = col0 + g1;                  // column within the stage
-          const uint32_t swz = (COLS == 16) ? uint32_t(beta & 7) : uint32_t((beta >> 1) & 3);   // TMA swizzle of the row
+          const uint32_t swz = (COLS == 16) ? uint32_t(beta & 7) : (COLS == 8 ? uint32_t((beta >> 1) & 3) : 0u);   // TMA swizzle of the row (none for 32-byte rows)
           base = uint32_t(beta) * kRowBytes + ((uint32_t(c >> 1) ^ swz) << 4) + uint32_t(c & 1) * 8u;
           stride = uint32_t(R) * kRowBytes;
           half = uint32_t(NL) * kRowBytes;
@@ -368,6 +375,31 @@ fft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_c
           const uint2 v = *reinterpret_cast<const uint2*>(stage + base + uint32_t(l) * stride);
           if (RX == 1) {
             xr[l] = __uint_as_float(v.x); xi[l] = __uint_as_float(v.y);
+          } else if (RX == 4) {
+            // radix-4 butterfly: u_q = x[m + q*N/4]; y_0 = (u0+u2)+(u1+u3), y_2 = (u0+u2)-(u1+u3),
+            // y_1 = (u0-u2) + w(u1-u3), y_3 = (u0-u2) - w(u1-u3) with w = exp(s*2*pi*i/4) = s*i; then the twiddle
+            const uint2 v1 = *reinterpret_cast<const uint2*>(stage + base + half + uint32_t(l) * stride);
+            const uint2 v2 = *reinterpret_cast<const uint2*>(stage + base + 2 * half + uint32_t(l) * stride);
+            const uint2 v3 = *reinterpret_cast<const uint2*>(stage + base + 3 * half + uint32_t(l) * stride);
+            const float u0r = __uint_as_float(v.x), u0i = __uint_as_float(v.y), u1r = __uint_as_float(v1.x), u1i = __uint_as_float(v1.y);
+            const float u2r = __uint_as_float(v2.x), u2i = __uint_as_float(v2.y), u3r = __uint_as_float(v3.x), u3i = __uint_as_float(v3.y);
+            float yr, yi;
+            if ((bsel1 & 1) == 0) {
+              const float ar = u0r + u2r, ai = u0i + u2i, cr = u1r + u3r, ci = u1i + u3i;
+              yr = bsel1 == 0 ? ar + cr : ar - cr;
+              yi = bsel1 == 0 ? ai + ci : ai - ci;
+            } else {
+              const float br = u0r - u2r, bi = u0i - u2i, dr = u1r - u3r, di = u1i - u3i;
+              const float wr = -pp.quarter_turn * di, wi = pp.quarter_turn * dr;       // (s*i) * d
+              yr = bsel1 == 1 ? br + wr : br - wr;
+              yi = bsel1 == 1 ? bi + wi : bi - wi;
+            }
+            if (bsel1 == 0) {
+              xr[l] = yr; xi[l] = yi;
+            } else {
+              const float2 tw = __ldg(p.twiddle2 + (bsel1 - 1) * NL + l * R + beta);   // exp(s*2*pi*i*b*m/N)
+              xr[l] = yr * tw.x - yi * tw.y; xi[l] = yr * tw.y + yi * tw.x;
+            }
           } else {
             const uint2 w = *reinterpret_cast<const uint2*>(stage + base + half + uint32_t(l) * stride);
             const float ur = __uint_as_float(v.x), ui = __uint_as_float(v.y);
@@ -397,7 +429,7 @@ fft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_c
         const float in_scale = __uint_as_float((267u - f) << 23);
         const uint64_t scale2 = pack2(in_scale, in_scale);
         inv_scale = __uint_as_float((f - 13u) << 23);
-        if (MODE == FFT_STRIDED || RX == 2) {
+        if (MODE == FFT_STRIDED || RX >= 2) {
           // the stage-2 lanes of this thread belong to another (sub-)line: exchange through shared memory
           // (a bounded mbarrier rather than a named barrier: a warp that gave up a wait must not strand the others)
           if (beta == 0) sh.line_scale[g][sl1] = inv_scale;
@@ -507,7 +539,7 @@ fft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_c
 #pragma unroll
             for (int j = 0; j < 16; ++j) {
               const int k = RX * (k1 + R * (ch * 16 + j)) + bsel2;
-              const uint32_t swz = (COLS == 16) ? uint32_t(k & 7) : uint32_t((k >> 1) & 3);
+              const uint32_t swz = (COLS == 16) ? uint32_t(k & 7) : (COLS == 8 ? uint32_t((k >> 1) & 3) : 0u);
               const uint32_t off = uint32_t(k) * kRowBytes + ((uint32_t(c >> 1) ^ swz) << 4) + uint32_t(c & 1) * 8u;
               *reinterpret_cast<float2*>(stage + off) = make_float2(f[2 * j], f[2 * j + 1]);
             }
