@@ -31,7 +31,7 @@ extern "C" {
 
 typedef struct dft3d_plan_s* dft3d_plan_t;
 
-enum { DFT3D_KDFT = 0, DFT3D_FFT = 1 };          /* mode */
+enum { DFT3D_KDFT = 0, DFT3D_FFT = 1, DFT3D_AUTO = 2 }; /* mode; AUTO: per axis, FFT where it applies, else KDFT */
 enum { DFT3D_FORWARD = -1, DFT3D_INVERSE = +1 }; /* sign of the exponent (Eq. 14 has the minus sign) */
 
 enum {
@@ -85,7 +85,10 @@ typedef struct dft3d_options_s {
  * Create a plan for an n0 x n1 x n2 transform (Eq. 11 / Eq. 12).
  *
  *   out      receives the handle; set to NULL on failure.
- *   mode     DFT3D_KDFT or DFT3D_FFT.
+ *   mode     DFT3D_KDFT, DFT3D_FFT, or DFT3D_AUTO: the FFT formulation on every transformed axis that has a uniform
+ *            grid, a length the FFT kernels take and at least 16 neighbouring lines, the KDFT formulation on the
+ *            others (nonuniform nodes, other even lengths).  A plan that ends up with both needs one cube of
+ *            workspace (or DFT3D_DESTROY_INPUT) and runs every pass in the natural layout.
  *   sign     DFT3D_FORWARD: kernel exp(-2*pi*i*k*t), unscaled (Eq. 14).
  *            DFT3D_INVERSE: conjugate kernel, each axis scaled by 1/n_a so that
  *            inverse(forward(x)) = x on uniform grids (the paper describes the inverse

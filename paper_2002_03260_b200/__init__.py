@@ -5,7 +5,7 @@ The binding (and with it libdft3d.so) is loaded on first use of any public name,
 """
 import importlib
 
-__all__ = ["Plan", "Dft3dError", "DFT3D_KDFT", "DFT3D_FFT", "DFT3D_FORWARD", "DFT3D_INVERSE",
+__all__ = ["Plan", "Dft3dError", "DFT3D_KDFT", "DFT3D_FFT", "DFT3D_AUTO", "DFT3D_FORWARD", "DFT3D_INVERSE",
            "DFT3D_NODES_ON_OUTPUT", "DFT3D_UNSCALED_INVERSE", "DFT3D_SPLIT_FP16", "DFT3D_SPLIT_TF32", "DFT3D_DESTROY_INPUT", "DFT3D_INVERSE_SOLVE", "generate_inverse_matrix", "generate_axis_matrix", "generate_real_table",
            "generate_twiddle", "kdft_execute_static", "library_path"]
 

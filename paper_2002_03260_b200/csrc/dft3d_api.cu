@@ -120,6 +120,7 @@ struct dft3d_plan_s {
   unsigned flags = 0;
   bool f16 = false;       // fp16 pieces (else TF32 pieces)
   bool in_is_ws = false;  // DFT3D_DESTROY_INPUT: the caller's input buffer serves as the workspace
+  int amode[3] = {0, 0, 0};  // DFT3D_AUTO with both formulations in one plan: the formulation of each axis
   unsigned axes = 7;            // bit a: axis a is transformed
   int device = 0;
   int sm_count = 0;
@@ -802,7 +803,8 @@ int dft3d_plan_create_ex(dft3d_plan_t* out, long long n0, long long n1, long lon
   if (!out) return fail(DFT3D_ERR_INVALID_ARG, "out is NULL");
   *out = nullptr;
   if (n0 < 1 || n1 < 1 || n2 < 1) return fail(DFT3D_ERR_INVALID_ARG, "sizes must be >= 1");
-  if (mode != DFT3D_KDFT && mode != DFT3D_FFT) return fail(DFT3D_ERR_INVALID_ARG, "mode must be DFT3D_KDFT or DFT3D_FFT");
+  if (mode != DFT3D_KDFT && mode != DFT3D_FFT && mode != DFT3D_AUTO)
+    return fail(DFT3D_ERR_INVALID_ARG, "mode must be DFT3D_KDFT, DFT3D_FFT or DFT3D_AUTO");
   if (sign != DFT3D_FORWARD && sign != DFT3D_INVERSE) return fail(DFT3D_ERR_INVALID_ARG, "sign must be -1 or +1");
   const long long nn[3] = {n0, n1, n2};
   const double* nodes[3] = {nodes0, nodes1, nodes2};
@@ -821,8 +823,8 @@ int dft3d_plan_create_ex(dft3d_plan_t* out, long long n0, long long n1, long lon
                     DFT3D_INVERSE_SOLVE))
     return fail(DFT3D_ERR_INVALID_ARG, "unknown flag");
   if (opt.flags & DFT3D_INVERSE_SOLVE) {
-    if (mode != DFT3D_KDFT || sign != DFT3D_INVERSE || (opt.flags & DFT3D_UNSCALED_INVERSE))
-      return fail(DFT3D_ERR_INVALID_ARG, "DFT3D_INVERSE_SOLVE needs mode KDFT, sign +1 and the scaled inverse");
+    if (mode == DFT3D_FFT || sign != DFT3D_INVERSE || (opt.flags & DFT3D_UNSCALED_INVERSE))
+      return fail(DFT3D_ERR_INVALID_ARG, "DFT3D_INVERSE_SOLVE needs mode KDFT (or AUTO), sign +1 and the scaled inverse");
     for (int a = 0; a < 3; ++a)
       if (nodes[a] && nn[a] > 2048)
         return fail(DFT3D_ERR_UNSUPPORTED, "DFT3D_INVERSE_SOLVE inverts the n x n matrix on the host: n%d = %lld exceeds 2048", a, nn[a]);
@@ -838,7 +840,7 @@ int dft3d_plan_create_ex(dft3d_plan_t* out, long long n0, long long n1, long lon
     if (a == 0 && !transformed) continue;   // a pure batch index
     // KDFT: rows of the table and of the data must start on 16-byte boundaries (TMA), i.e. even lengths;
     // FFT: the untransformed axes are split into groups of 16 lines
-    const long long quantum = (mode == DFT3D_KDFT) ? 2 : 64;
+    const long long quantum = (mode == DFT3D_FFT) ? 64 : 2;
     if (nn[a] % quantum != 0)
       return fail(DFT3D_ERR_UNSUPPORTED, "n%d = %lld is not a multiple of %lld", a, nn[a], quantum);
     if (transformed && nn[a] > 8192) return fail(DFT3D_ERR_UNSUPPORTED, "n%d = %lld exceeds 8192", a, nn[a]);
@@ -850,6 +852,26 @@ int dft3d_plan_create_ex(dft3d_plan_t* out, long long n0, long long n1, long lon
   }
   if (mode == DFT3D_FFT && (nodes0 || nodes1 || nodes2))
     return fail(DFT3D_ERR_UNSUPPORTED, "the FFT formulation needs a uniform grid (no nodes)");
+  // DFT3D_AUTO: the FFT formulation on every axis where it applies (uniform grid, a supported length, and enough
+  // neighbouring lines for its stages), the KDFT formulation on the others
+  int amode[3] = {mode, mode, mode};
+  if (mode == DFT3D_AUTO) {
+    const long long inner[3] = {n1 * n2, n2, n0 * n1};   // columns beside a line (axes 0, 1) / number of lines (axis 2)
+    bool all_fft = true, all_kdft = true, fft_sizes_ok = true;
+    for (int a = 0; a < 3; ++a) {
+      if (!((axes >> a) & 1u)) { if (a != 0 && nn[a] % 64 != 0) fft_sizes_ok = false; continue; }
+      const long long n = nn[a];
+      const bool length_ok = n == 256 || n == 512 || n == 1024 || n == 2048 || (n == 4096 && f16);
+      const bool fft_ok = !nodes[a] && length_ok && inner[a] % 16 == 0;
+      amode[a] = fft_ok ? DFT3D_FFT : DFT3D_KDFT;
+      (fft_ok ? all_kdft : all_fft) = false;
+      if (nn[a] % 64 != 0) fft_sizes_ok = false;
+    }
+    if (all_kdft) mode = DFT3D_KDFT;                       // one formulation only: its own schedules apply
+    else if (all_fft && fft_sizes_ok) mode = DFT3D_FFT;
+    if (mode != DFT3D_AUTO)
+      for (int a = 0; a < 3; ++a) amode[a] = mode;
+  }
 
   int ndev = 0;
   if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev < 1) return fail(DFT3D_ERR_CUDA, "no CUDA device available");
@@ -859,6 +881,7 @@ int dft3d_plan_create_ex(dft3d_plan_t* out, long long n0, long long n1, long lon
   do {
     for (int a = 0; a < 3; ++a) p->n[a] = nn[a];
     p->mode = mode;
+    for (int a = 0; a < 3; ++a) p->amode[a] = amode[a];
     p->sign = sign;
     p->flags = opt.flags;
     p->f16 = f16;
@@ -889,7 +912,32 @@ int dft3d_plan_create_ex(dft3d_plan_t* out, long long n0, long long n1, long lon
 #endif
     e = cudaMalloc(&p->d_amax, 4 * sizeof(unsigned int));
     if (e != cudaSuccess) { rc = fail(DFT3D_ERR_ALLOC, "cudaMalloc(amax): %s", cudaGetErrorString(e)); break; }
-    if (mode == DFT3D_KDFT) {
+    if (mode == DFT3D_AUTO) {
+      // both formulations in one plan: every pass goes from one cube to another in the natural layout
+      int count = 0;
+      for (int a = 0; a < 3 && rc == DFT3D_OK; ++a)
+        if ((axes >> a) & 1u) {
+          ++count;
+          rc = amode[a] == DFT3D_FFT ? build_fft_axis(p, a, opt.fft_split[a]) : build_kdft_axis(p, a, nodes[a]);
+        }
+      if (rc != DFT3D_OK) break;
+      p->group_planes = n0;
+      const size_t cube_bytes = size_t(n0) * n1 * n2 * 8;
+      const size_t limit = opt.workspace_limit ? opt.workspace_limit : (size_t(16) << 30);
+      if (count >= 2) {
+        if (opt.flags & DFT3D_DESTROY_INPUT) {
+          p->in_is_ws = true;
+        } else if (cube_bytes > limit) {
+          rc = fail(DFT3D_ERR_UNSUPPORTED, "a plan that mixes the formulations needs a workspace as large as the cube "
+                    "(%zu bytes): raise workspace_limit or pass DFT3D_DESTROY_INPUT", cube_bytes);
+          break;
+        } else {
+          e = cudaMalloc(&p->workspace, cube_bytes);
+          if (e != cudaSuccess) { rc = fail(DFT3D_ERR_ALLOC, "cudaMalloc(workspace %zu bytes): %s", cube_bytes, cudaGetErrorString(e)); break; }
+          p->workspace_bytes = cube_bytes;
+        }
+      }
+    } else if (mode == DFT3D_KDFT) {
       for (int a = 0; a < 3 && rc == DFT3D_OK; ++a)
         if ((axes >> a) & 1u) rc = build_kdft_axis(p, a, nodes[a]);
       if (rc != DFT3D_OK) break;
@@ -957,7 +1005,7 @@ int dft3d_execute_axis(dft3d_plan_t p, int axis, const void* in, void* out, void
   if (axis < 0 || axis > 2) return fail(DFT3D_ERR_INVALID_ARG, "axis must be 0, 1 or 2");
   if (!((p->axes >> axis) & 1u)) return fail(DFT3D_ERR_INVALID_ARG, "axis %d is not among the plan's axes", axis);
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-  if (p->mode == DFT3D_KDFT) {
+  if (p->amode[axis] == DFT3D_KDFT) {
     if ((rc = prepare_scales(p, static_cast<const float*>(in), stream)) != DFT3D_OK) return rc;
     return kdft_axis_pass(p, axis, static_cast<const float*>(in), static_cast<float*>(out), p->n[0], stream, 0);
   }
@@ -971,6 +1019,38 @@ int dft3d_execute(dft3d_plan_t p, const void* in, void* out, void* cuda_stream) 
   const float* fin = static_cast<const float*>(in);
   float* fout = static_cast<float*>(out);
   const unsigned axes = p->axes;
+  if (p->mode == DFT3D_AUTO) {
+    // mixed formulations: axis 0, 1, 2 in turn, natural layout throughout, alternating between the cubes so that the
+    // last pass writes `out` (three passes: in -> out -> workspace -> out; two: in -> workspace -> out)
+    float* ws = p->in_is_ws ? const_cast<float*>(fin) : static_cast<float*>(p->workspace);
+    int remaining = int((axes & 1u) + ((axes >> 1) & 1u) + ((axes >> 2) & 1u));
+    if (p->f16) DFT3D_CUDA(cudaMemsetAsync(p->d_amax, 0, 4 * sizeof(unsigned int), stream));
+    const float* src = fin;
+    int pos = 0;
+    bool have_amax = false;     // whether the word d_amax[pos] holds the largest magnitude of `src`
+    for (int a = 0; a < 3; ++a) {
+      if (!((axes >> a) & 1u)) continue;
+      float* dst = (remaining % 2 == 1) ? fout : ws;
+      if (p->amode[a] == DFT3D_FFT) {
+        if ((rc = fft_axis_pass(p, a, src, dst, stream, pos)) != DFT3D_OK) return rc;
+        have_amax = false;
+      } else {
+        if (p->f16 && !have_amax) {
+          // a KDFT pass with fp16 pieces scales by the largest magnitude of its input, which only a KDFT
+          // predecessor records: measure it
+          dft3d::amax_kernel<<<p->sm_count * 8, 256, 0, stream>>>(reinterpret_cast<const float4*>(src), points(p) / 2,
+                                                                 p->d_amax + pos);
+          DFT3D_CUDA(cudaGetLastError());
+        }
+        if ((rc = kdft_axis_pass(p, a, src, dst, p->n[0], stream, pos)) != DFT3D_OK) return rc;
+        have_amax = true;
+      }
+      src = dst;
+      ++pos;
+      --remaining;
+    }
+    return DFT3D_OK;
+  }
   if (p->mode == DFT3D_KDFT) {
     const long long g = p->group_planes;
     const long long plane_floats = p->n[1] * p->n[2] * 2;
@@ -1059,6 +1139,16 @@ size_t dft3d_plan_workspace_bytes(dft3d_plan_t p) { return p ? p->workspace_byte
 int dft3d_plan_launches(dft3d_plan_t p) {
   if (!p) return 0;
   const int count = int((p->axes & 1u) + ((p->axes >> 1) & 1u) + ((p->axes >> 2) & 1u));
+  if (p->mode == DFT3D_AUTO) {
+    int launches = 0;
+    bool have_amax = false;
+    for (int a = 0; a < 3; ++a) {
+      if (!((p->axes >> a) & 1u)) continue;
+      if (p->amode[a] == DFT3D_FFT) { ++launches; have_amax = false; }
+      else { launches += (p->f16 && !have_amax) ? 2 : 1; have_amax = true; }
+    }
+    return launches;
+  }
   const int pre = (p->f16 && p->mode == DFT3D_KDFT) ? 1 : 0;   // the reduction that finds the largest input magnitude
   if (p->mode == DFT3D_KDFT && p->axes == 7u) return pre + int(1 + 2 * (p->n[0] / p->group_planes));
   if (p->mode == DFT3D_KDFT && p->axes == 6u) return pre + int(2 * (p->n[0] / p->group_planes));

@@ -13,7 +13,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 # DFT3D_LIBRARY overrides the path of the shared library (for trying differently built variants)
 _LIB_PATH = os.environ.get("DFT3D_LIBRARY") or os.path.join(_HERE, "libdft3d.so")
 
-DFT3D_KDFT, DFT3D_FFT = 0, 1
+DFT3D_KDFT, DFT3D_FFT, DFT3D_AUTO = 0, 1, 2
 DFT3D_FORWARD, DFT3D_INVERSE = -1, +1
 DFT3D_NODES_ON_OUTPUT, DFT3D_UNSCALED_INVERSE, DFT3D_SPLIT_FP16, DFT3D_SPLIT_TF32, DFT3D_DESTROY_INPUT = 1, 2, 4, 8, 16
 DFT3D_INVERSE_SOLVE = 32

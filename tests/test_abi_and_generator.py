@@ -52,6 +52,8 @@ def test_argument_validation_needs_no_gpu(dft):
         (dict(n=(64, 64, 101)), 2), (dict(n=(16384, 64, 64)), 2), (dict(n=(256, 256, 100), mode=1), 2),
         (dict(n=(64, 64, 64), nodes=(np.array([np.nan] * 64), None, None)), 1),
         (dict(n=(64, 64, 64), mode=1, nodes=(np.arange(64) / 64.0, None, None)), 2),
+        (dict(n=(64, 64, 64), mode=3), 1),           # 0, 1, 2 (KDFT, FFT, AUTO) are the modes
+        (dict(n=(64, 64, 101), mode=2), 2),          # AUTO falls back to KDFT, which needs even lengths
         (dict(n=(64, 64, 64), flags=4 | 8), 1),      # both operand splits at once
         (dict(n=(64, 64, 66), flags=4), 2),          # fp16 pieces need lengths that are multiples of 4
     ]

@@ -767,3 +767,52 @@ def test_inverse_solve_undoes_the_nonuniform_forward_transform(lib, oracle, spli
     with pytest.raises(lib.Dft3dError) as e:
         lib.Plan(*shape, sign=lib.DFT3D_FORWARD, nodes=nodes, flags=lib.DFT3D_INVERSE_SOLVE)
     assert e.value.status == 1
+
+
+# ------------------------------------------------------------------ DFT3D_AUTO: the formulation chosen per axis
+
+@pytest.mark.parametrize("split", SPLITS)
+def test_auto_mode_mixes_the_formulations(lib, oracle, split):
+    """Axis 0 has a length only the KDFT kernels take (100), axes 1 and 2 lengths the FFT kernels take: one plan,
+    three passes through two cubes, against the oracle.  Then nonuniform nodes on axis 1 of a cube whose other axes
+    are FFT lengths, with the input cube as workspace."""
+    sf = _split_flag(lib, split)
+    shape = (100, 256, 512)
+    x = _inputs().cube(shape, "normal", 105, device="cuda")
+    plan = lib.Plan(*shape, mode=lib.DFT3D_AUTO, flags=sf)
+    assert plan.workspace_bytes == x.numel() * 8
+    assert plan.launches == (4 if split == "fp16" else 3)      # fp16 KDFT first: one reduction over the input
+    y = plan(x)
+    _finish(plan)
+    plan.destroy()
+    assert oracle.rel_l2(y.cpu().numpy(), oracle.dft3d(x.cpu().numpy())) < SANITY
+    shape = (256, 128, 256)
+    nodes = [None, _inputs().sorted_nodes(shape, 106)[1], None]
+    x = _inputs().cube(shape, "uniform", 107, device="cuda")
+    want = oracle.dft3d(x.cpu().numpy(), nodes=nodes)
+    plan = lib.Plan(*shape, mode=lib.DFT3D_AUTO, nodes=nodes, flags=sf | lib.DFT3D_DESTROY_INPUT)
+    assert plan.workspace_bytes == 0
+    y = plan(x.clone())
+    _finish(plan)
+    plan.destroy()
+    assert oracle.rel_l2(y.cpu().numpy(), want) < SANITY
+
+
+def test_auto_mode_with_one_formulation_uses_its_schedule(lib, oracle):
+    """When every axis resolves to the same formulation the plan is that formulation's plan."""
+    x = _inputs().cube((256, 256, 256), "normal", 108, device="cuda")
+    auto, fft = lib.Plan(256, 256, 256, mode=lib.DFT3D_AUTO), lib.Plan(256, 256, 256, mode=lib.DFT3D_FFT)
+    a, b = auto(x), fft(x)
+    _finish(auto)
+    fft.status()
+    assert torch.equal(a, b) and auto.launches == 3
+    auto.destroy()
+    fft.destroy()
+    x = _inputs().cube((64, 96, 130), "normal", 109, device="cuda")
+    auto, kd = lib.Plan(64, 96, 130, mode=lib.DFT3D_AUTO), lib.Plan(64, 96, 130, mode=lib.DFT3D_KDFT)
+    a, b = auto(x), kd(x)
+    _finish(auto)
+    kd.status()
+    assert torch.equal(a, b)
+    auto.destroy()
+    kd.destroy()
