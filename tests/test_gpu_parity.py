@@ -816,3 +816,37 @@ def test_auto_mode_with_one_formulation_uses_its_schedule(lib, oracle):
     assert torch.equal(a, b)
     auto.destroy()
     kd.destroy()
+
+
+# ------------------------------------------------------------------ closed forms straight on the CUDA path
+
+@pytest.mark.parametrize("mode_name", ["kdft", "fft"])
+def test_closed_forms_delta_and_constant(lib, mode_name):
+    """Degenerate inputs with textbook spectra, checked without the oracle: a delta at (3, 5, 7) gives the pure
+    phase exp(-2 pi i (3 k0/n0 + 5 k1/n1 + 7 k2/n2)) (Eq. 14 per axis); a constant gives P at the origin and zero
+    elsewhere; the inverse of the delta's spectrum is the delta."""
+    shape = (256, 256, 256)
+    mode = lib.DFT3D_KDFT if mode_name == "kdft" else lib.DFT3D_FFT
+    plan = lib.Plan(*shape, mode=mode)
+    x = torch.zeros(shape, dtype=torch.complex64, device="cuda")
+    x[3, 5, 7] = 1.0
+    y = plan(x)
+    _finish(plan)
+    k = [np.arange(n) for n in shape]
+    ph = [np.exp(-2j * np.pi * s_ * k_ / n) for s_, k_, n in zip((3, 5, 7), k, shape)]
+    want = ph[0][:, None, None] * ph[1][None, :, None] * ph[2][None, None, :]
+    assert np.abs(y.cpu().numpy() - want).max() < 2e-6           # |X| = 1 everywhere
+    inv = lib.Plan(*shape, mode=mode, sign=lib.DFT3D_INVERSE)
+    back = inv(y)
+    _finish(inv)
+    inv.destroy()
+    # (the peak is a fully coherent sum, the worst case for the tensor core's truncating accumulation: ~1e-6 per axis)
+    assert (back - x).abs().max().item() < 6e-6
+    c = torch.full(shape, 0.5 - 0.25j, dtype=torch.complex64, device="cuda")
+    z = plan(c)
+    _finish(plan)
+    plan.destroy()
+    P = float(np.prod(shape))
+    assert abs(z[0, 0, 0].item() - P * (0.5 - 0.25j)) < 1e-5 * P
+    z[0, 0, 0] = 0
+    assert z.abs().max().item() < 1e-5 * P                       # leakage relative to the one peak
