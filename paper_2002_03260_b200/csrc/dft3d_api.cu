@@ -552,7 +552,7 @@ int fft_cols_for(const dft3d_plan_s* p, int axis, int layout) {
   return cols;
 }
 
-int fft_axis_pass(dft3d_plan_s* p, int axis, const float* in, float* out, cudaStream_t stream, int chain_pos,
+int fft_axis_pass(dft3d_plan_s* p, int axis, const float* in, float* out, cudaStream_t stream,
                   int layout = FFT_NATURAL) {
   const FftAxis& ax = p->fax[axis];
   const int R = ax.R, RX = ax.RX, N = int(ax.n), Lg = 128 / (R * RX);
@@ -1009,7 +1009,7 @@ int dft3d_execute_axis(dft3d_plan_t p, int axis, const void* in, void* out, void
     if ((rc = prepare_scales(p, static_cast<const float*>(in), stream)) != DFT3D_OK) return rc;
     return kdft_axis_pass(p, axis, static_cast<const float*>(in), static_cast<float*>(out), p->n[0], stream, 0);
   }
-  return fft_axis_pass(p, axis, static_cast<const float*>(in), static_cast<float*>(out), stream, 0);
+  return fft_axis_pass(p, axis, static_cast<const float*>(in), static_cast<float*>(out), stream);
 }
 
 int dft3d_execute(dft3d_plan_t p, const void* in, void* out, void* cuda_stream) {
@@ -1032,7 +1032,7 @@ int dft3d_execute(dft3d_plan_t p, const void* in, void* out, void* cuda_stream) 
       if (!((axes >> a) & 1u)) continue;
       float* dst = (remaining % 2 == 1) ? fout : ws;
       if (p->amode[a] == DFT3D_FFT) {
-        if ((rc = fft_axis_pass(p, a, src, dst, stream, pos)) != DFT3D_OK) return rc;
+        if ((rc = fft_axis_pass(p, a, src, dst, stream)) != DFT3D_OK) return rc;
         have_amax = false;
       } else {
         if (p->f16 && !have_amax) {
@@ -1092,20 +1092,19 @@ int dft3d_execute(dft3d_plan_t p, const void* in, void* out, void* cuda_stream) 
 #ifdef DFT3D_PROFILE_WAITS
     if (const char* only = getenv("DFT3D_DEBUG_ONLY_PASS")) {   // diagnostic builds: one pass of the schedule alone
       const int k = atoi(only);
-      if (k == 0) return fft_axis_pass(p, 0, fin, fout, stream, 0, FFT_OUT_BLOCKED);
-      if (k == 1) return fft_axis_pass(p, 1, fout, ws, stream, 1, FFT_IN_BLOCKED);
-      return fft_axis_pass(p, 2, ws, fout, stream, 2);
+      if (k == 0) return fft_axis_pass(p, 0, fin, fout, stream, FFT_OUT_BLOCKED);
+      if (k == 1) return fft_axis_pass(p, 1, fout, ws, stream, FFT_IN_BLOCKED);
+      return fft_axis_pass(p, 2, ws, fout, stream);
     }
 #endif
-    if ((rc = fft_axis_pass(p, 0, fin, fout, stream, 0, FFT_OUT_BLOCKED)) != DFT3D_OK) return rc;
-    if ((rc = fft_axis_pass(p, 1, fout, ws, stream, 1, FFT_IN_BLOCKED)) != DFT3D_OK) return rc;
-    return fft_axis_pass(p, 2, ws, fout, stream, 2);
+    if ((rc = fft_axis_pass(p, 0, fin, fout, stream, FFT_OUT_BLOCKED)) != DFT3D_OK) return rc;
+    if ((rc = fft_axis_pass(p, 1, fout, ws, stream, FFT_IN_BLOCKED)) != DFT3D_OK) return rc;
+    return fft_axis_pass(p, 2, ws, fout, stream);
   }
   const float* src = fin;
-  int chain_pos = 0;
   for (int a = 2; a >= 0; --a) {
     if (!((axes >> a) & 1u)) continue;
-    if ((rc = fft_axis_pass(p, a, src, fout, stream, chain_pos++)) != DFT3D_OK) return rc;
+    if ((rc = fft_axis_pass(p, a, src, fout, stream)) != DFT3D_OK) return rc;
     src = fout;
   }
   return DFT3D_OK;

@@ -240,12 +240,15 @@ fft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_c
           ptx::tc_fence_after();
           const uint32_t d = tmem + g * 128;
           const uint32_t a_hi = d + 64, a_lo = a_hi + R;
+          // the small products first: the tensor core truncates when it adds into its accumulator, by up to one
+          // ulp of the accumulator, so the fewer additions happen once the large hi*hi terms are in, the better
 #pragma unroll
           for (int k = 0; k < KS; ++k) {
-            ptx::mma_f16_ts(d, a_hi + k * 8, wh + 2 * k, idesc, k != 0);
-            ptx::mma_f16_ts(d, a_lo + k * 8, wh + 2 * k, idesc, 1);
+            ptx::mma_f16_ts(d, a_lo + k * 8, wh + 2 * k, idesc, k != 0);
             ptx::mma_f16_ts(d, a_hi + k * 8, wl + 2 * k, idesc, 1);
           }
+#pragma unroll
+          for (int k = 0; k < KS; ++k) ptx::mma_f16_ts(d, a_hi + k * 8, wh + 2 * k, idesc, 1);
           ptx::tc_commit(&sh.d1_full[g]);
         }
       }
@@ -268,11 +271,12 @@ fft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_c
           const uint64_t ah = ah0 + ((t & 1) ? kBufStep : 0), al = al0 + ((t & 1) ? kBufStep : 0);
           const uint32_t d = tmem + g * 128 + 64;
 #pragma unroll
-          for (int k = 0; k < KS; ++k) {
-            ptx::mma_f16_ss(d, ah + 2 * k, wh + 2 * k, idesc, k != 0);
-            ptx::mma_f16_ss(d, al + 2 * k, wh + 2 * k, idesc, 1);
+          for (int k = 0; k < KS; ++k) {           // small products first, as in stage 1
+            ptx::mma_f16_ss(d, al + 2 * k, wh + 2 * k, idesc, k != 0);
             ptx::mma_f16_ss(d, ah + 2 * k, wl + 2 * k, idesc, 1);
           }
+#pragma unroll
+          for (int k = 0; k < KS; ++k) ptx::mma_f16_ss(d, ah + 2 * k, wh + 2 * k, idesc, 1);
           ptx::tc_commit(&sh.a2_empty[g]);
           ptx::tc_commit(&sh.d2_full[g]);
         }
