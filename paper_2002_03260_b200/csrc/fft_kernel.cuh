@@ -245,11 +245,12 @@ fft_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_const
             ptx::tc_fence_after();
             const uint32_t a_hi = tmem + kFftTmemA1 + b * 128, a_lo = a_hi + K;
 #pragma unroll
-            for (int k8 = 0; k8 < K / 8; ++k8) {
-              ptx::mma_tf32_ts(tmem + kFftTmemD1, a_hi + k8 * 8, wh[k8], idesc, k8 != 0);
-              ptx::mma_tf32_ts(tmem + kFftTmemD1, a_lo + k8 * 8, wh[k8], idesc, 1);
+            for (int k8 = 0; k8 < K / 8; ++k8) {   // small products first: each addition into the accumulator
+              ptx::mma_tf32_ts(tmem + kFftTmemD1, a_lo + k8 * 8, wh[k8], idesc, k8 != 0);   // truncates to its ulp
               ptx::mma_tf32_ts(tmem + kFftTmemD1, a_hi + k8 * 8, wl[k8], idesc, 1);
             }
+#pragma unroll
+            for (int k8 = 0; k8 < K / 8; ++k8) ptx::mma_tf32_ts(tmem + kFftTmemD1, a_hi + k8 * 8, wh[k8], idesc, 1);
             ptx::tc_commit(&sh.a1_empty[b]);
             ptx::tc_commit(&sh.d1_full);
           }
@@ -280,11 +281,12 @@ fft_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_const
         ptx::tc_fence_after();
         const uint64_t bstep = bi ? kBufStep : 0;
 #pragma unroll
-        for (int k8 = 0; k8 < K / 8; ++k8) {
-          ptx::mma_tf32_ss(tmem + kFftTmemD2, ah[k8] + bstep, wh[k8], idesc, k8 != 0);
-          ptx::mma_tf32_ss(tmem + kFftTmemD2, al[k8] + bstep, wh[k8], idesc, 1);
+        for (int k8 = 0; k8 < K / 8; ++k8) {   // small products first, as in stage 1
+          ptx::mma_tf32_ss(tmem + kFftTmemD2, al[k8] + bstep, wh[k8], idesc, k8 != 0);
           ptx::mma_tf32_ss(tmem + kFftTmemD2, ah[k8] + bstep, wl[k8], idesc, 1);
         }
+#pragma unroll
+        for (int k8 = 0; k8 < K / 8; ++k8) ptx::mma_tf32_ss(tmem + kFftTmemD2, ah[k8] + bstep, wh[k8], idesc, 1);
         ptx::tc_commit(&sh.a2_empty[bi]);
         ptx::tc_commit(&sh.d2_full);
       }
