@@ -63,7 +63,10 @@ def conv_flops(n):
 #   profiles/kdft_f16_axis_kernel_512.md          : mean of the three launches, (1.081 + 1.031) GB / 134.2 M points
 #   (the TF32-piece kernels, captured before: 15.80 and 15.79)
 NCU_DRAM_BYTES_PER_POINT = {"fft_axis_kernel": 15.80, "fft_f16_axis_kernel": 15.97, "kdft_axis_kernel": 15.79,
-                            "kdft_f16_axis_kernel": 15.73}
+                            "kdft_f16_axis_kernel": 15.73,
+                            # profiles/kdft_f16x2_axis_kernel_2048x128x128.md: (1.241 + 0.261) GB / 33.5 M points; the 64 MiB
+                            # table of a 2048-point axis is fetched again by every wave of tiles
+                            "kdft_f16x2_axis_kernel": 44.8}
 
 
 def measured_peaks():
@@ -273,7 +276,9 @@ def main():
             issued = 3.0 * algo_flops
             ach = issued / (ms * 1e-3) * 1e-12
             if split == dft.DFT3D_SPLIT_FP16:
-                kernel, peak = "kdft_f16_axis_kernel", peaks["bf16_tflops_sustained"]
+                paired = max(shape[a] for a in taxes) >= 2048 and os.environ.get("DFT3D_KDFT_PAIR", "1") != "0"
+                kernel = "kdft_f16x2_axis_kernel" if paired else "kdft_f16_axis_kernel"   # CTA pairs from 2048 points up
+                peak = peaks["bf16_tflops_sustained"]
                 src = "%s bf16 sustained (fp16 and bf16 share the tensor rate)" % peak_kind
                 axis_launches = nlaunch - 1
             else:
@@ -282,7 +287,8 @@ def main():
                 axis_launches = nlaunch
             return {"bound": "tensor", "kernel": kernel, "achieved": ach, "peak": peak, "unit": "TFLOP/s",
                     "frac": ach / peak, "traffic": NCU_DRAM_BYTES_PER_POINT[kernel] * P,
-                    "traffic_note": "DRAM bytes per launch, ncu capture at 512^3 scaled by points (algorithmic: 16 B/point)",
+                    "traffic_note": "DRAM bytes per launch, ncu capture at %s scaled by points (algorithmic: 16 B/point)"
+                                    % ("2048x128x128" if kernel == "kdft_f16x2_axis_kernel" else "512^3"),
                     "peak_source": src,
                     "flops": "issued tensor flops = 3 split products x 8*n_a flops per point per axis",
                     "useful_gemm_tflops": algo_flops / (ms * 1e-3) * 1e-12, "avg_launch_ms": ms / axis_launches}
