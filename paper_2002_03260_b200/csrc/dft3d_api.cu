@@ -75,8 +75,8 @@ int encode_map(CUtensorMap* map, CUtensorMapDataType dtype, const void* base, in
   EncodeTiledFn enc;
   int rc = get_encoder(&enc);
   if (rc != DFT3D_OK) return rc;
-  cuuint64_t d[4], s[3];
-  cuuint32_t b[4], es[4];
+  cuuint64_t d[5], s[4];
+  cuuint32_t b[5], es[5];
   for (int i = 0; i < rank; ++i) { d[i] = dims[i]; b[i] = box[i]; es[i] = 1; }
   for (int i = 0; i + 1 < rank; ++i) s[i] = strides_bytes[i];
   CUresult cr = enc(map, dtype, rank, const_cast<void*>(base), d, s, b, es,
@@ -555,6 +555,17 @@ int fft_cols_for(const dft3d_plan_s* p, int axis, int layout) {
   return cols;
 }
 
+// Blocked intermediate, fp16-piece kernel with direct stores: how many neighbouring rows i1 share the 128-byte lines
+// of a block (see FftParams::blk_pair).  1 when the stages are 128 bytes wide anyway, or where the two passes differ.
+int fft_blk_pair(const dft3d_plan_s* p) {
+  if (!p->f16 || getenv("DFT3D_FFT_NO_PAIR")) return 1;
+  if (const char* env = getenv("DFT3D_FFT_STAGE_OUT_BLOCKED")) if (atoi(env)) return 1;
+  const int colsA = fft_cols_for(p, 0, FFT_OUT_BLOCKED), cols1 = fft_cols_for(p, 1, FFT_IN_BLOCKED);
+  if (colsA >= 16 || cols1 != colsA) return 1;
+  const int P = 16 / colsA;
+  return (p->n[1] % P == 0 && 256 % P == 0) ? P : 1;
+}
+
 int fft_axis_pass(dft3d_plan_s* p, int axis, const float* in, float* out, cudaStream_t stream,
                   int layout = FFT_NATURAL) {
   const FftAxis& ax = p->fax[axis];
@@ -568,6 +579,7 @@ int fft_axis_pass(dft3d_plan_s* p, int axis, const float* in, float* out, cudaSt
   fp.profile = p->d_profile;
   fp.out = out;
   fp.status = p->d_status;
+  fp.blk_pair = 1;
   CUtensorMap map_data, map_out;
   int rc;
   int stage_out = 0;
@@ -608,7 +620,20 @@ int fft_axis_pass(dft3d_plan_s* p, int axis, const float* in, float* out, cudaSt
       const unsigned long long bstr[3] = {(unsigned long long)(colsA * 8), (unsigned long long)(n0 * colsA * 8),
                                           (unsigned long long)(n1 * n0 * colsA * 8)};
       const unsigned bbox[4] = {unsigned(2 * cols), 1u, 256u, 1u};
-      rc = encode_f32(&map_data, in, 4, bdims, bstr, bbox, cols * 8);
+      const int P = fft_blk_pair(p);
+      if (P > 1) {
+        // T[n2 tile][i1 / P][k0][i1 % P][cols]: a box takes the P neighbouring rows of one k0 (one 128-byte line) at a time
+        const unsigned long long line = (unsigned long long)(P * colsA * 8);
+        const unsigned long long pdims[5] = {(unsigned long long)(2 * colsA), (unsigned long long)P, (unsigned long long)n0,
+                                             (unsigned long long)(n1 / P), (unsigned long long)(n2 / colsA)};
+        const unsigned long long pstr[4] = {(unsigned long long)(colsA * 8), line, (unsigned long long)n0 * line,
+                                            (unsigned long long)(n1 / P) * n0 * line};
+        const unsigned pbox[5] = {unsigned(2 * cols), unsigned(P), 1u, unsigned(256 / P), 1u};
+        rc = encode_f32(&map_data, in, 5, pdims, pstr, pbox, cols * 8);
+        fp.blk_pair = P;
+      } else {
+        rc = encode_f32(&map_data, in, 4, bdims, bstr, bbox, cols * 8);
+      }
       fp.in_blocked = 1;
       fp.blk_ratio = colsA / cols;
       fp.l2_prefetch = 0;
@@ -620,6 +645,7 @@ int fft_axis_pass(dft3d_plan_s* p, int axis, const float* in, float* out, cudaSt
       const unsigned long long bstr[2] = {(unsigned long long)(cols * 8), (unsigned long long)N * cols * 8ull};
       if (rc == DFT3D_OK) rc = encode_f32(&map_out, out, 3, bdims, bstr, box, cols * 8);
       fp.out_blocked = 1;
+      fp.blk_pair = fft_blk_pair(p);
       fp.blk_tiles = int(p->n[2] / cols);
       fp.blk_rows = int(p->n[1]);
       // TF32 kernel: the stage returns through shared memory and leaves as TMA stores; fp16 kernel: plain stores

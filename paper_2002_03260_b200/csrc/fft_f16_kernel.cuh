@@ -53,6 +53,7 @@ struct FftF16Params {
 
 struct FftF16Shared {
   uint64_t raw_full[4], raw_empty[4], out_ready[4];
+  uint64_t split_done[4];      // STAGE_OUT with tiles that share lines: every tile of the stage has read its input
   uint64_t a1_full[4], d1_full[4], a2_full[4], a2_empty[4], d2_full[4], sc_full[4];
   uint64_t w_full;
   uint32_t tmem_base;
@@ -158,6 +159,7 @@ fft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_c
       ptx::mbar_init(&sh.raw_empty[i], STAGE_OUT ? 1 : 4 * p.mtiles_per_stage);   // the store warp / the split warps
       ptx::mbar_init(&sh.sc_full[i], 4);
       ptx::mbar_init(&sh.out_ready[i], 4 * p.mtiles_per_stage);
+      ptx::mbar_init(&sh.split_done[i], 4 * p.mtiles_per_stage);
       ptx::mbar_init(&sh.a1_full[i], 4);
       ptx::mbar_init(&sh.d1_full[i], 1);
       ptx::mbar_init(&sh.a2_full[i], 4);
@@ -210,7 +212,10 @@ fft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_c
           } else {
             const long long ct = sidx % p.c_tiles, bt = sidx / p.c_tiles;
             for (int r0 = 0; r0 < p.N; r0 += 256) {
-              if (p.in_blocked)
+              if (p.in_blocked && p.blk_pair > 1)
+                ptx::tma_load_5d(dst + size_t(r0) * kRowBytes, &map_data, &sh.raw_full[s], 0, 0, int(bt), r0 / p.blk_pair,
+                                 int(ct));
+              else if (p.in_blocked)
                 ptx::tma_load_4d(dst + size_t(r0) * kRowBytes, &map_data, &sh.raw_full[s],
                                  int(ct % p.blk_ratio) * 2 * COLS, int(bt), r0, int(ct / p.blk_ratio));
               else
@@ -423,6 +428,11 @@ fft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_c
           ptx::fence_proxy_async_smem();
           __syncwarp();
           if (lane == 0) ptx::mbar_arrive(&sh.raw_empty[s]);
+        } else if (kPairTiles) {
+          // the results return into the raw stage, and the RX tiles of a group of lines all read ALL rows of those
+          // lines: none of them may store before the others have read (the tile without twiddles is well ahead)
+          __syncwarp();
+          if (lane == 0) ptx::mbar_arrive(&sh.split_done[s]);
         }
         // the line's largest magnitude over its R lanes (all beta), then 2^(13 - e) and 2^(e - 13) from the exponent
         // field f = e + 127, clamped so that both are normal floats (lines of subnormal-sized data lose nothing:
@@ -509,9 +519,11 @@ fft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_c
           if (p.out_blocked) {
             // block [k][COLS] number n2tile*blk_rows + i1 of the blocked intermediate: pieces of one block are close
             // together, so plain stores from registers do (the L2 merges them into full lines)
-            const long long blk = (ct % p.blk_tiles) * p.blk_rows + ct / p.blk_tiles;
-            dst = reinterpret_cast<float2*>(p.out) + (blk * p.N + (RX * k1 + bsel2)) * COLS + (col0 + g2);
-            k2_stride = (long long)(RX * R) * COLS;
+            // (blk_pair = P > 1: P neighbouring rows i1 interleave their pieces, T[n2 tile][i1 / P][k][i1 % P][COLS])
+            const long long i1 = ct / p.blk_tiles, P = p.blk_pair;
+            const long long blk = (ct % p.blk_tiles) * (p.blk_rows / P) + i1 / P;
+            dst = reinterpret_cast<float2*>(p.out) + ((blk * p.N + (RX * k1 + bsel2)) * P + i1 % P) * COLS + (col0 + g2);
+            k2_stride = (long long)(RX * R) * COLS * P;
           } else {
             dst = reinterpret_cast<float2*>(p.out) + (bt * p.N + (RX * k1 + bsel2)) * p.C + col;
             k2_stride = (long long)(RX * R) * p.C;
@@ -521,6 +533,7 @@ fft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_c
         float om = om1 * inv_scale, om_b = 1.0f;
         if (!(om >= 1.1754944e-38f)) { om = om1; om_b = inv_scale; }
         F16_WAIT_WARP(&sh.d2_full[g], pk, 0x901);
+        if (STAGE_OUT && kPairTiles) F16_WAIT_WARP(&sh.split_done[s], phs, 0x903);
         ptx::tc_fence_after();
         uint32_t v0[K / 32][32];                      // all chunks in flight before the one wait
 #pragma unroll

@@ -69,6 +69,9 @@ struct FftParams {
   int blk_rows;          // out_blocked: n1
   int blk_ratio;         // in_blocked: columns of a block of T / COLS of this pass
   int in_blocked;        // load rows from T through a 4D map {COLS, k0, i1, n2 tile}; batch = k0
+  int blk_pair;          // fp16-piece kernel, stages narrower than 128 bytes: P = 128 / (8*COLS) rows i1 share the lines of
+                         // T, T[n2 tile][i1 / P][k0][i1 % P][COLS], so that the axis-1 pass reads whole 128-byte lines
+                         // (5D map {COLS, i1 % P, k0, i1 / P, n2 tile}); 1 otherwise
   const float2* twiddle; // [R][R] complex64, T[k1][beta] (times 1/RX for a scaled inverse)
   const float2* twiddle2;// RX == 2: [R*R] complex64, exp(s*2*pi*i*m/N)
   float* out;

@@ -26,6 +26,17 @@ def lib():
     return d
 
 
+@pytest.fixture(autouse=True)
+def _release_cached_blocks():
+    """The library allocates its workspaces with cudaMalloc, outside torch's caching allocator: blocks torch keeps
+    cached after a test with large tensors would be missing for the next test's plans (config 5 needs 128 GiB)."""
+    yield
+    if torch.cuda.is_available():
+        import gc
+        gc.collect()
+        torch.cuda.empty_cache()
+
+
 def _inputs():
     from paper_2002_03260_b200 import inputs
     return inputs
@@ -245,12 +256,14 @@ def test_fft_256_forward_inverse_and_kdft_agreement(lib, oracle, split):
 
 
 @pytest.mark.parametrize("split", SPLITS)
-@pytest.mark.parametrize("shape", [(256, 512, 256), (1024, 256, 256), (512, 1024, 256), (256, 4096, 256)])
+@pytest.mark.parametrize("shape", [(256, 512, 256), (1024, 256, 256), (512, 1024, 256), (256, 4096, 256),
+                                   (2048, 2048, 256)])
 def test_fft_schedules_agree(lib, oracle, split, shape):
     """With a cube of workspace the 3D FFT goes in -> out (blocked order) -> workspace -> out; without it the
     three passes run in place on out.  The small shape: both against the oracle.  The longer ones (1024-point strided
     axes, the blocked layout with 16-line and 8-line stages): against each other and against the KDFT kernels, whose
-    single axes are checked against the oracle above."""
+    single axes are checked against the oracle above.  (2048, 2048, 256): both strided passes have 8-line stages, where
+    the fp16 kernel interleaves pairs of rows in the blocked order so that the axis-1 pass reads whole 128-byte lines."""
     sf = _split_flag(lib, split)
     if max(shape) == 4096 and split == "tf32":
         pytest.skip("4096-point axes exist with fp16 pieces only")
@@ -277,6 +290,29 @@ def test_fft_schedules_agree(lib, oracle, split, shape):
         _finish(plan)
         assert oracle.rel_l2(y.cpu().numpy(), ref) < SANITY
         plan.destroy()
+
+
+@pytest.mark.slow
+def test_fft_blocked_order_with_four_rows_per_line(lib):
+    """4096-point strided axes have 4-line stages (32-byte pieces): in the blocked order between the axis-0 and the
+    axis-1 pass four neighbouring rows share each 128-byte line.  Needs 4096 points on axes 0 AND 1, i.e. 32 GiB per
+    cube; compared with the in-place schedule (whose 4096-point passes are checked against the oracle axis by axis)."""
+    free, total = torch.cuda.mem_get_info()
+    if total < 170 * 2 ** 30:
+        pytest.skip("needs a 180 GB device")
+    shape = (4096, 4096, 256)
+    x = _inputs().cube(shape, "normal", 67, device="cuda")
+    with_ws = lib.Plan(*shape, mode=lib.DFT3D_FFT, workspace_limit=40 * 2 ** 30)
+    assert with_ws.workspace_bytes == x.numel() * 8
+    a = with_ws(x)
+    _finish(with_ws)
+    with_ws.destroy()
+    in_place = lib.Plan(*shape, mode=lib.DFT3D_FFT, workspace_limit=1 << 20)
+    assert in_place.workspace_bytes == 0
+    b = in_place(x)
+    _finish(in_place)
+    in_place.destroy()
+    assert _rel_l2_gpu(a, b) < SANITY
 
 
 @pytest.mark.parametrize("split", SPLITS)
