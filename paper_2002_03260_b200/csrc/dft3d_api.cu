@@ -62,16 +62,17 @@ int get_encoder(EncodeTiledFn* fn) {
 // float32 tensor map with up to 4 dimensions; dims/box innermost first; strides in bytes for dims 1..rank-1
 int encode_map(CUtensorMap* map, CUtensorMapDataType dtype, const void* base, int rank,
                const unsigned long long* dims, const unsigned long long* strides_bytes, const unsigned* box,
-               int swizzle_bytes);
+               int swizzle_bytes, int promotion_bytes = -1);
 
 int encode_f32(CUtensorMap* map, const void* base, int rank, const unsigned long long* dims,
-               const unsigned long long* strides_bytes, const unsigned* box, int swizzle_bytes) {
-  return encode_map(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, base, rank, dims, strides_bytes, box, swizzle_bytes);
+               const unsigned long long* strides_bytes, const unsigned* box, int swizzle_bytes, int promotion_bytes = -1) {
+  return encode_map(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, base, rank, dims, strides_bytes, box, swizzle_bytes,
+                    promotion_bytes);
 }
 
 int encode_map(CUtensorMap* map, CUtensorMapDataType dtype, const void* base, int rank,
                const unsigned long long* dims, const unsigned long long* strides_bytes, const unsigned* box,
-               int swizzle_bytes) {
+               int swizzle_bytes, int promotion_bytes) {
   EncodeTiledFn enc;
   int rc = get_encoder(&enc);
   if (rc != DFT3D_OK) return rc;
@@ -79,11 +80,23 @@ int encode_map(CUtensorMap* map, CUtensorMapDataType dtype, const void* base, in
   cuuint32_t b[5], es[5];
   for (int i = 0; i < rank; ++i) { d[i] = dims[i]; b[i] = box[i]; es[i] = 1; }
   for (int i = 0; i + 1 < rank; ++i) s[i] = strides_bytes[i];
+  // L2 promotion: what a miss fetches around the requested bytes.  Rows of 128 bytes and more: 256 bytes (the
+  // neighbouring line belongs to the neighbouring stage, which runs at the same time).  Narrower rows: see below.
+  const unsigned inner_bytes = box[0] * (dtype == CU_TENSOR_MAP_DATA_TYPE_FLOAT32 ? 4u : 2u);
+  CUtensorMapL2promotion promo = CU_TENSOR_MAP_L2_PROMOTION_L2_256B;
+  if (inner_bytes < 128 || promotion_bytes >= 0) {
+    int v = 256;
+    if (const char* env = getenv("DFT3D_TMA_PROMO_NARROW")) v = atoi(env);
+    if (promotion_bytes >= 0) v = promotion_bytes;
+    promo = v == 0 ? CU_TENSOR_MAP_L2_PROMOTION_NONE
+                   : (v == 64 ? CU_TENSOR_MAP_L2_PROMOTION_L2_64B
+                              : (v == 128 ? CU_TENSOR_MAP_L2_PROMOTION_L2_128B : CU_TENSOR_MAP_L2_PROMOTION_L2_256B));
+  }
   CUresult cr = enc(map, dtype, rank, const_cast<void*>(base), d, s, b, es,
                     CU_TENSOR_MAP_INTERLEAVE_NONE,
                     swizzle_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
                                          : (swizzle_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_NONE),
-                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                    promo, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (cr != CUDA_SUCCESS)
     return fail(DFT3D_ERR_CUDA, "cuTensorMapEncodeTiled failed with %d (rank %d, dims %llu %llu %llu, box %u %u %u)",
                 int(cr), rank, dims[0], rank > 1 ? dims[1] : 0ull, rank > 2 ? dims[2] : 0ull, box[0],
@@ -629,7 +642,8 @@ int fft_axis_pass(dft3d_plan_s* p, int axis, const float* in, float* out, cudaSt
         const unsigned long long pstr[4] = {(unsigned long long)(colsA * 8), line, (unsigned long long)n0 * line,
                                             (unsigned long long)(n1 / P) * n0 * line};
         const unsigned pbox[5] = {unsigned(2 * cols), unsigned(P), 1u, unsigned(256 / P), 1u};
-        rc = encode_f32(&map_data, in, 5, pdims, pstr, pbox, cols * 8);
+        const char* penv = getenv("DFT3D_TMA_PROMO_PAIR");
+        rc = encode_f32(&map_data, in, 5, pdims, pstr, pbox, cols * 8, penv ? atoi(penv) : 128);
         fp.blk_pair = P;
       } else {
         rc = encode_f32(&map_data, in, 4, bdims, bstr, bbox, cols * 8);
