@@ -138,6 +138,20 @@ int dft3d_execute(dft3d_plan_t plan, const void* in, void* out, void* cuda_strea
  */
 int dft3d_execute_host(dft3d_plan_t plan, const void* host_in, void* host_out, void* cuda_stream);
 
+/*
+ * A sequence of `count` transforms of HOST cubes, streamed: host_in[i] / host_out[i] are HOST pointers to cubes of
+ * the plan's shape (pinned memory, or the copies cannot overlap anything).  Two plan-owned pairs of device buffers
+ * take turns, the uploads and the downloads run on two plan-owned streams, the transforms on `cuda_stream`: the
+ * download of cube i and the upload of cube i+1 use the two directions of the link at the same time, under the
+ * transform of whichever cube is on the device.  Results are the same as `count` calls of dft3d_execute_host (same
+ * kernels, same order per cube).  The same host buffer may appear several times in host_out (later results
+ * overwrite earlier ones, in order); a host_in buffer must not be one of the host_out buffers.  Synchronous:
+ * returns after the last download; status as dft3d_execute_host.  The extra device buffers and the streams are
+ * created on first use and kept until the plan is destroyed.  count == 0 is a no-op.
+ */
+int dft3d_execute_host_batch(dft3d_plan_t plan, const void* const* host_in, void* const* host_out, int count,
+                             void* cuda_stream);
+
 /* Transform one axis only (0, 1 or 2) with the plan's matrix for that axis; same pointer rules as
  * dft3d_execute.  KDFT: Eq. 5's left / right multiplication for that axis.  FFT: Eq. 17 along that axis. */
 int dft3d_execute_axis(dft3d_plan_t plan, int axis, const void* in, void* out, void* cuda_stream);

@@ -148,6 +148,11 @@ struct dft3d_plan_s {
   long long* d_profile = nullptr;   // wait-cycle counters, only allocated in DFT3D_PROFILE_WAITS builds
   void* host_in_dev = nullptr;  // device staging for dft3d_execute_host
   void* host_out_dev = nullptr;
+  // dft3d_execute_host_batch: a second pair of staging buffers, two copy streams and the events that order them
+  void* host_in_dev2 = nullptr;
+  void* host_out_dev2 = nullptr;
+  cudaStream_t copy_in = nullptr, copy_out = nullptr;
+  cudaEvent_t ev_in_ready[2] = {nullptr, nullptr}, ev_done[2] = {nullptr, nullptr}, ev_out_free[2] = {nullptr, nullptr};
   bool attrs_set = false;
 };
 
@@ -1171,6 +1176,60 @@ int dft3d_execute_host(dft3d_plan_t p, const void* host_in, void* host_out, void
   return dft3d_plan_status(p);
 }
 
+int dft3d_execute_host_batch(dft3d_plan_t p, const void* const* host_in, void* const* host_out, int count,
+                             void* cuda_stream) {
+  if (!p) return fail(DFT3D_ERR_INVALID_ARG, "plan is NULL");
+  if (count < 0 || (count > 0 && (!host_in || !host_out))) return fail(DFT3D_ERR_INVALID_ARG, "host_in/host_out/count");
+  for (int i = 0; i < count; ++i)
+    if (!host_in[i] || !host_out[i]) return fail(DFT3D_ERR_INVALID_ARG, "host_in[%d]/host_out[%d] must not be NULL", i, i);
+  if (count == 0) return DFT3D_OK;
+  const size_t bytes = size_t(points(p)) * 8;
+  if (!p->host_in_dev) DFT3D_CUDA(cudaMalloc(&p->host_in_dev, bytes));
+  if (!p->host_out_dev) DFT3D_CUDA(cudaMalloc(&p->host_out_dev, bytes));
+  if (count > 1) {
+    if (!p->host_in_dev2) DFT3D_CUDA(cudaMalloc(&p->host_in_dev2, bytes));
+    if (!p->host_out_dev2) DFT3D_CUDA(cudaMalloc(&p->host_out_dev2, bytes));
+  }
+  if (!p->copy_in) DFT3D_CUDA(cudaStreamCreateWithFlags(&p->copy_in, cudaStreamNonBlocking));
+  if (!p->copy_out) DFT3D_CUDA(cudaStreamCreateWithFlags(&p->copy_out, cudaStreamNonBlocking));
+  for (int b = 0; b < 2; ++b) {
+    if (!p->ev_in_ready[b]) DFT3D_CUDA(cudaEventCreateWithFlags(&p->ev_in_ready[b], cudaEventDisableTiming));
+    if (!p->ev_done[b]) DFT3D_CUDA(cudaEventCreateWithFlags(&p->ev_done[b], cudaEventDisableTiming));
+    if (!p->ev_out_free[b]) DFT3D_CUDA(cudaEventCreateWithFlags(&p->ev_out_free[b], cudaEventDisableTiming));
+  }
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  void* din[2] = {p->host_in_dev, p->host_in_dev2};
+  void* dout[2] = {p->host_out_dev, p->host_out_dev2};
+  // the copy streams start after whatever the caller's stream holds so far
+  DFT3D_CUDA(cudaEventRecord(p->ev_done[0], stream));
+  DFT3D_CUDA(cudaStreamWaitEvent(p->copy_in, p->ev_done[0], 0));
+  DFT3D_CUDA(cudaStreamWaitEvent(p->copy_out, p->ev_done[0], 0));
+  int rc = DFT3D_OK;
+  for (int i = 0; i < count; ++i) {
+    const int b = i & 1;
+    // item i uses buffer pair b; its upload may start once item i-2 has been transformed out of in[b] ...
+    if (i >= 2) DFT3D_CUDA(cudaStreamWaitEvent(p->copy_in, p->ev_done[b], 0));
+    DFT3D_CUDA(cudaMemcpyAsync(din[b], host_in[i], bytes, cudaMemcpyHostToDevice, p->copy_in));
+    DFT3D_CUDA(cudaEventRecord(p->ev_in_ready[b], p->copy_in));
+    // ... its transform once the upload is there and item i-2's result has left out[b] ...
+    DFT3D_CUDA(cudaStreamWaitEvent(stream, p->ev_in_ready[b], 0));
+    if (i >= 2) DFT3D_CUDA(cudaStreamWaitEvent(stream, p->ev_out_free[b], 0));
+    rc = dft3d_execute(p, din[b], dout[b], cuda_stream);
+    if (rc != DFT3D_OK) break;
+    DFT3D_CUDA(cudaEventRecord(p->ev_done[b], stream));
+    // ... and its download once the transform is done (downloads run in order on their own stream)
+    DFT3D_CUDA(cudaStreamWaitEvent(p->copy_out, p->ev_done[b], 0));
+    DFT3D_CUDA(cudaMemcpyAsync(host_out[i], dout[b], bytes, cudaMemcpyDeviceToHost, p->copy_out));
+    DFT3D_CUDA(cudaEventRecord(p->ev_out_free[b], p->copy_out));
+  }
+  // everything is done when the last download is: hand that back to the caller's stream, then wait for it
+  DFT3D_CUDA(cudaStreamSynchronize(p->copy_in));
+  DFT3D_CUDA(cudaStreamSynchronize(p->copy_out));
+  DFT3D_CUDA(cudaStreamSynchronize(stream));
+  if (rc != DFT3D_OK) return rc;
+  return dft3d_plan_status(p);
+}
+
 int dft3d_plan_status(dft3d_plan_t p) {
   if (!p) return fail(DFT3D_ERR_INVALID_ARG, "plan is NULL");
   unsigned int word = 0;
@@ -1219,6 +1278,15 @@ int dft3d_plan_destroy(dft3d_plan_t p) {
   if (p->d_profile) cudaFree(p->d_profile);
   if (p->host_in_dev) cudaFree(p->host_in_dev);
   if (p->host_out_dev) cudaFree(p->host_out_dev);
+  if (p->host_in_dev2) cudaFree(p->host_in_dev2);
+  if (p->host_out_dev2) cudaFree(p->host_out_dev2);
+  for (int b = 0; b < 2; ++b) {
+    if (p->ev_in_ready[b]) cudaEventDestroy(p->ev_in_ready[b]);
+    if (p->ev_done[b]) cudaEventDestroy(p->ev_done[b]);
+    if (p->ev_out_free[b]) cudaEventDestroy(p->ev_out_free[b]);
+  }
+  if (p->copy_in) cudaStreamDestroy(p->copy_in);
+  if (p->copy_out) cudaStreamDestroy(p->copy_out);
   delete p;
   return DFT3D_OK;
 }

@@ -19,7 +19,8 @@ DFT3D_NODES_ON_OUTPUT, DFT3D_UNSCALED_INVERSE, DFT3D_SPLIT_FP16, DFT3D_SPLIT_TF3
 DFT3D_INVERSE_SOLVE = 32
 
 EXPORTS = [
-    "dft3d_plan_create", "dft3d_plan_create_ex", "dft3d_execute", "dft3d_execute_host", "dft3d_execute_axis",
+    "dft3d_plan_create", "dft3d_plan_create_ex", "dft3d_execute", "dft3d_execute_host", "dft3d_execute_host_batch",
+    "dft3d_execute_axis",
     "dft3d_plan_status", "dft3d_plan_workspace_bytes", "dft3d_plan_launches", "dft3d_plan_split", "dft3d_plan_destroy",
     "dft3d_status_string", "dft3d_last_error", "dft3d_generate_axis_matrix", "dft3d_generate_twiddle", "dft3d_generate_inverse_matrix",
     "dft3d_generate_real_table", "dft3d_kdft_execute_static",
@@ -53,6 +54,7 @@ def _load():
     lib.dft3d_plan_create_ex.argtypes = [ctypes.POINTER(vp), ll, ll, ll, ci, ci, vp, vp, vp, ctypes.POINTER(_Options)]
     lib.dft3d_execute.argtypes = [vp, vp, vp, vp]
     lib.dft3d_execute_host.argtypes = [vp, vp, vp, vp]
+    lib.dft3d_execute_host_batch.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(vp), ci, vp]
     lib.dft3d_execute_axis.argtypes = [vp, ci, vp, vp, vp]
     lib.dft3d_plan_status.argtypes = [vp]
     lib.dft3d_plan_workspace_bytes.argtypes = [vp]
@@ -205,6 +207,19 @@ class Plan:
             return a.data_ptr() if hasattr(a, "data_ptr") else a.ctypes.data
         _check(_lib.dft3d_execute_host(self._h, ptr(x_host), ptr(out_host), _stream_ptr(stream)))
         return out_host
+
+    def execute_host_batch(self, xs_host, outs_host, stream=None):
+        """A sequence of host cubes, streamed: the download of one result overlaps the upload of the next input.
+        xs_host/outs_host: equally long lists of complex64 CPU tensors or numpy arrays (pinned, or nothing overlaps)."""
+        def ptr(a):
+            return a.data_ptr() if hasattr(a, "data_ptr") else a.ctypes.data
+        if len(xs_host) != len(outs_host):
+            raise ValueError("xs_host and outs_host must have the same length")
+        n = len(xs_host)
+        ins = (ctypes.c_void_p * max(n, 1))(*[ptr(a) for a in xs_host])
+        outs = (ctypes.c_void_p * max(n, 1))(*[ptr(a) for a in outs_host])
+        _check(_lib.dft3d_execute_host_batch(self._h, ins, outs, n, _stream_ptr(stream)))
+        return outs_host
 
     def status(self):
         """Raises Dft3dError if a kernel of an earlier execute abandoned a wait; call after synchronising."""

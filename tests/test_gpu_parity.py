@@ -315,6 +315,35 @@ def test_fft_blocked_order_with_four_rows_per_line(lib):
     assert _rel_l2_gpu(a, b) < SANITY
 
 
+def test_execute_host_batch_matches_single_calls(lib, oracle):
+    """The streamed host entry point (two device buffer pairs, uploads and downloads on their own streams) gives,
+    cube by cube, the bits of dft3d_execute_host; five cubes so that both buffer pairs are reused; one against the
+    oracle.  A plan that uses its input buffer as workspace must not lose an upload to the previous transform."""
+    shape = (64, 128, 256)
+    xs = [_inputs().cube(shape, "normal", 300 + i, device="cpu").pin_memory() for i in range(5)]
+    for flags in (0, lib.DFT3D_DESTROY_INPUT):
+        plan = lib.Plan(*shape, mode=lib.DFT3D_KDFT, flags=flags)
+        want = []
+        for x in xs:
+            y = torch.empty_like(x).pin_memory()
+            plan.execute_host(x, y)
+            want.append(y)
+        got = [torch.empty_like(x).pin_memory() for x in xs]
+        plan.execute_host_batch(xs, got)
+        for w, g in zip(want, got):
+            assert torch.equal(w, g)
+        plan.execute_host_batch([], [])
+        one = [torch.empty_like(xs[0]).pin_memory()]
+        plan.execute_host_batch(xs[:1], one)
+        assert torch.equal(one[0], want[0])
+        plan.destroy()
+    assert oracle.rel_l2(got[3].numpy(), oracle.dft3d(xs[3].numpy())) < SANITY
+    plan = lib.Plan(*shape, mode=lib.DFT3D_KDFT)
+    with pytest.raises(ValueError):
+        plan.execute_host_batch(xs, got[:2])
+    plan.destroy()
+
+
 @pytest.mark.parametrize("split", SPLITS)
 def test_fft_mixed_axis_lengths(lib, oracle, split):
     shape = (256, 1024, 256)
