@@ -579,8 +579,10 @@ int fft_blk_pair(const dft3d_plan_s* p) {
   if (!p->f16 || getenv("DFT3D_FFT_NO_PAIR")) return 1;
   if (const char* env = getenv("DFT3D_FFT_STAGE_OUT_BLOCKED")) if (atoi(env)) return 1;
   const int colsA = fft_cols_for(p, 0, FFT_OUT_BLOCKED), cols1 = fft_cols_for(p, 1, FFT_IN_BLOCKED);
-  if (colsA >= 16 || cols1 != colsA) return 1;
-  const int P = 16 / colsA;
+  if (cols1 != colsA) return 1;
+  int P = 16 / colsA;
+  if (const char* env = getenv("DFT3D_FFT_PAIR")) P = atoi(env);
+  if (P <= 1) return 1;
   return (p->n[1] % P == 0 && 256 % P == 0) ? P : 1;
 }
 

@@ -106,6 +106,11 @@ __device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
   asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
   return r;
 }
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+  uint64_t r;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
 __device__ __forceinline__ uint64_t sub2(uint64_t a, uint64_t b) {
   uint64_t r;
   asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
@@ -261,6 +266,7 @@ fft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_c
       // ---------------------------------------------------------- MMA issuer, stage 2: D2[g] = A2[t & 1] (shared memory) x W
       if (lane == 0) {
         const uint32_t idesc = ptx::make_idesc_f16(128, NB);
+        const uint32_t idesc_wide = ptx::make_idesc_f16(128, 2 * NB);
         const uint32_t w_addr = ptx::smem_u32(smem_w);
         const uint32_t a2_addr = ptx::smem_u32(smem_a2);
         const uint64_t wh = ptx::make_kmajor_sw128_desc(w_addr);
@@ -274,14 +280,17 @@ fft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_c
           F16_WAIT(&sh.a2_full[g], pk, 0x604);
           ptx::tc_fence_after();
           const uint64_t ah = ah0 + ((t & 1) ? kBufStep : 0), al = al0 + ((t & 1) ? kBufStep : 0);
-          const uint32_t d = tmem + g * 128 + 64;
+          // The lo piece of the table follows the hi piece row by row in shared memory, so [W_hi | W_lo] is one
+          // operand of 2*NB rows: hi x [W_hi | W_lo] is ONE MMA of N = 2*NB (the data operand is read once, not
+          // twice), and the hi*hi sums (columns 0..NB-1) stay apart from the small products (columns NB..2NB-1, where
+          // lo x W_hi is added), which the store adds in round-to-nearest fp32.  D2 takes the group's whole tensor
+          // memory: D1 has been drained, A1 consumed.
+          const uint32_t d = tmem + g * 128;
 #pragma unroll
-          for (int k = 0; k < KS; ++k) {           // small products first, as in stage 1
-            ptx::mma_f16_ss(d, al + 2 * k, wh + 2 * k, idesc, k != 0);
-            ptx::mma_f16_ss(d, ah + 2 * k, wl + 2 * k, idesc, 1);
+          for (int k = 0; k < KS; ++k) {
+            ptx::mma_f16_ss(d, ah + 2 * k, wh + 2 * k, idesc_wide, k != 0);
+            ptx::mma_f16_ss(d + NB, al + 2 * k, wh + 2 * k, idesc, 1);
           }
-#pragma unroll
-          for (int k = 0; k < KS; ++k) ptx::mma_f16_ss(d, ah + 2 * k, wh + 2 * k, idesc, 1);
           ptx::tc_commit(&sh.a2_empty[g]);
           ptx::tc_commit(&sh.d2_full[g]);
         }
@@ -332,7 +341,7 @@ fft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_c
     const int g2 = kPairTiles ? sl2 : sl2 / RX;
     const int bsel2_fixed = sl2 % RX;
     const uint32_t tm_d1 = tmem + (uint32_t(q * 32) << 16) + g * 128;
-    const uint32_t tm_a1 = tm_d1 + 64;          // A1 (hi | lo), later D2
+    const uint32_t tm_a1 = tm_d1 + 64;          // A1 (hi | lo); D2 takes the whole 128 columns
     // A2 row (= stage-2 lane) of (sub-line, k1): CONTIG line*RX*R + RX*k1 + b ; STRIDED k1*SL + sl.
     // K position (beta, re/im) = halves 2*beta, 2*beta+1 of the row: 16-byte chunk beta/4 (XORed with row % 8 by the
     // 128-byte swizzle), word beta%4.  row % 8 takes kSwzPer different values as k1 runs: offsets for each of them.
@@ -535,17 +544,19 @@ fft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_c
         F16_WAIT_WARP(&sh.d2_full[g], pk, 0x901);
         if (STAGE_OUT && kPairTiles) F16_WAIT_WARP(&sh.split_done[s], phs, 0x903);
         ptx::tc_fence_after();
-        uint32_t v0[K / 32][32];                      // all chunks in flight before the one wait
-#pragma unroll
-        for (int ch = 0; ch < K / 32; ++ch) ptx::tmem_ld_32x32(tm_a1 + ch * 32, v0[ch]);
-        ptx::tc_wait_ld();
         const uint64_t om2 = pack2(om, om);
 #pragma unroll
         for (int ch = 0; ch < K / 32; ++ch) {
+          uint32_t va[32], vb[32];                    // hi*hi sums and the small products of the same outputs
+          ptx::tmem_ld_32x32(tm_d1 + ch * 32, va);
+          ptx::tmem_ld_32x32(tm_d1 + NB + ch * 32, vb);
+          ptx::tc_wait_ld();
           float f[32];
 #pragma unroll
           for (int j = 0; j < 16; ++j)
-            unpack2(mul2(pack2(__uint_as_float(v0[ch][2 * j]), __uint_as_float(v0[ch][2 * j + 1])), om2), f[2 * j], f[2 * j + 1]);
+            unpack2(mul2(add2(pack2(__uint_as_float(va[2 * j]), __uint_as_float(va[2 * j + 1])),
+                              pack2(__uint_as_float(vb[2 * j]), __uint_as_float(vb[2 * j + 1]))), om2),
+                    f[2 * j], f[2 * j + 1]);
           if (om_b != 1.0f) {
 #pragma unroll
             for (int j = 0; j < 32; ++j) f[j] *= om_b;
