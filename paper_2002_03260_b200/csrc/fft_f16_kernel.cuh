@@ -71,6 +71,10 @@ __host__ __device__ constexpr size_t fft16_smem_bytes(int R, int RX) {   // RX =
          kFft16RawBytes + 1024 + 1024;
 }
 
+#ifndef FFT16_REGS_WG0
+#define FFT16_REGS_WG0 64
+#define FFT16_REGS_WORK 104
+#endif
 #define F16_WAIT(bar, parity, code)                                 \
   {                                                                 \
     FFT_PROF_BEGIN                                                  \
@@ -199,7 +203,7 @@ fft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_c
   // warp-group-wide instruction (one call site per group, executed by all four of its warps), and an increase can
   // only take what decreases of the same CTA released: 64 + 4 x 104 = 5 x 96.
   if (warp < 4) {
-    ptx::setmaxnreg_dec<64>();
+    ptx::setmaxnreg_dec<FFT16_REGS_WG0>();
     if (warp == 0) {
       // ---------------------------------------------------------- TMA producer
       if (lane == 0) {
@@ -321,7 +325,7 @@ fft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_c
     }
   } else {
     // ------------------------------------------------------------ worker groups: every fourth M-tile, start to end
-    ptx::setmaxnreg_inc<104>();
+    ptx::setmaxnreg_inc<FFT16_REGS_WORK>();
     const int g = (warp - 4) >> 2;              // group = tile number mod 4
     const int q = warp & 3;                     // lane quarter of tensor memory this warp may touch
     const int m = q * 32 + lane;
