@@ -60,10 +60,10 @@ def conv_flops(n):
 # DRAM bytes per point per launch (dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture divided by the
 # points of that launch; smaller cases than the bench workload, traffic grows in proportion to the points):
 #   profiles/fft_f16_axis_kernel_1024_dram.md     : the bench workload itself (one-pass capture of the three launches
-#                                                   at 1024^3), 51.79 GB / 3 launches / 1073.7 M points
+#                                                   at 1024^3), 51.68 GB / 3 launches / 1073.7 M points
 #   profiles/kdft_f16_axis_kernel_512.md          : mean of the three launches, (1.081 + 1.031) GB / 134.2 M points
 #   (the TF32-piece kernels, captured before: 15.80 and 15.79)
-NCU_DRAM_BYTES_PER_POINT = {"fft_axis_kernel": 15.80, "fft_f16_axis_kernel": 16.08, "kdft_axis_kernel": 15.79,
+NCU_DRAM_BYTES_PER_POINT = {"fft_axis_kernel": 15.80, "fft_f16_axis_kernel": 16.04, "kdft_axis_kernel": 15.79,
                             "kdft_f16_axis_kernel": 15.73,
                             # profiles/kdft_f16x2_axis_kernel_2048x128x128.md: (1.241 + 0.261) GB / 33.5 M points; the 64 MiB
                             # table of a 2048-point axis is fetched again by every wave of tiles
