@@ -124,7 +124,9 @@ int dft3d_plan_create_ex(dft3d_plan_t* out, long long n0, long long n1, long lon
  *   cuda_stream  a cudaStream_t (NULL = default stream).
  *
  * Asynchronous: kernels are enqueued on the stream and the call returns without
- * synchronising.  No allocation happens here.  One execute per plan may be in flight.
+ * synchronising.  No allocation happens here, and nothing is read back from the device, so the
+ * call may be captured into a CUDA graph and replayed on new data in the same buffers.
+ * One execute per plan may be in flight.
  * After the stream has been synchronised, dft3d_plan_status() tells whether any kernel
  * abandoned a bounded wait.
  */

@@ -315,6 +315,38 @@ def test_fft_blocked_order_with_four_rows_per_line(lib):
     assert _rel_l2_gpu(a, b) < SANITY
 
 
+@pytest.mark.parametrize("mode", ["kdft", "fft"])
+def test_execute_is_capturable_in_a_cuda_graph(lib, mode):
+    """dft3d_execute only enqueues work on the stream (no allocation, no synchronisation, no host-side reads of device
+    state), so a transform can be captured into a CUDA graph and replayed on new data in the same buffers."""
+    shape = (64, 128, 256) if mode == "kdft" else (256, 256, 256)
+    plan = lib.Plan(*shape, mode=lib.DFT3D_KDFT if mode == "kdft" else lib.DFT3D_FFT)
+    x = _inputs().cube(shape, "normal", 410, device="cuda")
+    y = torch.empty_like(x)
+    plan(x, y)                      # eager, also the warm-up
+    _finish(plan)
+    want = y.clone()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    y.zero_()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            plan.execute(x, y, stream=side)
+    graph.replay()
+    _finish(plan)
+    assert torch.equal(y, want)
+    x2 = _inputs().cube(shape, "normal", 411, device="cuda")
+    x.copy_(x2)
+    graph.replay()
+    _finish(plan)
+    got = y.clone()
+    plan(x2, y)
+    _finish(plan)
+    assert torch.equal(got, y)
+    plan.destroy()
+
+
 def test_execute_host_batch_matches_single_calls(lib, oracle):
     """The streamed host entry point (two device buffer pairs, uploads and downloads on their own streams) gives,
     cube by cube, the bits of dft3d_execute_host; five cubes so that both buffer pairs are reused; one against the
