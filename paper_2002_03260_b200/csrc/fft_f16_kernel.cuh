@@ -42,6 +42,7 @@
 #pragma once
 #include <cuda_fp16.h>
 #include "fft_kernel.cuh"
+#include "split_f16.cuh"
 
 namespace dft3d {
 
@@ -95,43 +96,6 @@ __host__ __device__ constexpr size_t fft16_smem_bytes(int R, int RX) {   // RX =
     }                                                                                     \
     FFT_PROF_END(code)                                                                    \
   }
-
-// Two fp32 values in one 64-bit register for the packed fp32 instructions of sm_100 (one issue slot for two results).
-__device__ __forceinline__ uint64_t pack2(float a, float b) {
-  uint64_t r;
-  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
-  return r;
-}
-__device__ __forceinline__ void unpack2(uint64_t v, float& a, float& b) {
-  asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v));
-}
-__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
-  uint64_t r;
-  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
-  return r;
-}
-__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
-  uint64_t r;
-  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
-  return r;
-}
-__device__ __forceinline__ uint64_t sub2(uint64_t a, uint64_t b) {
-  uint64_t r;
-  asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
-  return r;
-}
-
-// (re, im) -> packed fp16 pairs: hi = the value rounded to fp16, lo = the exact remainder x - hi rounded to fp16.
-__device__ __forceinline__ void split_half2(uint64_t x, uint32_t& hi, uint32_t& lo) {
-  float re, im, lr, li;
-  unpack2(x, re, im);
-  const __half2 h = __floats2half2_rn(re, im);
-  const float2 hf = __half22float2(h);
-  unpack2(sub2(x, pack2(hf.x, hf.y)), lr, li);
-  const __half2 l = __floats2half2_rn(lr, li);
-  hi = *reinterpret_cast<const uint32_t*>(&h);
-  lo = *reinterpret_cast<const uint32_t*>(&l);
-}
 
 template <int MODE, int R, int RX, int COLS, int STAGE_OUT>
 __global__ void __launch_bounds__(kFftThreads, 1)

@@ -283,6 +283,7 @@ kdft_f16x2_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __gri
     const uint32_t lane_addr = tmem + (uint32_t(q * 32) << 16);
     int strided_off = 0;                    // float2 index of (j = 0) for this lane in a STRIDED stage
     if (MODE == KDFT_STRIDED) strided_off = (m / p.lpb) * (kF16BlockK / 2) * p.lpb + (m % p.lpb);
+    const uint64_t scale2 = pack2(in_scale, in_scale);
     uint32_t ia = 0, it = 0;
     for (long long tp = pair0; tp < total_pairs; tp += pair_step) {
       for (int kb = 0; kb < num_kb; ++kb) {
@@ -316,14 +317,8 @@ kdft_f16x2_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __gri
             if (lane == 0) ptx::mbar_arrive(&sh.a_empty[sa]);
           }
 #pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            const float s0 = __uint_as_float(x[2 * i]) * in_scale, s1 = __uint_as_float(x[2 * i + 1]) * in_scale;
-            const __half2 hi2 = __floats2half2_rn(s0, s1);          // element 2i in the low half
-            const float2 hf = __half22float2(hi2);
-            const __half2 lo2 = __floats2half2_rn(s0 - hf.x, s1 - hf.y);
-            ph[h * 16 + i] = *reinterpret_cast<const uint32_t*>(&hi2);
-            pl[h * 16 + i] = *reinterpret_cast<const uint32_t*>(&lo2);
-          }
+          for (int i = 0; i < 16; ++i)   // element 2i in the low half of each fp16 pair; packed fp32 instructions
+            split_half2(mul2(pack2_bits(x[2 * i], x[2 * i + 1]), scale2), ph[h * 16 + i], pl[h * 16 + i]);
         }
         DFT3D_WAIT_WARP(&sh.t_empty[st], pht ^ 1, 0x302);
         ptx::tc_fence_after();
