@@ -233,6 +233,10 @@ def main():
 
     plan, ms_step, clocks = time_mode(mode, args.steps, args.warmup, True)
     launches = plan.launches
+    psplit, pws = plan.split, plan.workspace_bytes
+    if args.no_e2e:
+        plan.destroy()     # its workspace (half a cube at 2048^3) would sit beside the KDFT leg's
+        plan = None
     kdft_info = None
     if mode == "fft" and not args.no_kdft:
         ksteps = max(1, min(args.steps, 3))
@@ -309,12 +313,12 @@ def main():
                     "useful_gemm_tflops": algo_flops / (ms * 1e-3) * 1e-12, "avg_launch_ms": ms / axis_launches}
 
         if mode == "kdft":
-            roofline = kdft_roofline(ms_step, launches, plan.split)
+            roofline = kdft_roofline(ms_step, launches, psplit)
         else:
             # only kernel: fft_axis_kernel, one launch per axis; algorithmic traffic 16 B per point per axis
             algo_bytes = len(taxes) * 16.0 * P
             achieved = algo_bytes / (ms_step * 1e-3) * 1e-9
-            fkernel = "fft_f16_axis_kernel" if plan.split == dft.DFT3D_SPLIT_FP16 else "fft_axis_kernel"
+            fkernel = "fft_f16_axis_kernel" if psplit == dft.DFT3D_SPLIT_FP16 else "fft_axis_kernel"
             roofline = {"bound": "hbm", "kernel": fkernel, "achieved": achieved, "peak": peaks["hbm_gbs"],
                         "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
                         "traffic": NCU_DRAM_BYTES_PER_POINT[fkernel] * P,
@@ -334,16 +338,17 @@ def main():
         line = {"metric": "3D C2C DFT GFLOP/s (5*P*log2P) at %s" % wl,
                 "value": world * conv_flops(shape) / ms_step * 1e-6, "unit": "GFLOP/s", "n_gpus": world,
                 "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
-                "scaling": "weak", "vs_baseline": None, "dtype": "fp16x3" if plan.split == dft.DFT3D_SPLIT_FP16 else "tf32x3", "data": "synthetic",
+                "scaling": "weak", "vs_baseline": None, "dtype": "fp16x3" if psplit == dft.DFT3D_SPLIT_FP16 else "tf32x3", "data": "synthetic",
                 "config": {"workload": "%s forward 3D complex64 DFT %s, re/im iid U(-1,1), seed 1003+rank" % (mode.upper(), wl),
                            "mode": mode, "shape": list(shape), "axes": list(taxes),
                            "l2": "input and output (%.2f GiB each) are larger than L2" % (P * 8 / 2**30),
                            "per_rank": "one independent cube per GPU",
-                           "destroy_input": bool(args.destroy_input)},
+                           "destroy_input": bool(args.destroy_input), "workspace_bytes": pws},
                 "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches * args.steps,
                 "clocks": clocks, "kdft": kdft_info}
         print(json.dumps(line))
-    plan.destroy()
+    if plan is not None:
+        plan.destroy()
     if world > 1:
         dist.destroy_process_group()
 

@@ -133,6 +133,7 @@ struct dft3d_plan_s {
   unsigned flags = 0;
   bool f16 = false;       // fp16 pieces (else TF32 pieces)
   bool in_is_ws = false;  // DFT3D_DESTROY_INPUT: the caller's input buffer serves as the workspace
+  bool half_ws = false;   // FFT, fp16 pieces: the workspace holds half a cube; the strided passes run once per half of axis 2
   int amode[3] = {0, 0, 0};  // DFT3D_AUTO with both formulations in one plan: the formulation of each axis
   unsigned axes = 7;            // bit a: axis a is transformed
   int device = 0;
@@ -586,8 +587,11 @@ int fft_blk_pair(const dft3d_plan_s* p) {
   return (p->n[1] % P == 0 && 256 % P == 0) ? P : 1;
 }
 
+// n2_sub != 0 (fp16-piece kernel, strided axes, blocked layouts only): the pass covers the slice
+// [n2_off, n2_off + n2_sub) of the last axis.  FFT_OUT_BLOCKED: `in` is the full array, `out` receives the blocked
+// order of the slice alone; FFT_IN_BLOCKED: `in` holds that, `out` is the full array (natural order).
 int fft_axis_pass(dft3d_plan_s* p, int axis, const float* in, float* out, cudaStream_t stream,
-                  int layout = FFT_NATURAL) {
+                  int layout = FFT_NATURAL, long long n2_off = 0, long long n2_sub = 0) {
   const FftAxis& ax = p->fax[axis];
   const int R = ax.R, RX = ax.RX, N = int(ax.n), Lg = 128 / (R * RX);
   const int cols = fft_cols_for(p, axis, layout);
@@ -616,25 +620,36 @@ int fft_axis_pass(dft3d_plan_s* p, int axis, const float* in, float* out, cudaSt
     map_out = map_data;   // unused on this axis
   } else {
     const long long batches = (axis == 0) ? 1 : p->n[0];
-    const long long C = (axis == 0) ? p->n[1] * p->n[2] : p->n[2];
+    const long long n2v = n2_sub ? n2_sub : p->n[2];                            // columns of the last axis this pass covers
+    const long long C = (axis == 0) ? p->n[1] * n2v : n2v;                      // columns per batch of this pass
+    const long long Cmap = (axis == 0) ? p->n[1] * p->n[2] : p->n[2];           // columns per batch of the full array
+    if (n2_sub && (!p->f16 || layout == FFT_NATURAL)) return fail(DFT3D_ERR_UNSUPPORTED, "internal: sliced pass");
     fp.C = C;
+    fp.out_pitch = (n2_sub && layout == FFT_IN_BLOCKED) ? Cmap : C;
+    fp.out_off = (n2_sub && layout == FFT_IN_BLOCKED) ? n2_off : 0;
+    if (n2_sub && layout == FFT_OUT_BLOCKED) {
+      fp.col_tiles_row = int(n2_sub / cols);
+      fp.col_pitch = p->n[2];
+      fp.col_off = n2_off;
+    }
     fp.c_tiles = C / cols;
     {
       // prefetching helps while rows are close (axis 1); with rows MiBs apart (axis 0) the pass is bound by the
       // rate of address translations and every extra request costs more than it hides (measured: 10.0 -> 12.2 ms)
       const char* env = getenv("DFT3D_FFT_L2_PREFETCH");
       fp.l2_prefetch = env ? atoi(env) : (C * 8 < (1ll << 20) ? 1 : 0);
+      if (n2_sub) fp.l2_prefetch = 0;
     }
     fp.mtiles_per_stage = cols / Lg;
     fp.stage_bytes = N * cols * 8;
     fp.num_stages = batches * fp.c_tiles;
-    const unsigned long long dims[3] = {(unsigned long long)(2 * C), (unsigned long long)N, (unsigned long long)batches};
-    const unsigned long long strides[2] = {(unsigned long long)(C * 8), (unsigned long long)N * C * 8ull};
+    const unsigned long long dims[3] = {(unsigned long long)(2 * Cmap), (unsigned long long)N, (unsigned long long)batches};
+    const unsigned long long strides[2] = {(unsigned long long)(Cmap * 8), (unsigned long long)N * Cmap * 8ull};
     const unsigned box[3] = {unsigned(2 * cols), 256u, 1u};
     if (layout == FFT_IN_BLOCKED) {
       // `in` = T[n2 tile][i1][k0][colsA] written by the axis-0 pass; this stage is (k0 = batch, n2 tile) and its rows are i1
       const int colsA = fft_cols_for(p, 0, FFT_OUT_BLOCKED);
-      const long long n0 = p->n[0], n1 = p->n[1], n2 = p->n[2];
+      const long long n0 = p->n[0], n1 = p->n[1], n2 = n2v;
       const unsigned long long bdims[4] = {(unsigned long long)(2 * colsA), (unsigned long long)n0,
                                            (unsigned long long)n1, (unsigned long long)(n2 / colsA)};
       const unsigned long long bstr[3] = {(unsigned long long)(colsA * 8), (unsigned long long)(n0 * colsA * 8),
@@ -670,7 +685,7 @@ int fft_axis_pass(dft3d_plan_s* p, int axis, const float* in, float* out, cudaSt
       if (rc == DFT3D_OK) rc = encode_f32(&map_out, out, 3, bdims, bstr, box, cols * 8);
       fp.out_blocked = 1;
       fp.blk_pair = fft_blk_pair(p);
-      fp.blk_tiles = int(p->n[2] / cols);
+      fp.blk_tiles = int(n2v / cols);
       fp.blk_rows = int(p->n[1]);
       // TF32 kernel: the stage returns through shared memory and leaves as TMA stores; fp16 kernel: plain stores
       // from registers (a block is one contiguous region), which frees the raw stage right after the split
@@ -680,8 +695,9 @@ int fft_axis_pass(dft3d_plan_s* p, int axis, const float* in, float* out, cudaSt
       if (rc == DFT3D_OK) rc = encode_f32(&map_out, out, 3, dims, strides, box, cols * 8);
       // rows MiBs apart: send the results out as full rows through TMA stores instead of 32-byte pieces
       const char* env = getenv("DFT3D_FFT_STAGE_OUT");
-      stage_out = env ? atoi(env) : (C * 8 >= (1ll << 20) ? 1 : 0);
+      stage_out = env ? atoi(env) : (Cmap * 8 >= (1ll << 20) ? 1 : 0);
     }
+    if (n2_sub && stage_out) return fail(DFT3D_ERR_UNSUPPORTED, "internal: sliced pass with staged output");
   }
   if (rc != DFT3D_OK) return rc;
   if (p->f16) {
@@ -1033,6 +1049,19 @@ int dft3d_plan_create_ex(dft3d_plan_t* out, long long n0, long long n1, long lon
         e = cudaMalloc(&p->workspace, cube_bytes);
         if (e == cudaSuccess) p->workspace_bytes = cube_bytes;
         else { p->workspace = nullptr; (void)cudaGetLastError(); }   // fall back to the in-place schedule
+      } else if (axes == 7u && nests && p->f16 && !getenv("DFT3D_FFT_NO_HALF")) {
+        // Too large for a whole cube of workspace: half a cube, if that fits (by default up to 32 GiB, which is what
+        // 2048^3 needs and what is left beside its two cubes).  The two strided passes then run once per half of the
+        // last axis through the blocked order in the workspace, writing their half of `out` in natural order, and the
+        // contiguous pass runs in place on `out`.
+        const size_t half_limit = opt.workspace_limit ? opt.workspace_limit : (size_t(32) << 30);
+        const long long sub = n2 / 2;
+        const int c0 = fft_cols_for(p, 0, FFT_OUT_BLOCKED), c1 = fft_cols_for(p, 1, FFT_IN_BLOCKED);
+        if (n2 % 2 == 0 && sub % c0 == 0 && sub % c1 == 0 && cube_bytes / 2 <= half_limit && n2 * 8 < (1ll << 20)) {
+          e = cudaMalloc(&p->workspace, cube_bytes / 2);
+          if (e == cudaSuccess) { p->workspace_bytes = cube_bytes / 2; p->half_ws = true; }
+          else { p->workspace = nullptr; (void)cudaGetLastError(); }
+        }
       }
     }
   } while (0);
@@ -1138,7 +1167,16 @@ int dft3d_execute(dft3d_plan_t p, const void* in, void* out, void* cuda_stream) 
   }
   // FFT: the first transformed axis (last axis first) in -> out, the others in place on out (a CTA loads a group of
   // lines completely into shared memory before it stores any of their results, and groups are disjoint)
-  if (axes == 7u && (p->workspace || p->in_is_ws) && !getenv("DFT3D_FFT_INPLACE")) {
+  if (axes == 7u && p->half_ws && !getenv("DFT3D_FFT_INPLACE")) {
+    float* ws = static_cast<float*>(p->workspace);
+    const long long sub = p->n[2] / 2;
+    for (int h = 0; h < 2; ++h) {
+      if ((rc = fft_axis_pass(p, 0, fin, ws, stream, FFT_OUT_BLOCKED, h * sub, sub)) != DFT3D_OK) return rc;
+      if ((rc = fft_axis_pass(p, 1, ws, fout, stream, FFT_IN_BLOCKED, h * sub, sub)) != DFT3D_OK) return rc;
+    }
+    return fft_axis_pass(p, 2, fout, fout, stream);   // in place: a CTA has its lines in shared memory before it stores them
+  }
+  if (axes == 7u && ((p->workspace && !p->half_ws) || p->in_is_ws) && !getenv("DFT3D_FFT_INPLACE")) {
     // with a cube of workspace: axis 0 in -> out (blocked order: its far-apart rows are only read, never written
     // piecewise), axis 1 out -> workspace (natural order), axis 2 workspace -> out
     float* ws = p->in_is_ws ? const_cast<float*>(fin) : static_cast<float*>(p->workspace);
@@ -1258,6 +1296,7 @@ int dft3d_plan_launches(dft3d_plan_t p) {
   const int pre = (p->f16 && p->mode == DFT3D_KDFT) ? 1 : 0;   // the reduction that finds the largest input magnitude
   if (p->mode == DFT3D_KDFT && p->axes == 7u) return pre + int(1 + 2 * (p->n[0] / p->group_planes));
   if (p->mode == DFT3D_KDFT && p->axes == 6u) return pre + int(2 * (p->n[0] / p->group_planes));
+  if (p->mode == DFT3D_FFT && p->half_ws && !getenv("DFT3D_FFT_INPLACE")) return 5;   // two strided passes per half, one contiguous
   return pre + count;
 }
 

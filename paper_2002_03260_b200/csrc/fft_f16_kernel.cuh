@@ -191,6 +191,10 @@ fft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_c
               else if (p.in_blocked)
                 ptx::tma_load_4d(dst + size_t(r0) * kRowBytes, &map_data, &sh.raw_full[s],
                                  int(ct % p.blk_ratio) * 2 * COLS, int(bt), r0, int(ct / p.blk_ratio));
+              else if (p.col_tiles_row)   // a slice of the last axis: tile ct % tiles of row ct / tiles of the full array
+                ptx::tma_load_3d(dst + size_t(r0) * kRowBytes, &map_data, &sh.raw_full[s],
+                                 int(2 * ((ct / p.col_tiles_row) * p.col_pitch + p.col_off + (ct % p.col_tiles_row) * COLS)),
+                                 r0, int(bt));
               else
                 ptx::tma_load_3d(dst + size_t(r0) * kRowBytes, &map_data, &sh.raw_full[s], int(ct * 2 * COLS), r0, int(bt));
             }
@@ -502,8 +506,8 @@ fft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_c
             dst = reinterpret_cast<float2*>(p.out) + ((blk * p.N + (RX * k1 + bsel2)) * P + i1 % P) * COLS + (col0 + g2);
             k2_stride = (long long)(RX * R) * COLS * P;
           } else {
-            dst = reinterpret_cast<float2*>(p.out) + (bt * p.N + (RX * k1 + bsel2)) * p.C + col;
-            k2_stride = (long long)(RX * R) * p.C;
+            dst = reinterpret_cast<float2*>(p.out) + (bt * p.N + (RX * k1 + bsel2)) * p.out_pitch + p.out_off + col;
+            k2_stride = (long long)(RX * R) * p.out_pitch;
           }
         }
         // one factor when the product of the two is a normal float (always, except for subnormal-sized data)

@@ -69,6 +69,13 @@ struct FftParams {
   int blk_rows;          // out_blocked: n1
   int blk_ratio;         // in_blocked: columns of a block of T / COLS of this pass
   int in_blocked;        // load rows from T through a 4D map {COLS, k0, i1, n2 tile}; batch = k0
+  // fp16-piece kernel: a pass over a slice [n2_off, n2_off + n2_sub) of the last axis (the cube in halves through a
+  // half-cube workspace).  Column tile ct of the slice is tile ct % col_tiles_row of row ct / col_tiles_row:
+  int col_tiles_row;     // 0: the columns of a batch are contiguous (no slice); else n2_sub / COLS
+  long long col_pitch;   // natural input, sliced: columns per row of the full array (n2)
+  long long col_off;     // natural input, sliced: first column of the slice (n2_off)
+  long long out_pitch;   // natural output: columns per output row (C, or n2 when the pass writes a slice of the full array)
+  long long out_off;     // natural output: first column (0, or n2_off)
   int blk_pair;          // fp16-piece kernel, stages narrower than 128 bytes: P = 128 / (8*COLS) rows i1 share the lines of
                          // T, T[n2 tile][i1 / P][k0][i1 % P][COLS], so that the axis-1 pass reads whole 128-byte lines
                          // (5D map {COLS, i1 % P, k0, i1 / P, n2 tile}); 1 otherwise

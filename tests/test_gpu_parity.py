@@ -292,6 +292,31 @@ def test_fft_schedules_agree(lib, oracle, split, shape):
         plan.destroy()
 
 
+@pytest.mark.parametrize("shape", [(256, 256, 512), (2048, 2048, 256), (256, 4096, 256)])
+def test_fft_half_cube_workspace(lib, oracle, shape):
+    """When a whole cube of workspace is too much but half a cube is not, the two strided passes run once per half of
+    the last axis (slice of the natural input -> blocked order in the workspace -> that half of `out` in natural
+    order) and the contiguous pass runs in place on `out`: five launches.  The small shape against the oracle; the
+    others (8-line stages with interleaved rows; 16-line axis-0 blocks read by 4-line axis-1 stages) against the
+    in-place schedule."""
+    x = _inputs().cube(shape, "normal", 68, device="cuda")
+    half_bytes = x.numel() * 8 // 2
+    half = lib.Plan(*shape, mode=lib.DFT3D_FFT, workspace_limit=half_bytes)
+    assert half.workspace_bytes == half_bytes and half.launches == 5
+    a = half(x)
+    _finish(half)
+    half.destroy()
+    if shape == (256, 256, 512):
+        assert oracle.rel_l2(a.cpu().numpy(), oracle.dft3d(x.cpu().numpy())) < SANITY
+        return
+    in_place = lib.Plan(*shape, mode=lib.DFT3D_FFT, workspace_limit=1 << 20)
+    assert in_place.workspace_bytes == 0 and in_place.launches == 3
+    b = in_place(x)
+    _finish(in_place)
+    in_place.destroy()
+    assert _rel_l2_gpu(a, b) < SANITY
+
+
 @pytest.mark.slow
 def test_fft_blocked_order_with_four_rows_per_line(lib):
     """4096-point strided axes have 4-line stages (32-byte pieces): in the blocked order between the axis-0 and the
@@ -503,7 +528,7 @@ def test_config3_fft_1024_vs_kdft_and_oracle_subset(lib, oracle):
 def test_config5_2048_exponentials_both_modes(lib, oracle):
     """Largest single-GPU instance.  Input: 16 unit exponentials (distinct integer frequencies, seeded phases)
     plus N(0, sigma = 1e-3) noise, so the spectrum is 16 peaks of magnitude P over a floor of about sigma*sqrt(2P).
-    Only two 64 GiB tensors fit, so FFT and KDFT run one after the other into the same output and are compared
+    Only two 64 GiB tensors (and half a cube of workspace) fit, so FFT and KDFT run one after the other into the same output and are compared
     on sampled planes; each is compared with the float64 oracle on a product grid of coefficients that contains
     all peaks.  Gate: the norm-wise relative L2 error of the whole output, estimated from the subset by strata.
     A coefficient's error level depends on how many of its three indices coincide with a peak's index on that axis
@@ -547,7 +572,10 @@ def test_config5_2048_exponentials_both_modes(lib, oracle):
     out = torch.empty_like(x)
     kept = None
     for mode in (lib.DFT3D_FFT, lib.DFT3D_KDFT):
-        plan = lib.Plan(*shape, mode=mode, workspace_limit=4 * 2 ** 30)
+        # FFT: the default limit, i.e. half a cube of workspace (32 GiB) beside the two cubes; KDFT: groups of planes
+        plan = lib.Plan(*shape, mode=mode) if mode == lib.DFT3D_FFT else lib.Plan(*shape, mode=mode, workspace_limit=4 * 2 ** 30)
+        if mode == lib.DFT3D_FFT:
+            assert plan.workspace_bytes == x.numel() * 4 and plan.launches == 5
         plan(x, out)
         _finish(plan)
         plan.destroy()
