@@ -73,11 +73,11 @@ typedef struct dft3d_options_s {
   size_t struct_size;     /* sizeof(dft3d_options_t), for forward compatibility */
   unsigned flags;         /* DFT3D_NODES_ON_OUTPUT | DFT3D_UNSCALED_INVERSE | DFT3D_SPLIT_* | DFT3D_DESTROY_INPUT */
   int fft_split[3][2];    /* FFT mode: {N1, N2} per axis with N1*N2 = n_a; {0,0} = default split */
-  size_t workspace_limit; /* upper bound in bytes for the plan-owned workspace; 0 = default (16 GiB; for the FFT's
-                             half-cube form below 32 GiB).  KDFT needs a workspace and shrinks it to groups of
-                             n0-planes.  FFT uses one cube of workspace when it fits (fastest schedule), else half a
-                             cube when that fits (fp16 pieces, even n2: the strided passes run once per half of the
-                             last axis), and otherwise runs in place on `out`. */
+  size_t workspace_limit; /* upper bound in bytes for the plan-owned workspace; 0 = default (16 GiB).  KDFT needs a
+                             workspace and shrinks it to groups of n0-planes.  FFT uses one cube of workspace when it
+                             fits (fewest launches), else a half, a quarter or an eighth of a cube, whichever fits
+                             first (fp16 pieces: the strided passes run once per slice of the last axis), and
+                             otherwise runs in place on `out`. */
   unsigned axes;          /* bit a set = transform axis a; 0 = all three.  6 (axes 1 and 2) is a batch of n0
                              two-dimensional transforms (Eq. 5), 4 a batch of n0*n1 one-dimensional ones (Eq. 2).
                              An axis that is not transformed may have any length >= 1 if it is axis 0. */

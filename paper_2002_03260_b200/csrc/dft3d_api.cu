@@ -133,7 +133,8 @@ struct dft3d_plan_s {
   unsigned flags = 0;
   bool f16 = false;       // fp16 pieces (else TF32 pieces)
   bool in_is_ws = false;  // DFT3D_DESTROY_INPUT: the caller's input buffer serves as the workspace
-  bool half_ws = false;   // FFT, fp16 pieces: the workspace holds half a cube; the strided passes run once per half of axis 2
+  int ws_slices = 0;      // FFT, fp16 pieces: the workspace holds 1/ws_slices of a cube (2, 4 or 8); the strided passes run
+                          // once per slice of axis 2; 0 = not this schedule
   int amode[3] = {0, 0, 0};  // DFT3D_AUTO with both formulations in one plan: the formulation of each axis
   unsigned axes = 7;            // bit a: axis a is transformed
   int device = 0;
@@ -1050,17 +1051,20 @@ int dft3d_plan_create_ex(dft3d_plan_t* out, long long n0, long long n1, long lon
         if (e == cudaSuccess) p->workspace_bytes = cube_bytes;
         else { p->workspace = nullptr; (void)cudaGetLastError(); }   // fall back to the in-place schedule
       } else if (axes == 7u && nests && p->f16 && !getenv("DFT3D_FFT_NO_HALF")) {
-        // Too large for a whole cube of workspace: half a cube, if that fits (by default up to 32 GiB, which is what
-        // 2048^3 needs and what is left beside its two cubes).  The two strided passes then run once per half of the
-        // last axis through the blocked order in the workspace, writing their half of `out` in natural order, and the
-        // contiguous pass runs in place on `out`.
-        const size_t half_limit = opt.workspace_limit ? opt.workspace_limit : (size_t(32) << 30);
-        const long long sub = n2 / 2;
+        // Too large for a whole cube of workspace: a half, a quarter or an eighth of a cube, whichever fits first.
+        // The two strided passes then run once per slice of the last axis through the blocked order in the workspace,
+        // each writing its slice of `out` in natural order, and the contiguous pass runs in place on `out`.
         const int c0 = fft_cols_for(p, 0, FFT_OUT_BLOCKED), c1 = fft_cols_for(p, 1, FFT_IN_BLOCKED);
-        if (n2 % 2 == 0 && sub % c0 == 0 && sub % c1 == 0 && cube_bytes / 2 <= half_limit && n2 * 8 < (1ll << 20)) {
-          e = cudaMalloc(&p->workspace, cube_bytes / 2);
-          if (e == cudaSuccess) { p->workspace_bytes = cube_bytes / 2; p->half_ws = true; }
-          else { p->workspace = nullptr; (void)cudaGetLastError(); }
+        int forced = 0;
+        if (const char* env = getenv("DFT3D_FFT_SLICES")) forced = atoi(env);
+        for (int k = 2; k <= 8 && !p->ws_slices; k *= 2) {
+          const long long sub = n2 / k;
+          if (forced && k != forced) continue;
+          if (n2 % k != 0 || sub % c0 != 0 || sub % c1 != 0 || n2 * 8 >= (1ll << 20)) break;
+          if (cube_bytes / k > limit && !forced) continue;
+          e = cudaMalloc(&p->workspace, cube_bytes / k);
+          if (e == cudaSuccess) { p->workspace_bytes = cube_bytes / k; p->ws_slices = k; }
+          else { p->workspace = nullptr; (void)cudaGetLastError(); break; }
         }
       }
     }
@@ -1167,16 +1171,16 @@ int dft3d_execute(dft3d_plan_t p, const void* in, void* out, void* cuda_stream) 
   }
   // FFT: the first transformed axis (last axis first) in -> out, the others in place on out (a CTA loads a group of
   // lines completely into shared memory before it stores any of their results, and groups are disjoint)
-  if (axes == 7u && p->half_ws && !getenv("DFT3D_FFT_INPLACE")) {
+  if (axes == 7u && p->ws_slices && !getenv("DFT3D_FFT_INPLACE")) {
     float* ws = static_cast<float*>(p->workspace);
-    const long long sub = p->n[2] / 2;
-    for (int h = 0; h < 2; ++h) {
+    const long long sub = p->n[2] / p->ws_slices;
+    for (int h = 0; h < p->ws_slices; ++h) {
       if ((rc = fft_axis_pass(p, 0, fin, ws, stream, FFT_OUT_BLOCKED, h * sub, sub)) != DFT3D_OK) return rc;
       if ((rc = fft_axis_pass(p, 1, ws, fout, stream, FFT_IN_BLOCKED, h * sub, sub)) != DFT3D_OK) return rc;
     }
     return fft_axis_pass(p, 2, fout, fout, stream);   // in place: a CTA has its lines in shared memory before it stores them
   }
-  if (axes == 7u && ((p->workspace && !p->half_ws) || p->in_is_ws) && !getenv("DFT3D_FFT_INPLACE")) {
+  if (axes == 7u && ((p->workspace && !p->ws_slices) || p->in_is_ws) && !getenv("DFT3D_FFT_INPLACE")) {
     // with a cube of workspace: axis 0 in -> out (blocked order: its far-apart rows are only read, never written
     // piecewise), axis 1 out -> workspace (natural order), axis 2 workspace -> out
     float* ws = p->in_is_ws ? const_cast<float*>(fin) : static_cast<float*>(p->workspace);
@@ -1296,7 +1300,8 @@ int dft3d_plan_launches(dft3d_plan_t p) {
   const int pre = (p->f16 && p->mode == DFT3D_KDFT) ? 1 : 0;   // the reduction that finds the largest input magnitude
   if (p->mode == DFT3D_KDFT && p->axes == 7u) return pre + int(1 + 2 * (p->n[0] / p->group_planes));
   if (p->mode == DFT3D_KDFT && p->axes == 6u) return pre + int(2 * (p->n[0] / p->group_planes));
-  if (p->mode == DFT3D_FFT && p->half_ws && !getenv("DFT3D_FFT_INPLACE")) return 5;   // two strided passes per half, one contiguous
+  if (p->mode == DFT3D_FFT && p->ws_slices && !getenv("DFT3D_FFT_INPLACE"))
+    return 2 * p->ws_slices + 1;   // two strided passes per slice, one contiguous
   return pre + count;
 }
 

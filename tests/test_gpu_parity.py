@@ -294,8 +294,8 @@ def test_fft_schedules_agree(lib, oracle, split, shape):
 
 @pytest.mark.parametrize("shape", [(256, 256, 512), (2048, 2048, 256), (256, 4096, 256)])
 def test_fft_half_cube_workspace(lib, oracle, shape):
-    """When a whole cube of workspace is too much but half a cube is not, the two strided passes run once per half of
-    the last axis (slice of the natural input -> blocked order in the workspace -> that half of `out` in natural
+    """When a whole cube of workspace is too much but a half (quarter, eighth) is not, the two strided passes run once
+    per half (quarter, eighth) of the last axis (slice of the natural input -> blocked order in the workspace -> that half of `out` in natural
     order) and the contiguous pass runs in place on `out`: five launches.  The small shape against the oracle; the
     others (8-line stages with interleaved rows; 16-line axis-0 blocks read by 4-line axis-1 stages) against the
     in-place schedule."""
@@ -306,6 +306,15 @@ def test_fft_half_cube_workspace(lib, oracle, shape):
     a = half(x)
     _finish(half)
     half.destroy()
+    # an eighth of a cube: eight slices, seventeen launches, the same result as with two slices up to rounding order
+    # (bit for bit in fact: the slices only regroup independent columns)
+    eighth = lib.Plan(*shape, mode=lib.DFT3D_FFT, workspace_limit=half_bytes // 4)
+    assert eighth.workspace_bytes == half_bytes // 4 and eighth.launches == 17
+    a8 = eighth(x)
+    _finish(eighth)
+    eighth.destroy()
+    assert torch.equal(a, a8)
+    del a8
     if shape == (256, 256, 512):
         assert oracle.rel_l2(a.cpu().numpy(), oracle.dft3d(x.cpu().numpy())) < SANITY
         return
@@ -528,7 +537,7 @@ def test_config3_fft_1024_vs_kdft_and_oracle_subset(lib, oracle):
 def test_config5_2048_exponentials_both_modes(lib, oracle):
     """Largest single-GPU instance.  Input: 16 unit exponentials (distinct integer frequencies, seeded phases)
     plus N(0, sigma = 1e-3) noise, so the spectrum is 16 peaks of magnitude P over a floor of about sigma*sqrt(2P).
-    Only two 64 GiB tensors (and half a cube of workspace) fit, so FFT and KDFT run one after the other into the same output and are compared
+    Only two 64 GiB tensors (and a fraction of a cube of workspace) fit, so FFT and KDFT run one after the other into the same output and are compared
     on sampled planes; each is compared with the float64 oracle on a product grid of coefficients that contains
     all peaks.  Gate: the norm-wise relative L2 error of the whole output, estimated from the subset by strata.
     A coefficient's error level depends on how many of its three indices coincide with a peak's index on that axis
@@ -572,10 +581,11 @@ def test_config5_2048_exponentials_both_modes(lib, oracle):
     out = torch.empty_like(x)
     kept = None
     for mode in (lib.DFT3D_FFT, lib.DFT3D_KDFT):
-        # FFT: the default limit, i.e. half a cube of workspace (32 GiB) beside the two cubes; KDFT: groups of planes
+        # FFT: the default limit (16 GiB), i.e. a quarter of a cube of workspace beside the two cubes and the strided
+        # passes once per quarter of the last axis; KDFT: groups of planes
         plan = lib.Plan(*shape, mode=mode) if mode == lib.DFT3D_FFT else lib.Plan(*shape, mode=mode, workspace_limit=4 * 2 ** 30)
         if mode == lib.DFT3D_FFT:
-            assert plan.workspace_bytes == x.numel() * 4 and plan.launches == 5
+            assert plan.workspace_bytes == x.numel() * 2 and plan.launches == 9
         plan(x, out)
         _finish(plan)
         plan.destroy()
