@@ -167,8 +167,9 @@ int dft3d_plan_status(dft3d_plan_t plan);
 /* Bytes of device workspace the plan owns (0 for NULL). */
 size_t dft3d_plan_workspace_bytes(dft3d_plan_t plan);
 
-/* Number of kernels one dft3d_execute enqueues (0 for NULL).  With fp16 pieces this counts the small reduction
- * that finds the largest input magnitude before the first axis pass. */
+/* Number of kernels one dft3d_execute enqueues (0 for NULL).  KDFT with fp16 pieces: this counts the small
+ * reduction that finds the largest input magnitude before the first axis pass.  FFT: 3 for a 3D transform, or
+ * 2 * slices + 1 when the workspace holds only a half, a quarter or an eighth of a cube. */
 int dft3d_plan_launches(dft3d_plan_t plan);
 
 /* DFT3D_SPLIT_FP16 or DFT3D_SPLIT_TF32: the operand split the plan uses; 0 for NULL. */
