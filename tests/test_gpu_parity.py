@@ -317,6 +317,12 @@ def test_fft_half_cube_workspace(lib, oracle, shape):
     del a8
     if shape == (256, 256, 512):
         assert oracle.rel_l2(a.cpu().numpy(), oracle.dft3d(x.cpu().numpy())) < SANITY
+        inv = lib.Plan(*shape, mode=lib.DFT3D_FFT, sign=lib.DFT3D_INVERSE, workspace_limit=half_bytes // 2)
+        assert inv.launches == 9
+        back = inv(a)
+        _finish(inv)
+        inv.destroy()
+        assert _rel_l2_gpu(back, x) < SANITY
         return
     in_place = lib.Plan(*shape, mode=lib.DFT3D_FFT, workspace_limit=1 << 20)
     assert in_place.workspace_bytes == 0 and in_place.launches == 3
