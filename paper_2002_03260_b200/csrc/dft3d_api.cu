@@ -73,7 +73,7 @@ int encode_f32(CUtensorMap* map, const void* base, int rank, const unsigned long
 int encode_map(CUtensorMap* map, CUtensorMapDataType dtype, const void* base, int rank,
                const unsigned long long* dims, const unsigned long long* strides_bytes, const unsigned* box,
                int swizzle_bytes, int promotion_bytes) {
-  EncodeTiledFn enc;
+  EncodeTiledFn enc = nullptr;
   int rc = get_encoder(&enc);
   if (rc != DFT3D_OK) return rc;
   cuuint64_t d[5], s[4];
