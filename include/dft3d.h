@@ -49,7 +49,8 @@ enum {
                                    evaluation points, integer powers).  Default is M[k,j] = exp(s*2*pi*i * k * node[j])
                                    (nonuniform input samples, integer output frequencies). */
   DFT3D_UNSCALED_INVERSE = 2u,  /* sign=+1 without the 1/n_a factors */
-  /* Operand split of the tensor-core products (the "decompose and accumulate" of Section II-A).  Both use 3
+  /* Operand split of the tensor-core products (Section II-A: float32 accuracy from several reduced-precision
+     pieces whose products are accumulated).  Both use 3
      products of 11-bit pieces with fp32 accumulation and meet the same error bound.  Default: fp16 pieces (KDFT:
      when every transformed n_a % 4 == 0, TF32 pieces otherwise). */
   DFT3D_SPLIT_FP16 = 4u,        /* insist on fp16 pieces (operands scaled by exact powers of two: KDFT from the largest
@@ -61,8 +62,8 @@ enum {
                                    cube as its workspace and allocates none, which keeps the fast schedules available
                                    when input + output fill the memory (2048^3).  Ignored by plans over fewer axes. */
   DFT3D_INVERSE_SOLVE = 32u     /* KDFT, sign = +1, axes with nodes: the true inverse of the nonuniform transform
-                                   (Section III-A: for points that are not roots of unity the inverse "amounts to
-                                   solving the linear system").  The n_a x n_a forward matrix of the nodes is inverted
+                                   (Section III-A: for points that are not roots of unity the inverse is the
+                                   solution of the linear system of Eq. 2).  The n_a x n_a forward matrix of the nodes is inverted
                                    once at plan creation (float64, on the host; n_a <= 2048) and the solve becomes
                                    one more matrix product, so inverse(forward(x)) = x for distinct nodes.  Axes
                                    without nodes use the usual scaled inverse, which is that inverse.  Singular or
@@ -223,9 +224,9 @@ int dft3d_generate_real_table(long long n, int sign, double scale, const double*
  * previous call's contents (the call clears the one word that must start at zero).  Calls that overlap on the
  * same GPU, from any stream or thread, therefore race; run them one after the other.
  * The first call on a device resolves the array's address and sets kernel attributes; make that first call
- * before any stream capture.  The call enqueues its kernels, then waits for the stream and returns
- * DFT3D_ERR_DEVICE_TIMEOUT if a kernel abandoned a wait.  It calls no cudaMalloc, cudaFree or other
- * allocating routine.
+ * before any stream capture.  Every call is synchronous: it enqueues its kernels, copies one status word back,
+ * waits for the stream (cudaStreamSynchronize) and returns DFT3D_ERR_DEVICE_TIMEOUT if a kernel abandoned a wait.
+ * It calls no cudaMalloc, cudaFree or other allocating routine.
  */
 int dft3d_kdft_execute_static(long long n0, long long n1, long long n2, const float* w0, const float* w1,
                               const float* w2, const void* in, void* out, void* cuda_stream,

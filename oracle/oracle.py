@@ -8,7 +8,7 @@ The functions mirror oracle_dft.c one to one; see that file for the passages
 of the paper each of them follows (Eq. 11-14, Eq. 3, Eq. 5).  solve_axis /
 solve3d (the inverse nonuniform transform of Section III-A as a linear solve)
 are written here, with numpy.linalg.solve as the library step.  Every function
-is pinned in tests/test_oracle_pins.py; none is "parity unpinned".
+is pinned in tests/test_oracle_pins.py.
 """
 import ctypes
 import os
@@ -127,8 +127,8 @@ def dft3d(x, sign=-1, scaled_inverse=False, nodes=None, nodes_on_output=False):
 
 def solve_axis(X, axis, nodes, nodes_on_output=False):
     """Inverse nonuniform transform of one axis (Section III-A, below Eq. 3: for sample points that are not the roots
-    of unity the inverse "amounts to solving the linear system"): x with V x = X along `axis`, V the forward matrix
-    of Eq. 3 for these nodes.  numpy.linalg.solve (LAPACK, float64) is the library step."""
+    of unity the inverse is the solution of the linear system of Eq. 2): x with V x = X along `axis`, V the forward
+    matrix of Eq. 3 for these nodes.  numpy.linalg.solve (LAPACK, float64) is the library step."""
     X = np.ascontiguousarray(X, dtype=np.complex128)
     assert X.ndim == 3
     n = X.shape[axis]

@@ -26,7 +26,7 @@
  * k*x_j with the product's rounding error recovered by fma for nodes.
  *
  * Every function here is pinned by tests/test_oracle_pins.py (closed forms,
- * brute force, invariants, library special cases); none is "parity unpinned".
+ * brute force, invariants, library special cases).
  *
  * Layout everywhere: row-major [n0][n1][n2], interleaved complex (re, im).
  */

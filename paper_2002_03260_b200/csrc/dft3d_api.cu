@@ -5,7 +5,10 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <map>
+#include <mutex>
 #include <new>
+#include <tuple>
 #include <vector>
 
 #include <cuda.h>
@@ -46,33 +49,81 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 // The driver entry point is fetched through the runtime so that the library has no link-time
 // dependency on libcuda and can be loaded (for its host-only entry points) on a machine without a GPU.
 int get_encoder(EncodeTiledFn* fn) {
+  static std::once_flag once;
   static EncodeTiledFn cached = nullptr;
-  if (!cached) {
+  static cudaError_t err = cudaSuccess;
+  std::call_once(once, [] {
     void* p = nullptr;
     cudaDriverEntryPointQueryResult qr;
-    cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qr);
-    if (e != cudaSuccess || !p || qr != cudaDriverEntryPointSuccess)
-      return fail(DFT3D_ERR_CUDA, "cuTensorMapEncodeTiled is not available: %s", cudaGetErrorString(e));
-    cached = reinterpret_cast<EncodeTiledFn>(p);
-  }
+    err = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qr);
+    if (err == cudaSuccess && p && qr == cudaDriverEntryPointSuccess) cached = reinterpret_cast<EncodeTiledFn>(p);
+  });
+  if (!cached) return fail(DFT3D_ERR_CUDA, "cuTensorMapEncodeTiled is not available: %s", cudaGetErrorString(err));
   *fn = cached;
   return DFT3D_OK;
 }
 
+// Tuning knobs.  Environment variables are read ONCE, when a plan is created, and the values live in the plan:
+// nothing a later dft3d_execute does depends on the environment.  -1 = not set (the measured default applies).
+struct Knobs {
+  int promo_narrow = -1, promo_pair = -1, promo_blocked = -1;   // L2 promotion of tensor maps (0/64/128/256 bytes)
+  int fft_cols[2] = {-1, -1};                                   // lines per strided FFT stage, axis 0 / axis 1
+  int fft_no_pair = 0, fft_pair = -1;                           // blocked order: rows per 128-byte line
+  int fft_stage_out = -1, fft_stage_out_blocked = -1;           // results leave through the raw stage + TMA stores
+  int fft_l2_prefetch = -1, fft_nb2 = -1;
+  int fft_inplace = 0, fft_no_half = 0, fft_slices = 0;
+  int fft_fuse = -1;                                            // axes 1 and 2 in one launch through an L2-resident ring
+  int kdft_pair = -1, chunk_kb = -1;
+  long long wait_limit = 0;                                     // clock budget of the kernels' bounded waits (0 = default)
+  int test_silent_producer = 0;                                 // test of the give-up path: TMA producers issue nothing
+};
+
+int env_int(const char* name, int unset) {
+  const char* v = getenv(name);
+  return v ? atoi(v) : unset;
+}
+
+Knobs read_knobs() {
+  Knobs k;
+  k.promo_narrow = env_int("DFT3D_TMA_PROMO_NARROW", -1);
+  k.promo_pair = env_int("DFT3D_TMA_PROMO_PAIR", -1);
+  k.promo_blocked = env_int("DFT3D_TMA_PROMO_BLOCKED", -1);
+  const int cols = env_int("DFT3D_FFT_COLS", -1);
+  k.fft_cols[0] = env_int("DFT3D_FFT_COLS0", cols);
+  k.fft_cols[1] = env_int("DFT3D_FFT_COLS1", cols);
+  k.fft_no_pair = getenv("DFT3D_FFT_NO_PAIR") ? 1 : 0;
+  k.fft_pair = env_int("DFT3D_FFT_PAIR", -1);
+  k.fft_stage_out = env_int("DFT3D_FFT_STAGE_OUT", -1);
+  k.fft_stage_out_blocked = env_int("DFT3D_FFT_STAGE_OUT_BLOCKED", -1);
+  k.fft_l2_prefetch = env_int("DFT3D_FFT_L2_PREFETCH", -1);
+  k.fft_nb2 = env_int("DFT3D_FFT_NB2", -1);
+  k.fft_inplace = getenv("DFT3D_FFT_INPLACE") ? 1 : 0;
+  k.fft_no_half = getenv("DFT3D_FFT_NO_HALF") ? 1 : 0;
+  k.fft_slices = env_int("DFT3D_FFT_SLICES", 0);
+  k.fft_fuse = env_int("DFT3D_FFT_FUSE", -1);
+  k.kdft_pair = env_int("DFT3D_KDFT_PAIR", -1);
+  k.chunk_kb = env_int("DFT3D_CHUNK_KB", -1);
+  if (const char* v = getenv("DFT3D_WAIT_LIMIT_CLOCKS")) k.wait_limit = atoll(v);
+  k.test_silent_producer = env_int("DFT3D_TEST_SILENT_PRODUCER", 0);
+  return k;
+}
+
 // float32 tensor map with up to 4 dimensions; dims/box innermost first; strides in bytes for dims 1..rank-1
+// promotion_bytes >= 0 fixes the L2 promotion; otherwise 256 bytes, or `narrow_promo` (if >= 0) for rows under 128 bytes
 int encode_map(CUtensorMap* map, CUtensorMapDataType dtype, const void* base, int rank,
                const unsigned long long* dims, const unsigned long long* strides_bytes, const unsigned* box,
-               int swizzle_bytes, int promotion_bytes = -1);
+               int swizzle_bytes, int promotion_bytes = -1, int narrow_promo = -1);
 
 int encode_f32(CUtensorMap* map, const void* base, int rank, const unsigned long long* dims,
-               const unsigned long long* strides_bytes, const unsigned* box, int swizzle_bytes, int promotion_bytes = -1) {
+               const unsigned long long* strides_bytes, const unsigned* box, int swizzle_bytes, int promotion_bytes = -1,
+               int narrow_promo = -1) {
   return encode_map(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, base, rank, dims, strides_bytes, box, swizzle_bytes,
-                    promotion_bytes);
+                    promotion_bytes, narrow_promo);
 }
 
 int encode_map(CUtensorMap* map, CUtensorMapDataType dtype, const void* base, int rank,
                const unsigned long long* dims, const unsigned long long* strides_bytes, const unsigned* box,
-               int swizzle_bytes, int promotion_bytes) {
+               int swizzle_bytes, int promotion_bytes, int narrow_promo) {
   EncodeTiledFn enc = nullptr;
   int rc = get_encoder(&enc);
   if (rc != DFT3D_OK) return rc;
@@ -85,8 +136,7 @@ int encode_map(CUtensorMap* map, CUtensorMapDataType dtype, const void* base, in
   const unsigned inner_bytes = box[0] * (dtype == CU_TENSOR_MAP_DATA_TYPE_FLOAT32 ? 4u : 2u);
   CUtensorMapL2promotion promo = CU_TENSOR_MAP_L2_PROMOTION_L2_256B;
   if (inner_bytes < 128 || promotion_bytes >= 0) {
-    int v = 256;
-    if (const char* env = getenv("DFT3D_TMA_PROMO_NARROW")) v = atoi(env);
+    int v = narrow_promo >= 0 ? narrow_promo : 256;
     if (promotion_bytes >= 0) v = promotion_bytes;
     promo = v == 0 ? CU_TENSOR_MAP_L2_PROMOTION_NONE
                    : (v == 64 ? CU_TENSOR_MAP_L2_PROMOTION_L2_64B
@@ -156,15 +206,42 @@ struct dft3d_plan_s {
   cudaStream_t copy_in = nullptr, copy_out = nullptr;
   cudaEvent_t ev_in_ready[2] = {nullptr, nullptr}, ev_done[2] = {nullptr, nullptr}, ev_out_free[2] = {nullptr, nullptr};
   bool attrs_set = false;
+  Knobs knobs;                  // environment knobs as they were when the plan was created
+  // Tensor maps of the data operands, encoded once per (pass, base pointer, slice) and reused by later executes on the
+  // same buffers (a plan serves one execute at a time, so no lock)
+  typedef std::tuple<int, const void*, long long, long long> MapKey;
+  std::map<MapKey, CUtensorMap> map_cache;
 };
 
 namespace {
 
 long long points(const dft3d_plan_s* p) { return p->n[0] * p->n[1] * p->n[2]; }
 
+// Looks up the tensor map of (tag, base, x0, x1) in the plan's cache; `make` encodes it on a miss.
+template <class Make>
+int cached_map(dft3d_plan_s* p, CUtensorMap* map, int tag, const void* base, long long x0, long long x1, Make&& make) {
+  const dft3d_plan_s::MapKey key(tag, base, x0, x1);
+  auto it = p->map_cache.find(key);
+  if (it != p->map_cache.end()) { *map = it->second; return DFT3D_OK; }
+  const int rc = make(map);
+  if (rc != DFT3D_OK) return rc;
+  if (p->map_cache.size() >= 8192) p->map_cache.clear();   // a caller that keeps changing buffers: start over
+  try { p->map_cache.emplace(key, *map); } catch (const std::bad_alloc&) { /* uncached is still correct */ }
+  return DFT3D_OK;
+}
+
+dft3d::WaitControl wait_control(const dft3d_plan_s* p) {
+  dft3d::WaitControl wc;
+  wc.limit_clocks = p->knobs.wait_limit;
+  wc.silent_producer = p->knobs.test_silent_producer;
+  return wc;
+}
+
 // the opt-in to large dynamic shared memory is a per-device property of each kernel
 int set_kernel_attributes(int device) {
+  static std::mutex mu;
   static bool done_on[64] = {false};
+  std::lock_guard<std::mutex> lock(mu);
   bool& done = done_on[device & 63];
   if (done) return DFT3D_OK;
   DFT3D_CUDA(cudaFuncSetAttribute(dft3d::kdft_axis_kernel<dft3d::KDFT_CONTIG>,
@@ -289,12 +366,12 @@ int build_kdft_axis(dft3d_plan_s* p, int a, const double* nodes) {
     const unsigned hbox[3] = {unsigned(dft3d::kF16BlockK), unsigned(ax.bn), 2u};
     {
       // pairs of CTAs (cta_group::2) share a 256-column table tile, each loading 128 of its rows
-      const char* env = getenv("DFT3D_KDFT_PAIR");
+      const int env = p->knobs.kdft_pair;
       // Same bits as the one-CTA kernel.  Its MMAs run at full rate but every chain end waits for a cross-CTA round
       // trip, which cancels out at n = 1024 (77.6 vs 78.5 ms); at n = 2048, where the 64 MiB table no longer sits in
       // L2 beside the data and the part runs at its 1 kW cap, fetching every table tile once per CTA pair wins
       // (1365 -> 1235 ms, 1305 -> 1522 MHz).  Default: pairs from n = 2048 on.
-      ax.pair = ax.bn == 256 && (p->sm_count % 2 == 0) && (env ? atoi(env) != 0 : n >= 2048);
+      ax.pair = ax.bn == 256 && (p->sm_count % 2 == 0) && (env >= 0 ? env != 0 : n >= 2048);
       if (ax.pair) {
         const unsigned pbox[3] = {unsigned(dft3d::kF16BlockK), 128u, 2u};
         int rc = encode_map(&ax.map_w_pair, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, ax.d_w, 3, hdims, hstrides, pbox, 128);
@@ -323,6 +400,7 @@ void fill_f16_params(Params& fp, const dft3d::KdftParams& kp, const KdftAxis& ax
   fp.out_mul = ax.out_mul;
   fp.amax_in = p->d_amax + chain_pos;
   fp.amax_out = p->d_amax + chain_pos + 1;
+  fp.wc = kp.wc;
 }
 
 // chain_pos: position of this pass in the sequence of passes of one execute (fp16 pieces: which amax word to read)
@@ -346,12 +424,15 @@ int launch_kdft_strided(dft3d_plan_s* p, int a, const float* in, float* out, lon
   kp.out = out;
   kp.status = p->d_status;
   kp.profile = p->d_profile;
+  kp.wc = wait_control(p);
   CUtensorMap map_data;
-  const unsigned long long dims[3] = {(unsigned long long)(2 * C), (unsigned long long)J, (unsigned long long)batches};
-  const unsigned long long strides[2] = {(unsigned long long)(C * 8), (unsigned long long)(J * C * 8)};
   const bool f16 = p->f16;
-  const unsigned box[3] = {unsigned(2 * kp.lpb), unsigned((f16 ? dft3d::kF16BlockK : dft3d::kBlockK) / 2), unsigned(kp.bpt)};
-  int rc = encode_f32(&map_data, in, 3, dims, strides, box, 0);
+  int rc = cached_map(p, &map_data, 0x100 + a, in, batches, C, [&](CUtensorMap* m) {
+    const unsigned long long dims[3] = {(unsigned long long)(2 * C), (unsigned long long)J, (unsigned long long)batches};
+    const unsigned long long strides[2] = {(unsigned long long)(C * 8), (unsigned long long)(J * C * 8)};
+    const unsigned box[3] = {unsigned(2 * kp.lpb), unsigned((f16 ? dft3d::kF16BlockK : dft3d::kBlockK) / 2), unsigned(kp.bpt)};
+    return encode_f32(m, in, 3, dims, strides, box, 0, -1, p->knobs.promo_narrow);
+  });
   if (rc != DFT3D_OK) return rc;
   const long long total = kp.m_tiles * kp.n_tiles;
   const int grid = int(total < p->sm_count ? total : p->sm_count);
@@ -392,11 +473,14 @@ int launch_kdft_contig(dft3d_plan_s* p, int a, const float* in, float* out, long
   kp.out = out;
   kp.status = p->d_status;
   kp.profile = p->d_profile;
+  kp.wc = wait_control(p);
   CUtensorMap map_data;
-  const unsigned long long dims[2] = {(unsigned long long)(2 * J), (unsigned long long)rows};
-  const unsigned long long strides[1] = {(unsigned long long)(J * 8)};
-  const unsigned box[2] = {unsigned(dft3d::kBlockK), unsigned(dft3d::kTileM)};
-  int rc = encode_f32(&map_data, in, 2, dims, strides, box, 128);
+  int rc = cached_map(p, &map_data, 0x110 + a, in, rows, 0, [&](CUtensorMap* m) {
+    const unsigned long long dims[2] = {(unsigned long long)(2 * J), (unsigned long long)rows};
+    const unsigned long long strides[1] = {(unsigned long long)(J * 8)};
+    const unsigned box[2] = {unsigned(dft3d::kBlockK), unsigned(dft3d::kTileM)};
+    return encode_f32(m, in, 2, dims, strides, box, 128);
+  });
   if (rc != DFT3D_OK) return rc;
   const long long total = kp.m_tiles * kp.n_tiles;
   const int grid = int(total < p->sm_count ? total : p->sm_count);
@@ -559,17 +643,16 @@ int fft_cols_for(const dft3d_plan_s* p, int axis, int layout) {
     // 1024-point strided axes: 16 lines per stage (128-byte rows) leave room for one stage-2 operand buffer only;
     // 8 lines per stage (64-byte rows) allow two.  Rows far apart (large strides) favour the wider rows.
     const long long C = (axis == 0) ? p->n[1] * p->n[2] : p->n[2];
-    const char* env = getenv(axis == 0 ? "DFT3D_FFT_COLS0" : "DFT3D_FFT_COLS1");
-    if (!env) env = getenv("DFT3D_FFT_COLS");
+    const int env = p->knobs.fft_cols[axis];
     // measured at 1024^3: natural layout, rows >= 1 MiB apart: 16; otherwise (close rows, or the blocked layout
     // where every stage is one contiguous block) 8-line stages, which leave room to load the next stage early
-    cols = env ? atoi(env) : ((layout == FFT_NATURAL && C * 8 >= (1ll << 20)) ? 16 : 8);
+    cols = env >= 0 ? env : ((layout == FFT_NATURAL && C * 8 >= (1ll << 20)) ? 16 : 8);
     // fp16 kernel: always 16 (its raw stage is free again as soon as it has been split, so the second stage matters
     // less than the 128-byte pieces).  Measured at 1024^3: axis 1 in natural order 3.47 ms against 4.1 ms with 8;
     // from the blocked intermediate the same speed within 1 %, but 11 % less DRAM read traffic (no 64-byte halves
     // of lines), and the pass no longer has the slower second equilibrium that small timing changes tipped the
     // two-stage form into (3.6 -> 5.9 ms).
-    if (!env && p->f16) cols = 16;
+    if (env < 0 && p->f16) cols = 16;
     if (cols != 8 && cols != 16) cols = 16;
   }
   return cols;
@@ -578,12 +661,12 @@ int fft_cols_for(const dft3d_plan_s* p, int axis, int layout) {
 // Blocked intermediate, fp16-piece kernel with direct stores: how many neighbouring rows i1 share the 128-byte lines
 // of a block (see FftParams::blk_pair).  1 when the stages are 128 bytes wide anyway, or where the two passes differ.
 int fft_blk_pair(const dft3d_plan_s* p) {
-  if (!p->f16 || getenv("DFT3D_FFT_NO_PAIR")) return 1;
-  if (const char* env = getenv("DFT3D_FFT_STAGE_OUT_BLOCKED")) if (atoi(env)) return 1;
+  if (!p->f16 || p->knobs.fft_no_pair) return 1;
+  if (p->knobs.fft_stage_out_blocked > 0) return 1;
   const int colsA = fft_cols_for(p, 0, FFT_OUT_BLOCKED), cols1 = fft_cols_for(p, 1, FFT_IN_BLOCKED);
   if (cols1 != colsA) return 1;
   int P = 16 / colsA;
-  if (const char* env = getenv("DFT3D_FFT_PAIR")) P = atoi(env);
+  if (p->knobs.fft_pair >= 0) P = p->knobs.fft_pair;
   if (P <= 1) return 1;
   return (p->n[1] % P == 0 && 256 % P == 0) ? P : 1;
 }
@@ -605,19 +688,24 @@ int fft_axis_pass(dft3d_plan_s* p, int axis, const float* in, float* out, cudaSt
   fp.out = out;
   fp.status = p->d_status;
   fp.blk_pair = 1;
+  fp.wc = wait_control(p);
   CUtensorMap map_data, map_out;
   int rc;
   int stage_out = 0;
+  const Knobs& kn = p->knobs;
+  const int tag_in = 0x200 + axis * 8 + layout, tag_out = 0x300 + axis * 8 + layout;
   if (axis == 2) {
     const long long rows = p->n[0] * p->n[1];
     fp.rows = rows;
     fp.mtiles_per_stage = 1;
     fp.stage_bytes = Lg * N * 8;
     fp.num_stages = rows / Lg;
-    const unsigned long long dims[3] = {256ull, (unsigned long long)(N / 128), (unsigned long long)rows};
-    const unsigned long long strides[2] = {1024ull, (unsigned long long)N * 8ull};
-    const unsigned box[3] = {256u, unsigned(N / 128), unsigned(Lg)};
-    rc = encode_f32(&map_data, in, 3, dims, strides, box, 0);
+    rc = cached_map(p, &map_data, tag_in, in, 0, 0, [&](CUtensorMap* m) {
+      const unsigned long long dims[3] = {256ull, (unsigned long long)(N / 128), (unsigned long long)rows};
+      const unsigned long long strides[2] = {1024ull, (unsigned long long)N * 8ull};
+      const unsigned box[3] = {256u, unsigned(N / 128), unsigned(Lg)};
+      return encode_f32(m, in, 3, dims, strides, box, 0);
+    });
     map_out = map_data;   // unused on this axis
   } else {
     const long long batches = (axis == 0) ? 1 : p->n[0];
@@ -637,8 +725,7 @@ int fft_axis_pass(dft3d_plan_s* p, int axis, const float* in, float* out, cudaSt
     {
       // prefetching helps while rows are close (axis 1); with rows MiBs apart (axis 0) the pass is bound by the
       // rate of address translations and every extra request costs more than it hides (measured: 10.0 -> 12.2 ms)
-      const char* env = getenv("DFT3D_FFT_L2_PREFETCH");
-      fp.l2_prefetch = env ? atoi(env) : (C * 8 < (1ll << 20) ? 1 : 0);
+      fp.l2_prefetch = kn.fft_l2_prefetch >= 0 ? kn.fft_l2_prefetch : (C * 8 < (1ll << 20) ? 1 : 0);
       if (n2_sub) fp.l2_prefetch = 0;
     }
     fp.mtiles_per_stage = cols / Lg;
@@ -665,38 +752,47 @@ int fft_axis_pass(dft3d_plan_s* p, int axis, const float* in, float* out, cudaSt
         const unsigned long long pstr[4] = {(unsigned long long)(colsA * 8), line, (unsigned long long)n0 * line,
                                             (unsigned long long)(n1 / P) * n0 * line};
         const unsigned pbox[5] = {unsigned(2 * cols), unsigned(P), 1u, unsigned(256 / P), 1u};
-        const char* penv = getenv("DFT3D_TMA_PROMO_PAIR");
-        rc = encode_f32(&map_data, in, 5, pdims, pstr, pbox, cols * 8, penv ? atoi(penv) : 128);
+        rc = cached_map(p, &map_data, tag_in, in, n2_off, n2_sub, [&](CUtensorMap* m) {
+          return encode_f32(m, in, 5, pdims, pstr, pbox, cols * 8, kn.promo_pair >= 0 ? kn.promo_pair : 128);
+        });
         fp.blk_pair = P;
       } else {
         // rows of whole lines: fetch just them (the line after a row belongs to the next k0, a much later stage;
         // measured at 1024^3: 13 % less DRAM read traffic, same speed)
-        const char* benv = getenv("DFT3D_TMA_PROMO_BLOCKED");
-        rc = encode_f32(&map_data, in, 4, bdims, bstr, bbox, cols * 8, benv ? atoi(benv) : (cols * 8 >= 128 ? 128 : -1));
+        rc = cached_map(p, &map_data, tag_in, in, n2_off, n2_sub, [&](CUtensorMap* m) {
+          return encode_f32(m, in, 4, bdims, bstr, bbox, cols * 8,
+                            kn.promo_blocked >= 0 ? kn.promo_blocked : (cols * 8 >= 128 ? 128 : -1), kn.promo_narrow);
+        });
       }
       fp.in_blocked = 1;
       fp.blk_ratio = colsA / cols;
       fp.l2_prefetch = 0;
     } else {
-      rc = encode_f32(&map_data, in, 3, dims, strides, box, cols * 8);
+      rc = cached_map(p, &map_data, tag_in, in, n2_off, n2_sub, [&](CUtensorMap* m) {
+        return encode_f32(m, in, 3, dims, strides, box, cols * 8, -1, kn.promo_narrow);
+      });
     }
     if (layout == FFT_OUT_BLOCKED) {
       const unsigned long long bdims[3] = {(unsigned long long)(2 * cols), (unsigned long long)N, (unsigned long long)(C / cols)};
       const unsigned long long bstr[2] = {(unsigned long long)(cols * 8), (unsigned long long)N * cols * 8ull};
-      if (rc == DFT3D_OK) rc = encode_f32(&map_out, out, 3, bdims, bstr, box, cols * 8);
+      if (rc == DFT3D_OK)
+        rc = cached_map(p, &map_out, tag_out, out, n2_off, n2_sub, [&](CUtensorMap* m) {
+          return encode_f32(m, out, 3, bdims, bstr, box, cols * 8, -1, kn.promo_narrow);
+        });
       fp.out_blocked = 1;
       fp.blk_pair = fft_blk_pair(p);
       fp.blk_tiles = int(n2v / cols);
       fp.blk_rows = int(p->n[1]);
       // TF32 kernel: the stage returns through shared memory and leaves as TMA stores; fp16 kernel: plain stores
       // from registers (a block is one contiguous region), which frees the raw stage right after the split
-      const char* env = getenv("DFT3D_FFT_STAGE_OUT_BLOCKED");
-      stage_out = env ? atoi(env) : (p->f16 ? 0 : 1);
+      stage_out = kn.fft_stage_out_blocked >= 0 ? kn.fft_stage_out_blocked : (p->f16 ? 0 : 1);
     } else {
-      if (rc == DFT3D_OK) rc = encode_f32(&map_out, out, 3, dims, strides, box, cols * 8);
+      if (rc == DFT3D_OK)
+        rc = cached_map(p, &map_out, tag_out, out, n2_off, n2_sub, [&](CUtensorMap* m) {
+          return encode_f32(m, out, 3, dims, strides, box, cols * 8, -1, kn.promo_narrow);
+        });
       // rows MiBs apart: send the results out as full rows through TMA stores instead of 32-byte pieces
-      const char* env = getenv("DFT3D_FFT_STAGE_OUT");
-      stage_out = env ? atoi(env) : (Cmap * 8 >= (1ll << 20) ? 1 : 0);
+      stage_out = kn.fft_stage_out >= 0 ? kn.fft_stage_out : (Cmap * 8 >= (1ll << 20) ? 1 : 0);
     }
     if (n2_sub && stage_out) return fail(DFT3D_ERR_UNSUPPORTED, "internal: sliced pass with staged output");
   }
@@ -749,8 +845,7 @@ int fft_axis_pass(dft3d_plan_s* p, int axis, const float* in, float* out, cudaSt
   if (axis != 2 && R == 32 && RX == 1 && cols == 8) {
     // 8-line stages: two stage-2 operand buffers and one raw stage (best with direct stores), or one operand
     // buffer and two raw stages (best when the results return through the raw stage, which then stays busy longer)
-    const char* env = getenv("DFT3D_FFT_NB2");
-    nb2 = env ? atoi(env) : (layout != FFT_NATURAL ? 1 : 2);
+    nb2 = kn.fft_nb2 >= 0 ? kn.fft_nb2 : (layout != FFT_NATURAL ? 1 : 2);
     if (nb2 != 1 && nb2 != 2) nb2 = 2;
   }
   fp.raw_stages = dft3d::fft_raw_bytes(R, nb2) / fp.stage_bytes;
@@ -967,10 +1062,8 @@ int dft3d_plan_create_ex(dft3d_plan_t* out, long long n0, long long n1, long lon
       break;
     }
     p->sm_count = prop.multiProcessorCount;
-    if (const char* env = getenv("DFT3D_CHUNK_KB")) {   // tuning knob: stages per accumulation chain
-      const int v = atoi(env);
-      if (v >= 1) p->chunk_kb = v;
-    }
+    p->knobs = read_knobs();
+    if (p->knobs.chunk_kb >= 1) p->chunk_kb = p->knobs.chunk_kb;   // tuning knob: stages per accumulation chain
     if ((rc = set_kernel_attributes(p->device)) != DFT3D_OK) break;
     cudaError_t e = cudaMalloc(&p->d_status, sizeof(unsigned int));
     if (e == cudaSuccess) e = cudaMemset(p->d_status, 0, sizeof(unsigned int));
@@ -995,7 +1088,10 @@ int dft3d_plan_create_ex(dft3d_plan_t* out, long long n0, long long n1, long lon
       const size_t cube_bytes = size_t(n0) * n1 * n2 * 8;
       const size_t limit = opt.workspace_limit ? opt.workspace_limit : (size_t(16) << 30);
       if (count >= 2) {
-        if (opt.flags & DFT3D_DESTROY_INPUT) {
+        // Three passes go in -> out -> workspace -> out, so the input may serve as the workspace once the first pass
+        // has read it.  Two passes go in -> workspace -> out: the first would run in place on the input, which a KDFT
+        // pass cannot (every output tile re-reads whole lines), so two-axis plans allocate their workspace.
+        if ((opt.flags & DFT3D_DESTROY_INPUT) && count == 3) {
           p->in_is_ws = true;
         } else if (cube_bytes > limit) {
           rc = fail(DFT3D_ERR_UNSUPPORTED, "a plan that mixes the formulations needs a workspace as large as the cube "
@@ -1050,13 +1146,12 @@ int dft3d_plan_create_ex(dft3d_plan_t* out, long long n0, long long n1, long lon
         e = cudaMalloc(&p->workspace, cube_bytes);
         if (e == cudaSuccess) p->workspace_bytes = cube_bytes;
         else { p->workspace = nullptr; (void)cudaGetLastError(); }   // fall back to the in-place schedule
-      } else if (axes == 7u && nests && p->f16 && !getenv("DFT3D_FFT_NO_HALF")) {
+      } else if (axes == 7u && nests && p->f16 && !p->knobs.fft_no_half) {
         // Too large for a whole cube of workspace: a half, a quarter or an eighth of a cube, whichever fits first.
         // The two strided passes then run once per slice of the last axis through the blocked order in the workspace,
         // each writing its slice of `out` in natural order, and the contiguous pass runs in place on `out`.
         const int c0 = fft_cols_for(p, 0, FFT_OUT_BLOCKED), c1 = fft_cols_for(p, 1, FFT_IN_BLOCKED);
-        int forced = 0;
-        if (const char* env = getenv("DFT3D_FFT_SLICES")) forced = atoi(env);
+        const int forced = p->knobs.fft_slices;
         for (int k = 2; k <= 8 && !p->ws_slices; k *= 2) {
           const long long sub = n2 / k;
           if (forced && k != forced) continue;
@@ -1171,7 +1266,7 @@ int dft3d_execute(dft3d_plan_t p, const void* in, void* out, void* cuda_stream) 
   }
   // FFT: the first transformed axis (last axis first) in -> out, the others in place on out (a CTA loads a group of
   // lines completely into shared memory before it stores any of their results, and groups are disjoint)
-  if (axes == 7u && p->ws_slices && !getenv("DFT3D_FFT_INPLACE")) {
+  if (axes == 7u && p->ws_slices && !p->knobs.fft_inplace) {
     float* ws = static_cast<float*>(p->workspace);
     const long long sub = p->n[2] / p->ws_slices;
     for (int h = 0; h < p->ws_slices; ++h) {
@@ -1180,7 +1275,7 @@ int dft3d_execute(dft3d_plan_t p, const void* in, void* out, void* cuda_stream) 
     }
     return fft_axis_pass(p, 2, fout, fout, stream);   // in place: a CTA has its lines in shared memory before it stores them
   }
-  if (axes == 7u && ((p->workspace && !p->ws_slices) || p->in_is_ws) && !getenv("DFT3D_FFT_INPLACE")) {
+  if (axes == 7u && ((p->workspace && !p->ws_slices) || p->in_is_ws) && !p->knobs.fft_inplace) {
     // with a cube of workspace: axis 0 in -> out (blocked order: its far-apart rows are only read, never written
     // piecewise), axis 1 out -> workspace (natural order), axis 2 workspace -> out
     float* ws = p->in_is_ws ? const_cast<float*>(fin) : static_cast<float*>(p->workspace);
@@ -1300,7 +1395,7 @@ int dft3d_plan_launches(dft3d_plan_t p) {
   const int pre = (p->f16 && p->mode == DFT3D_KDFT) ? 1 : 0;   // the reduction that finds the largest input magnitude
   if (p->mode == DFT3D_KDFT && p->axes == 7u) return pre + int(1 + 2 * (p->n[0] / p->group_planes));
   if (p->mode == DFT3D_KDFT && p->axes == 6u) return pre + int(2 * (p->n[0] / p->group_planes));
-  if (p->mode == DFT3D_FFT && p->ws_slices && !getenv("DFT3D_FFT_INPLACE"))
+  if (p->mode == DFT3D_FFT && p->ws_slices && !p->knobs.fft_inplace)
     return 2 * p->ws_slices + 1;   // two strided passes per slice, one contiguous
   return pre + count;
 }

@@ -156,6 +156,12 @@ extern "C" int dft3d_kdft_execute_static(long long n0, long long n1, long long n
     if (n0 < 1 || n1 < 1 || n2 < 1) { rc = fail(DFT3D_ERR_INVALID_ARG, "sizes must be >= 1"); break; }
     if (!w0 || !w1 || !w2 || !in || !out) { rc = fail(DFT3D_ERR_INVALID_ARG, "NULL pointer argument"); break; }
     if ((n0 % 64) || (n1 % 64) || (n2 % 64)) { rc = fail(DFT3D_ERR_UNSUPPORTED, "every size must be a multiple of 64"); break; }
+    // bound every factor before forming the product (which could otherwise wrap around)
+    if (n0 > kStaticMaxPoints || n1 > kStaticMaxPoints || n2 > kStaticMaxPoints) {
+      rc = fail(DFT3D_ERR_UNSUPPORTED, "%lld x %lld x %lld points exceed the static scratch of %lld points (16 MiB); use "
+                "dft3d_plan_create for larger transforms", n0, n1, n2, kStaticMaxPoints);
+      break;
+    }
     const long long P = n0 * n1 * n2;
     if (P > kStaticMaxPoints) {
       rc = fail(DFT3D_ERR_UNSUPPORTED, "%lld x %lld x %lld = %lld points exceed the static scratch of %lld points "

@@ -59,6 +59,7 @@ struct FftF16Shared {
   uint64_t w_full;
   uint32_t tmem_base;
   volatile int abort_flag;
+  long long wait_limit;
   float line_scale[4][8];      // per group, 2^(e - 13) of the tile's (sub-)lines, from the split to the store (where a
                                // thread's stage-2 lane belongs to another sub-line than its stage-1 lane)
 };
@@ -79,7 +80,7 @@ __host__ __device__ constexpr size_t fft16_smem_bytes(int R, int RX) {   // RX =
 #define F16_WAIT(bar, parity, code)                                 \
   {                                                                 \
     FFT_PROF_BEGIN                                                  \
-    if (!bounded_wait((bar), (parity), &sh.abort_flag)) {           \
+    if (!bounded_wait((bar), (parity), &sh.abort_flag, sh.wait_limit)) {           \
       sh.abort_flag = 1;                                            \
       atomicCAS(p.status, 0u, (unsigned)(code));                    \
       goto role_done;                                               \
@@ -89,7 +90,7 @@ __host__ __device__ constexpr size_t fft16_smem_bytes(int R, int RX) {   // RX =
 #define F16_WAIT_WARP(bar, parity, code)                                                  \
   {                                                                                       \
     FFT_PROF_BEGIN                                                                        \
-    if (!__all_sync(0xffffffffu, bounded_wait((bar), (parity), &sh.abort_flag) ? 1 : 0)) { \
+    if (!__all_sync(0xffffffffu, bounded_wait((bar), (parity), &sh.abort_flag, sh.wait_limit) ? 1 : 0)) { \
       sh.abort_flag = 1;                                                                  \
       atomicCAS(p.status, 0u, (unsigned)(code));                                          \
       goto role_done;                                                                     \
@@ -141,6 +142,7 @@ fft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_c
     }
     ptx::mbar_init(&sh.w_full, 1);
     sh.abort_flag = 0;
+    sh.wait_limit = p.wc.limit_clocks > 0 ? p.wc.limit_clocks : kDefaultWaitClocks;
     ptx::fence_mbar_init();
   }
   for (int i = tid; i < R * R; i += kFftThreads) smem_tw[i] = __ldg(p.twiddle + i);
@@ -170,7 +172,7 @@ fft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_c
     ptx::setmaxnreg_dec<FFT16_REGS_WG0>();
     if (warp == 0) {
       // ---------------------------------------------------------- TMA producer
-      if (lane == 0) {
+      if (lane == 0 && !p.wc.silent_producer) {
         ptx::mbar_arrive_expect_tx(&sh.w_full, uint32_t(fft16_w_bytes(R)));
         for (int pc = 0; pc < 2; ++pc)                // [piece][2R rows][64 halves]
           ptx::tma_load_2d(smem_w + pc * kWPiece, &map_w, &sh.w_full, 0, pc * NB);

@@ -84,6 +84,7 @@ struct FftParams {
   float* out;
   unsigned int* status;
   long long* profile;    // optional cycle counters (builds with DFT3D_PROFILE_WAITS): [grid][16][8]
+  WaitControl wc;
 };
 
 struct FftShared {
@@ -96,6 +97,7 @@ struct FftShared {
   uint64_t out_ready;      // STAGE_OUT: the four drain-2 warps have written the stage's last M-tile
   uint32_t tmem_base;
   volatile int abort_flag;
+  long long wait_limit;
 };
 
 // shared memory: [W: 2 pieces x 2R/32 panels of 2R rows x 128 B] [A2: hi panels, lo panels] [raw ring] [barriers]
@@ -117,7 +119,7 @@ __host__ __device__ constexpr size_t fft_smem_bytes(int R, int NB2) {
 #define FFT_WAIT(bar, parity, code)                                 \
   {                                                                 \
     FFT_PROF_BEGIN                                                  \
-    if (!bounded_wait((bar), (parity), &sh.abort_flag)) {           \
+    if (!bounded_wait((bar), (parity), &sh.abort_flag, sh.wait_limit)) {           \
       sh.abort_flag = 1;                                            \
       atomicCAS(p.status, 0u, (unsigned)(code));                    \
       goto role_done;                                               \
@@ -127,7 +129,7 @@ __host__ __device__ constexpr size_t fft_smem_bytes(int R, int NB2) {
 #define FFT_WAIT_WARP(bar, parity, code)                                                  \
   {                                                                                       \
     FFT_PROF_BEGIN                                                                        \
-    if (!__all_sync(0xffffffffu, bounded_wait((bar), (parity), &sh.abort_flag) ? 1 : 0)) { \
+    if (!__all_sync(0xffffffffu, bounded_wait((bar), (parity), &sh.abort_flag, sh.wait_limit) ? 1 : 0)) { \
       sh.abort_flag = 1;                                                                  \
       atomicCAS(p.status, 0u, (unsigned)(code));                                          \
       goto role_done;                                                                     \
@@ -174,6 +176,7 @@ fft_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_const
     ptx::mbar_init(&sh.d2_full, 1); ptx::mbar_init(&sh.d2_empty, 4);
     ptx::mbar_init(&sh.w_full, 1);
     sh.abort_flag = 0;
+    sh.wait_limit = p.wc.limit_clocks > 0 ? p.wc.limit_clocks : kDefaultWaitClocks;
     ptx::fence_mbar_init();
   }
   if (warp == 1) {

@@ -35,6 +35,7 @@ struct KdftF16Params {
   float out_mul;                        // 2^-10, times 1/n for a scaled inverse
   const unsigned int* amax_in;          // float bits: largest |input| (an upper bound is enough)
   unsigned int* amax_out;               // float bits: receives the largest |output| (atomic max)
+  WaitControl wc;
 };
 
 struct KdftF16Shared {
@@ -44,6 +45,7 @@ struct KdftF16Shared {
   uint64_t acc_full, acc_empty;
   uint32_t tmem_base;
   volatile int abort_flag;
+  long long wait_limit;
 };
 
 // largest magnitude of a float array (grid-stride, one atomic per warp); `result` must start at zero
@@ -60,7 +62,7 @@ __global__ void amax_kernel(const float4* x, long long n4, unsigned int* result)
 
 // single-thread wait (producer, MMA issuer)
 #define DFT3D_WAIT(bar, parity, code)                               \
-  if (!bounded_wait((bar), (parity), &sh.abort_flag)) {             \
+  if (!bounded_wait((bar), (parity), &sh.abort_flag, sh.wait_limit)) {             \
     sh.abort_flag = 1;                                              \
     atomicCAS(p.status, 0u, (unsigned)(code));                      \
     goto role_done;                                                 \
@@ -68,7 +70,7 @@ __global__ void amax_kernel(const float4* x, long long n4, unsigned int* result)
 // whole-warp wait: the warp leaves together, so the .sync.aligned tensor-memory
 // instructions that follow are never executed by a partial warp
 #define DFT3D_WAIT_WARP(bar, parity, code)                                              \
-  if (!__all_sync(0xffffffffu, bounded_wait((bar), (parity), &sh.abort_flag) ? 1 : 0)) { \
+  if (!__all_sync(0xffffffffu, bounded_wait((bar), (parity), &sh.abort_flag, sh.wait_limit) ? 1 : 0)) { \
     sh.abort_flag = 1;                                                                  \
     atomicCAS(p.status, 0u, (unsigned)(code));                                          \
     goto role_done;                                                                     \
@@ -95,6 +97,7 @@ kdft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_
     ptx::mbar_init(&sh.acc_full, 1);
     ptx::mbar_init(&sh.acc_empty, kEpilogueWarps);
     sh.abort_flag = 0;
+    sh.wait_limit = p.wc.limit_clocks > 0 ? p.wc.limit_clocks : kDefaultWaitClocks;
     ptx::fence_mbar_init();
   }
   if (warp == 1) {
@@ -133,7 +136,7 @@ kdft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_
     ptx::setmaxnreg_dec<DFT3D_REGS_WG0>();
     if (warp == 0) {
       // ------------------------------------------------------------ TMA producer
-      if (lane == 0) {
+      if (lane == 0 && !p.wc.silent_producer) {
         uint32_t ib = 0, ia = 0;   // running stage counters
         for (long long t = blockIdx.x; t < total_tiles; t += gridDim.x) {
           const long long mt = t / p.n_tiles;

@@ -29,6 +29,7 @@ struct KdftX2Shared {
   uint64_t acc_full, acc_empty;
   uint32_t tmem_base;
   volatile int abort_flag;
+  long long wait_limit;
 };
 constexpr size_t kKdftX2SmemBytes = size_t(kX2StagesB) * kX2BytesStageB + size_t(kX2StagesA) * kF16BytesStageA +
                                     sizeof(KdftX2Shared) + 1024;
@@ -91,7 +92,7 @@ __device__ __forceinline__ void tc_commit_pair(uint64_t* bar) {
 
 // single-thread wait (producer, MMA issuer)
 #define DFT3D_WAIT(bar, parity, code)                               \
-  if (!bounded_wait((bar), (parity), &sh.abort_flag)) {             \
+  if (!bounded_wait((bar), (parity), &sh.abort_flag, sh.wait_limit)) {             \
     sh.abort_flag = 1;                                              \
     atomicCAS(p.status, 0u, (unsigned)(code));                      \
     goto role_done;                                                 \
@@ -99,7 +100,7 @@ __device__ __forceinline__ void tc_commit_pair(uint64_t* bar) {
 // whole-warp wait: the warp leaves together, so the .sync.aligned tensor-memory
 // instructions that follow are never executed by a partial warp
 #define DFT3D_WAIT_WARP(bar, parity, code)                                              \
-  if (!__all_sync(0xffffffffu, bounded_wait((bar), (parity), &sh.abort_flag) ? 1 : 0)) { \
+  if (!__all_sync(0xffffffffu, bounded_wait((bar), (parity), &sh.abort_flag, sh.wait_limit) ? 1 : 0)) { \
     sh.abort_flag = 1;                                                                  \
     atomicCAS(p.status, 0u, (unsigned)(code));                                          \
     goto role_done;                                                                     \
@@ -127,6 +128,7 @@ kdft_f16x2_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __gri
     ptx::mbar_init(&sh.acc_full, 1);
     ptx::mbar_init(&sh.acc_empty, 2 * kEpilogueWarps);                                                           // both CTAs' epilogues
     sh.abort_flag = 0;
+    sh.wait_limit = p.wc.limit_clocks > 0 ? p.wc.limit_clocks : kDefaultWaitClocks;
     ptx::fence_mbar_init();
   }
   if (warp == 1) {

@@ -14,8 +14,8 @@
 //                                brings rows j of 128 neighbouring columns and the split step below
 //                                transposes while it copies (no standalone transpose pass).
 //
-// fp32-level accuracy from TF32 tensor cores (the paper's "decompose and accumulate" remark in
-// Section II-A, here with TF32 pieces): x = x_hi + x_lo, W = W_hi + W_lo, and
+// fp32-level accuracy from TF32 tensor cores (Section II-A describes float32 accuracy from several
+// reduced-precision pieces whose products are accumulated; here the pieces are TF32): x = x_hi + x_lo, W = W_hi + W_lo, and
 //     D += x_hi*W_hi + x_lo*W_hi + x_hi*W_lo      (the x_lo*W_lo term is below fp32 rounding).
 // W_hi/W_lo come pre-split from the float64 generator.  x_hi is the raw fp32 word (the tensor core
 // ignores the low 13 mantissa bits, i.e. truncates), x_lo = x - trunc(x) rounded to TF32.
@@ -58,6 +58,14 @@ constexpr int kKdftThreads = 512;      // 4 warp groups: {producer, MMA, 2 idle}
 constexpr int kEpilogueWarps = 8;
 constexpr size_t kKdftSmemBytes = size_t(kStagesB) * kBytesStageB + size_t(kStagesA) * kBytesStageA + 1024 + 512;
 
+constexpr long long kDefaultWaitClocks = 4000000000LL;   // about two seconds
+
+// what a launch may override for tests of the give-up path (0 / 0 = the defaults)
+struct WaitControl {
+  long long limit_clocks;   // clock budget of every bounded wait; 0 = kDefaultWaitClocks
+  int silent_producer;      // test only: the TMA producer issues nothing, so every wait of the CTA runs out
+};
+
 struct KdftParams {
   int k2;              // 2*N: real contraction length = real output length per line
   int bn;              // output reals per tile: min(256, 2N)
@@ -75,6 +83,7 @@ struct KdftParams {
   float* out;
   unsigned int* status;  // device word, set non-zero when a wait gives up
   long long* profile;    // optional [grid][4] cycle counters of the MMA issuer (builds with DFT3D_PROFILE_WAITS)
+  WaitControl wc;
 };
 
 struct KdftShared {
@@ -84,9 +93,11 @@ struct KdftShared {
   uint64_t acc_full, acc_empty;
   uint32_t tmem_base;
   volatile int abort_flag;
+  long long wait_limit;
 };
 
-__device__ __forceinline__ bool bounded_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool bounded_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                             long long limit = kDefaultWaitClocks) {
   const long long t0 = clock64();
   const uint32_t addr = ptx::smem_u32(bar);
   for (uint32_t spin = 0;; ++spin) {
@@ -103,14 +114,14 @@ __device__ __forceinline__ bool bounded_wait(uint64_t* bar, uint32_t parity, vol
     if (done) return true;
     if ((spin & 0xff) == 0xff) {
       if (*abort_flag) return false;
-      if (clock64() - t0 > 4000000000LL) return false;   // about two seconds
+      if (clock64() - t0 > limit) return false;
     }
   }
 }
 
 // single-thread wait (producer, MMA issuer)
 #define DFT3D_WAIT(bar, parity, code)                               \
-  if (!bounded_wait((bar), (parity), &sh.abort_flag)) {             \
+  if (!bounded_wait((bar), (parity), &sh.abort_flag, sh.wait_limit)) {             \
     sh.abort_flag = 1;                                              \
     atomicCAS(p.status, 0u, (unsigned)(code));                      \
     goto role_done;                                                 \
@@ -118,7 +129,7 @@ __device__ __forceinline__ bool bounded_wait(uint64_t* bar, uint32_t parity, vol
 // whole-warp wait: the warp leaves together, so the .sync.aligned tensor-memory
 // instructions that follow are never executed by a partial warp
 #define DFT3D_WAIT_WARP(bar, parity, code)                                              \
-  if (!__all_sync(0xffffffffu, bounded_wait((bar), (parity), &sh.abort_flag) ? 1 : 0)) { \
+  if (!__all_sync(0xffffffffu, bounded_wait((bar), (parity), &sh.abort_flag, sh.wait_limit) ? 1 : 0)) { \
     sh.abort_flag = 1;                                                                  \
     atomicCAS(p.status, 0u, (unsigned)(code));                                          \
     goto role_done;                                                                     \
@@ -145,6 +156,7 @@ kdft_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_cons
     ptx::mbar_init(&sh.acc_full, 1);
     ptx::mbar_init(&sh.acc_empty, kEpilogueWarps);
     sh.abort_flag = 0;
+    sh.wait_limit = p.wc.limit_clocks > 0 ? p.wc.limit_clocks : kDefaultWaitClocks;
     ptx::fence_mbar_init();
   }
   if (warp == 1) {
@@ -169,7 +181,7 @@ kdft_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_cons
     ptx::setmaxnreg_dec<DFT3D_REGS_WG0>();
     if (warp == 0) {
       // ------------------------------------------------------------ TMA producer
-      if (lane == 0) {
+      if (lane == 0 && !p.wc.silent_producer) {
         uint32_t ib = 0, ia = 0;   // running stage counters
         for (long long t = blockIdx.x; t < total_tiles; t += gridDim.x) {
           const long long mt = t / p.n_tiles;

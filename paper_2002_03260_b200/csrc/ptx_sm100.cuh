@@ -2,9 +2,9 @@
 // mbarriers, TMA tensor copies, tensor memory (TMEM) management, tcgen05.mma
 // (kind::tf32, A from tensor memory or shared memory), tcgen05.ld/st.
 //
-// Every wait is bounded: a spin that runs out of its budget returns false and
-// the caller records an error status and unwinds, so a protocol bug shows up
-// as an error code instead of a hung GPU.
+// The kernels' waits on mbarriers are bounded (bounded_wait in kdft_kernel.cuh): a spin that runs out of
+// its clock budget returns false and the caller records an error status and unwinds, so a protocol bug
+// shows up as an error code instead of a hung GPU.
 #pragma once
 #include <cstdint>
 #include <cuda.h>
@@ -64,26 +64,6 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
 __device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
                : "memory");
-}
-
-// Bounded wait. `budget` counts try_wait attempts (each may block for a
-// hardware-chosen time slice), so the limit is generous in wall time and still finite.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, uint32_t budget = (1u << 24)) {
-  uint32_t addr = smem_u32(bar);
-  for (uint32_t it = 0; it < budget; ++it) {
-    uint32_t done;
-    asm volatile(
-        "{\n\t"
-        ".reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.b32 %0, 1, 0, p;\n\t"
-        "}\n"
-        : "=r"(done)
-        : "r"(addr), "r"(parity)
-        : "memory");
-    if (done) return true;
-  }
-  return false;
 }
 
 // ---------------------------------------------------------------- TMA (no multicast anywhere)

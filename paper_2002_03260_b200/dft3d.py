@@ -133,6 +133,21 @@ def kdft_execute_static(x, out, tables, stream=None):
     float32 CUDA tensors of shape [2, 2*n_a, 2*n_a] (the hi and lo pieces of dft3d_generate_real_table for
     each axis), owned by the caller.  Limited to n0*n1*n2 <= 2**21 points; calls on one GPU must not overlap.
     """
+    import torch
+    for name, t in (("x", x), ("out", out)):
+        if not (isinstance(t, torch.Tensor) and t.is_cuda and t.dtype == torch.complex64 and t.dim() == 3
+                and t.is_contiguous()):
+            raise ValueError("%s must be a contiguous three-dimensional complex64 CUDA tensor" % name)
+    if out.shape != x.shape or out.device != x.device:
+        raise ValueError("out must have the shape and device of x")
+    if len(tables) != 3:
+        raise ValueError("tables must hold one tensor per axis")
+    for a, t in enumerate(tables):
+        want = (2, 2 * x.shape[a], 2 * x.shape[a])
+        if not (isinstance(t, torch.Tensor) and t.is_cuda and t.dtype == torch.float32 and tuple(t.shape) == want
+                and t.is_contiguous() and t.device == x.device):
+            raise ValueError("tables[%d] must be a contiguous float32 CUDA tensor of shape %s on the device of x"
+                             % (a, want))
     n0, n1, n2 = x.shape
     msg = ctypes.create_string_buffer(384)
     status = _lib.dft3d_kdft_execute_static(n0, n1, n2, tables[0].data_ptr(), tables[1].data_ptr(),

@@ -177,3 +177,19 @@ def test_inverse_matrix_matches_the_solve(dft, oracle):
     # nodes that coincide up to rounding (1.1 is not 0.1 + 1 in binary): no zero pivot, but the growth figure says it
     _, growth = dft.generate_inverse_matrix(4, np.array([0.1, 0.3, 1.1, 0.7]))
     assert growth > 1e12
+
+
+def test_static_entry_wrapper_refuses_tensors_it_cannot_vouch_for(dft):
+    """The C side sees only pointers, so the binding checks what they point at before it calls the library: wrong
+    device, dtype, shape or layout raise ValueError here, with no GPU involved."""
+    torch = pytest.importorskip("torch")
+    x = torch.zeros((64, 64, 64), dtype=torch.complex64)
+    tables = [torch.zeros((2, 128, 128), dtype=torch.float32) for _ in range(3)]
+    with pytest.raises(ValueError, match="CUDA"):
+        dft.kdft_execute_static(x, torch.empty_like(x), tables)          # CPU tensors
+    with pytest.raises(ValueError):
+        dft.kdft_execute_static(x.to(torch.complex128), x, tables)       # wrong dtype
+    with pytest.raises(ValueError):
+        dft.kdft_execute_static(x[:, :, ::2], x, tables)                 # not contiguous
+    with pytest.raises(ValueError):
+        dft.kdft_execute_static(np.zeros((64, 64, 64), np.complex64), x, tables)   # not a tensor

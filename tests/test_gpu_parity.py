@@ -586,11 +586,14 @@ def test_config5_2048_exponentials_both_modes(lib, oracle):
     planes = [torch.as_tensor(inp.stratified_indices(n, 16, 6005 + a), device="cuda") for a in range(3)]
     out = torch.empty_like(x)
     kept = None
-    for mode in (lib.DFT3D_FFT, lib.DFT3D_KDFT):
+    floor_only = {}
+    for mode, split in ((lib.DFT3D_FFT, "fp16"), (lib.DFT3D_KDFT, "fp16"), (lib.DFT3D_FFT, "tf32")):
         # FFT: the default limit (16 GiB), i.e. a quarter of a cube of workspace beside the two cubes and the strided
-        # passes once per quarter of the last axis; KDFT: groups of planes
-        plan = lib.Plan(*shape, mode=mode) if mode == lib.DFT3D_FFT else lib.Plan(*shape, mode=mode, workspace_limit=4 * 2 ** 30)
-        if mode == lib.DFT3D_FFT:
+        # passes once per quarter of the last axis; KDFT: groups of planes.  The TF32-piece FFT plan (three passes in
+        # place) is there for the floor-only figure below.
+        sf = _split_flag(lib, split)
+        plan = lib.Plan(*shape, mode=mode, flags=sf) if mode == lib.DFT3D_FFT else lib.Plan(*shape, mode=mode, workspace_limit=4 * 2 ** 30, flags=sf)
+        if mode == lib.DFT3D_FFT and split == "fp16":
             assert plan.workspace_bytes == x.numel() * 2 and plan.launches == 9
         plan(x, out)
         _finish(plan)
@@ -600,6 +603,15 @@ def test_config5_2048_exponentials_both_modes(lib, oracle):
         strata = [pop[c] * d2[count == c].mean() for c in range(4)]
         est = sum(strata) / (P * ex)
         assert est < TOL ** 2, (mode, np.sqrt(est), [np.sqrt(v / (P * ex)) for v in strata])
+        # Reported, not gated: the error of the floor-only coefficients (no index shared with a peak) normalised by
+        # their OWN norm.  No fp32 pipeline can bring this to 1e-5: a floor coefficient is what is left after
+        # peak-sized terms cancel, and it inherits their rounding.
+        name = ("fft" if mode == lib.DFT3D_FFT else "kdft") + "_" + split
+        floor_only[name] = float(np.sqrt(d2[count == 0].sum() / (np.abs(ref[count == 0]) ** 2).sum()))
+        print("config 5, %s: norm-wise estimate %.3g, floor-only subset-normalised error %.3g"
+              % (name, np.sqrt(est), floor_only[name]))
+        if split == "tf32":
+            continue
         for pp in peak_pos:
             assert abs(got[pp] - ref[pp]) < TOL * abs(ref[pp]), (mode, pp, got[pp], ref[pp])
         ey = sum(float((torch.view_as_real(out[i]).double() ** 2).sum()) for i in range(n))
@@ -616,6 +628,12 @@ def test_config5_2048_exponentials_both_modes(lib, oracle):
                 # Parseval is sum|x|^2
                 assert num / a.numel() < (TOL ** 2) * ex, (num / a.numel(), den / a.numel(), ex)
     del kept
+    import json
+    import os
+    record = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "gpurun_out")
+    if os.path.isdir(record):
+        with open(os.path.join(record, "config5_floor_only_error.json"), "w") as f:
+            json.dump(floor_only, f)
 
 
 # ------------------------------------------------------------------ batched 2D / 1D transforms (subset of the axes)

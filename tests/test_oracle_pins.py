@@ -323,3 +323,27 @@ def test_solve_undoes_the_forward_nonuniform_transform(oracle):
     y = rng.standard_normal((1, n, 1)) + 1j * rng.standard_normal((1, n, 1))
     sol = oracle.solve_axis(y, 1, nodes[1]).reshape(n)
     assert np.abs(V @ sol - y.reshape(n)).max() < 1e-11
+
+
+def test_solve_axis_nodes_on_output_solves_the_literal_system_of_eq_1(oracle):
+    """nodes_on_output=True: the rows of V are the arbitrary evaluation points, V[k, n] = z_k^(-n) with
+    z_k = exp(2 pi i w_k) (Eq. 1 read literally, typed here).  The solution must satisfy THAT system and not the
+    transposed one (nodes on the input samples), so an orientation argument dropped on the way fails here."""
+    rng = np.random.default_rng(8)
+    n = 12
+    w = (np.arange(n) + 0.35 * rng.uniform(-1, 1, n)) / n          # distinct, not roots of unity
+    V_out = np.exp(-2j * np.pi * np.outer(w, np.arange(n)))        # V[k, n] = exp(-2 pi i w_k n)
+    X = rng.standard_normal((2, n, 3)) + 1j * rng.standard_normal((2, n, 3))
+    sol = oracle.solve_axis(X, 1, w, nodes_on_output=True)
+    back = np.einsum("kn,anc->akc", V_out, sol)
+    assert np.abs(back - X).max() < 1e-11
+    back_wrong = np.einsum("kn,anc->akc", V_out.T, sol)
+    assert np.abs(back_wrong - X).max() > 1e-2
+    # and it undoes the forward transform of the same orientation
+    x = rng.standard_normal((2, n, 3)) + 1j * rng.standard_normal((2, n, 3))
+    fwd = oracle.dft_axis(x, 1, nodes=w, nodes_on_output=True)
+    assert np.abs(oracle.solve_axis(fwd, 1, w, nodes_on_output=True) - x).max() < 1e-11
+    # solve3d passes the orientation on to every axis that has nodes
+    nodes = [None, w, None]
+    X3 = oracle.dft3d(x, nodes=nodes, nodes_on_output=True)
+    assert np.abs(oracle.solve3d(X3, nodes, nodes_on_output=True) - x).max() < 1e-11

@@ -1,5 +1,5 @@
 """The N>1 path is "replicas only": independent cubes per rank, max-over-ranks timing.  Exercised here with
-two CPU processes over gloo (127.0.0.1), as the GPU machine used for tests has a single GPU."""
+two CPU processes over gloo (127.0.0.1): the replica logic needs no GPU."""
 import os
 import socket
 

@@ -38,6 +38,15 @@ def test_static_entry_point_matches_plan_twice_in_a_row():
         before = torch.cuda.memory_allocated()
         dft.kdft_execute_static(x, out, tables)
         assert torch.cuda.memory_allocated() == before
+        # torch's counter sees only torch's own allocator; the driver's free-memory figure sees a cudaMalloc from
+        # anywhere in the process.  Compare it across a second call (the first one on a device may load kernels),
+        # with no torch allocation in between.
+        torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info()[0]
+        dft.kdft_execute_static(x, out, tables)
+        assert torch.cuda.mem_get_info()[0] == free_before
+        # and against the float64 oracle directly, not only against the plan-based path
+        assert oracle.rel_l2(out.cpu().numpy(), oracle.dft3d(x.cpu().numpy())) < SANITY
         plan = dft.Plan(*shape, mode=dft.DFT3D_KDFT, flags=dft.DFT3D_SPLIT_TF32)  # same TF32 tables and kernel as the static entry
         want = plan(x)
         torch.cuda.synchronize()
