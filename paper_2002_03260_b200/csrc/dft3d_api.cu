@@ -73,6 +73,7 @@ struct Knobs {
   int fft_l2_prefetch = -1, fft_nb2 = -1;
   int fft_inplace = 0, fft_no_half = 0, fft_slices = 0;
   int fft_fuse = -1;                                            // axes 1 and 2 in one launch through an L2-resident ring
+  int fft_fuse_ring = -1, fft_fuse_writers = -1, fft_fuse_hints = -1;   // its ring length (planes), writer CTAs, L2 hints
   int kdft_pair = -1, chunk_kb = -1;
   long long wait_limit = 0;                                     // clock budget of the kernels' bounded waits (0 = default)
   int test_silent_producer = 0;                                 // test of the give-up path: TMA producers issue nothing
@@ -101,6 +102,9 @@ Knobs read_knobs() {
   k.fft_no_half = getenv("DFT3D_FFT_NO_HALF") ? 1 : 0;
   k.fft_slices = env_int("DFT3D_FFT_SLICES", 0);
   k.fft_fuse = env_int("DFT3D_FFT_FUSE", -1);
+  k.fft_fuse_ring = env_int("DFT3D_FFT_FUSE_RING", -1);
+  k.fft_fuse_writers = env_int("DFT3D_FFT_FUSE_WRITERS", -1);
+  k.fft_fuse_hints = env_int("DFT3D_FFT_FUSE_HINTS", -1);
   k.kdft_pair = env_int("DFT3D_KDFT_PAIR", -1);
   k.chunk_kb = env_int("DFT3D_CHUNK_KB", -1);
   if (const char* v = getenv("DFT3D_WAIT_LIMIT_CLOCKS")) k.wait_limit = atoll(v);
@@ -195,6 +199,11 @@ struct dft3d_plan_s {
   size_t workspace_bytes = 0;
   long long group_planes = 0;   // n0-planes per workspace group (KDFT)
   int chunk_kb = 4;             // 32-real stages per tensor-core accumulation chain (KDFT)
+  // FFT, axes 1 and 2 in one launch: a ring of n0-planes between them (meant to stay in L2) and per-plane counters
+  bool fuse12 = false;
+  int ring_planes = 0, fuse_writers = 0;
+  void* ring = nullptr;
+  unsigned int* d_fuse_counters = nullptr;   // [2][n0]: written, consumed
   unsigned int* d_status = nullptr;
   unsigned int* d_amax = nullptr;   // fp16 pieces: float bits of the largest magnitude before pass 0, 1, 2, (3)
   long long* d_profile = nullptr;   // wait-cycle counters, only allocated in DFT3D_PROFILE_WAITS builds
@@ -297,6 +306,10 @@ int set_kernel_attributes(int device) {
   DFT3D_FFT16_ATTR(dft3d::FFT_STRIDED, 32, 4, 4, 0);
   DFT3D_FFT16_ATTR(dft3d::FFT_STRIDED, 32, 4, 4, 1);
 #undef DFT3D_FFT16_ATTR
+  DFT3D_CUDA(cudaFuncSetAttribute(dft3d::fft_f16_fused_kernel<32, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  int(dft3d::fft16_smem_bytes(32, 1))));
+  DFT3D_CUDA(cudaFuncSetAttribute(dft3d::fft_f16_fused_kernel<16, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  int(dft3d::fft16_smem_bytes(16, 1))));
   done = true;
   return DFT3D_OK;
 }
@@ -674,8 +687,17 @@ int fft_blk_pair(const dft3d_plan_s* p) {
 // n2_sub != 0 (fp16-piece kernel, strided axes, blocked layouts only): the pass covers the slice
 // [n2_off, n2_off + n2_sub) of the last axis.  FFT_OUT_BLOCKED: `in` is the full array, `out` receives the blocked
 // order of the slice alone; FFT_IN_BLOCKED: `in` holds that, `out` is the full array (natural order).
+// What fft_axis_pass prepares for one launch of the fp16-piece kernel; with `capture` it hands this back instead of
+// launching (the two-axes launch combines two of them).
+struct FftCapture {
+  CUtensorMap map_data;
+  dft3d::FftF16Params hp;
+};
+
+// map_rows != 0 (axis 2 only): the input is a ring of that many lines (the tensor map covers just them).
 int fft_axis_pass(dft3d_plan_s* p, int axis, const float* in, float* out, cudaStream_t stream,
-                  int layout = FFT_NATURAL, long long n2_off = 0, long long n2_sub = 0) {
+                  int layout = FFT_NATURAL, long long n2_off = 0, long long n2_sub = 0, long long map_rows = 0,
+                  FftCapture* capture = nullptr) {
   const FftAxis& ax = p->fax[axis];
   const int R = ax.R, RX = ax.RX, N = int(ax.n), Lg = 128 / (R * RX);
   const int cols = fft_cols_for(p, axis, layout);
@@ -700,8 +722,8 @@ int fft_axis_pass(dft3d_plan_s* p, int axis, const float* in, float* out, cudaSt
     fp.mtiles_per_stage = 1;
     fp.stage_bytes = Lg * N * 8;
     fp.num_stages = rows / Lg;
-    rc = cached_map(p, &map_data, tag_in, in, 0, 0, [&](CUtensorMap* m) {
-      const unsigned long long dims[3] = {256ull, (unsigned long long)(N / 128), (unsigned long long)rows};
+    rc = cached_map(p, &map_data, tag_in, in, map_rows, 0, [&](CUtensorMap* m) {
+      const unsigned long long dims[3] = {256ull, (unsigned long long)(N / 128), (unsigned long long)(map_rows ? map_rows : rows)};
       const unsigned long long strides[2] = {1024ull, (unsigned long long)N * 8ull};
       const unsigned box[3] = {256u, unsigned(N / 128), unsigned(Lg)};
       return encode_f32(m, in, 3, dims, strides, box, 0);
@@ -787,12 +809,14 @@ int fft_axis_pass(dft3d_plan_s* p, int axis, const float* in, float* out, cudaSt
       // from registers (a block is one contiguous region), which frees the raw stage right after the split
       stage_out = kn.fft_stage_out_blocked >= 0 ? kn.fft_stage_out_blocked : (p->f16 ? 0 : 1);
     } else {
-      if (rc == DFT3D_OK)
+      if (capture) map_out = map_data;   // the two-axes launch stores straight from registers
+      else if (rc == DFT3D_OK)
         rc = cached_map(p, &map_out, tag_out, out, n2_off, n2_sub, [&](CUtensorMap* m) {
           return encode_f32(m, out, 3, dims, strides, box, cols * 8, -1, kn.promo_narrow);
         });
       // rows MiBs apart: send the results out as full rows through TMA stores instead of 32-byte pieces
       stage_out = kn.fft_stage_out >= 0 ? kn.fft_stage_out : (Cmap * 8 >= (1ll << 20) ? 1 : 0);
+      if (capture) stage_out = 0;
     }
     if (n2_sub && stage_out) return fail(DFT3D_ERR_UNSUPPORTED, "internal: sliced pass with staged output");
   }
@@ -811,6 +835,11 @@ int fft_axis_pass(dft3d_plan_s* p, int axis, const float* in, float* out, cudaSt
     if (fp.mtiles_per_stage == 2 && hp.base.raw_stages == 3) hp.base.raw_stages = 2;
     if (fp.mtiles_per_stage != 1 && fp.mtiles_per_stage != 2 && fp.mtiles_per_stage != 4)
       return fail(DFT3D_ERR_UNSUPPORTED, "internal: %d tiles per stage", fp.mtiles_per_stage);
+    if (capture) {
+      capture->map_data = map_data;
+      capture->hp = hp;
+      return DFT3D_OK;
+    }
     const int grid = int(fp.num_stages < p->sm_count ? fp.num_stages : p->sm_count);
     const size_t smem = dft3d::fft16_smem_bytes(R, RX);
 #define DFT3D_FFT16_LAUNCH(MODE, R_, RX_, COLS_, SO_)                                         \
@@ -876,6 +905,43 @@ int fft_axis_pass(dft3d_plan_s* p, int axis, const float* in, float* out, cudaSt
     else DFT3D_FFT_LAUNCH(dft3d::FFT_STRIDED, 16, 2, 16, 2, 1);
   }
 #undef DFT3D_FFT_LAUNCH
+  DFT3D_CUDA(cudaGetLastError());
+  return DFT3D_OK;
+}
+
+// Axes 1 and 2 of a 3D FFT plan in one launch: `blocked` holds the axis-0 pass's result in the blocked order, the
+// result goes to `out`; the intermediate lives in the plan's ring of n0-planes.
+int fft_fused12_pass(dft3d_plan_s* p, const float* blocked, float* out, cudaStream_t stream) {
+  FftCapture w, r;
+  int rc = fft_axis_pass(p, 1, blocked, static_cast<float*>(p->ring), stream, FFT_IN_BLOCKED, 0, 0, 0, &w);
+  if (rc != DFT3D_OK) return rc;
+  const long long ring_rows = (long long)p->ring_planes * p->n[1];
+  rc = fft_axis_pass(p, 2, static_cast<const float*>(p->ring), out, stream, FFT_NATURAL, 0, 0, ring_rows, &r);
+  if (rc != DFT3D_OK) return rc;
+  const long long n0 = p->n[0];
+  DFT3D_CUDA(cudaMemsetAsync(p->d_fuse_counters, 0, sizeof(unsigned int) * 2 * size_t(n0), stream));
+  dft3d::FftFuse fz;
+  memset(&fz, 0, sizeof(fz));
+  fz.written = p->d_fuse_counters;
+  fz.consumed = p->d_fuse_counters + n0;
+  fz.ring = p->ring_planes;
+  fz.ring_rows = ring_rows;
+  fz.ctas_writer = p->fuse_writers;
+  fz.evict_hints = p->knobs.fft_fuse_hints >= 0 ? p->knobs.fft_fuse_hints : 0;
+  // every worker warp (4 per tile) counts itself in once per tile
+  fz.written_target = unsigned(w.hp.base.c_tiles * w.hp.base.mtiles_per_stage * 4);
+  const long long reader_spp = p->n[1] / (128 / (p->fax[2].R * p->fax[2].RX));
+  fz.consumed_target = unsigned(reader_spp * r.hp.base.mtiles_per_stage * 4);
+  // each side counts planes in its own stages
+  w.hp.base.fuse_stages_per_plane = w.hp.base.c_tiles;
+  r.hp.base.fuse_stages_per_plane = reader_spp;
+  const int grid = p->sm_count;
+  if (p->fax[1].R == 32)
+    dft3d::fft_f16_fused_kernel<32, 16><<<grid, dft3d::kFftThreads, dft3d::fft16_smem_bytes(32, 1), stream>>>(
+        w.map_data, p->fax[1].map_w, r.map_data, w.hp, r.hp, fz);
+  else
+    dft3d::fft_f16_fused_kernel<16, 16><<<grid, dft3d::kFftThreads, dft3d::fft16_smem_bytes(16, 1), stream>>>(
+        w.map_data, p->fax[1].map_w, r.map_data, w.hp, r.hp, fz);
   DFT3D_CUDA(cudaGetLastError());
   return DFT3D_OK;
 }
@@ -1146,6 +1212,34 @@ int dft3d_plan_create_ex(dft3d_plan_t* out, long long n0, long long n1, long lon
         e = cudaMalloc(&p->workspace, cube_bytes);
         if (e == cudaSuccess) p->workspace_bytes = cube_bytes;
         else { p->workspace = nullptr; (void)cudaGetLastError(); }   // fall back to the in-place schedule
+        // On request (DFT3D_FFT_FUSE=1): axes 1 and 2 in one launch through a ring of n0-planes that stays in L2 (fp16
+        // pieces, both axes R*R points with the same R, 16-line stages on both strided passes); the axis-0 pass then
+        // writes the blocked order into the workspace.  Not the default: measured at 1024^3 the launch moves 33 instead
+        // of 48 bytes per point through HBM (every ring read hits L2) but takes as long as the two launches it replaces,
+        // because each SM's tile rate, not the HBM stream, bounds these passes (12.1 against 11.6 ms per transform).
+        const FftAxis& a1 = p->fax[1];
+        const FftAxis& a2 = p->fax[2];
+        const int ring = p->knobs.fft_fuse_ring > 0 ? p->knobs.fft_fuse_ring : 4;
+        if (p->workspace && p->f16 && p->knobs.fft_fuse > 0 && a1.R == a2.R && a1.RX == 1 && a2.RX == 1 &&
+            fft_cols_for(p, 0, FFT_OUT_BLOCKED) == 16 && fft_cols_for(p, 1, FFT_IN_BLOCKED) == 16 && n0 >= 2 * ring &&
+            p->sm_count >= 8 && p->knobs.fft_stage_out_blocked <= 0) {
+          const size_t ring_bytes = size_t(ring) * n1 * n2 * 8;
+          e = cudaMalloc(&p->ring, ring_bytes);
+          if (e == cudaSuccess) e = cudaMalloc(&p->d_fuse_counters, sizeof(unsigned int) * 2 * size_t(n0));
+          if (e == cudaSuccess) {
+            p->fuse12 = true;
+            p->ring_planes = ring;
+            p->workspace_bytes += ring_bytes;
+            // CTAs of the axis-1 side; the rest run the axis-2 side.  The strided side needs a little more time per
+            // point than the contiguous one (3.5 against 2.9 ms per pass of 1024^3), so it gets the larger share.
+            int wr = p->knobs.fft_fuse_writers > 0 ? p->knobs.fft_fuse_writers : (p->sm_count * 80 + 74) / 148;
+            if (wr >= p->sm_count) wr = p->sm_count - 1;
+            p->fuse_writers = wr;
+          } else {
+            if (p->ring) { cudaFree(p->ring); p->ring = nullptr; }
+            (void)cudaGetLastError();
+          }
+        }
       } else if (axes == 7u && nests && p->f16 && !p->knobs.fft_no_half) {
         // Too large for a whole cube of workspace: a half, a quarter or an eighth of a cube, whichever fits first.
         // The two strided passes then run once per slice of the last axis through the blocked order in the workspace,
@@ -1287,6 +1381,11 @@ int dft3d_execute(dft3d_plan_t p, const void* in, void* out, void* cuda_stream) 
       return fft_axis_pass(p, 2, ws, fout, stream);
     }
 #endif
+    if (p->fuse12) {
+      // axis 0 in -> workspace (blocked order), then axes 1 and 2 in one launch: workspace -> ring (L2) -> out
+      if ((rc = fft_axis_pass(p, 0, fin, ws, stream, FFT_OUT_BLOCKED)) != DFT3D_OK) return rc;
+      return fft_fused12_pass(p, ws, fout, stream);
+    }
     if ((rc = fft_axis_pass(p, 0, fin, fout, stream, FFT_OUT_BLOCKED)) != DFT3D_OK) return rc;
     if ((rc = fft_axis_pass(p, 1, fout, ws, stream, FFT_IN_BLOCKED)) != DFT3D_OK) return rc;
     return fft_axis_pass(p, 2, ws, fout, stream);
@@ -1397,6 +1496,7 @@ int dft3d_plan_launches(dft3d_plan_t p) {
   if (p->mode == DFT3D_KDFT && p->axes == 6u) return pre + int(2 * (p->n[0] / p->group_planes));
   if (p->mode == DFT3D_FFT && p->ws_slices && !p->knobs.fft_inplace)
     return 2 * p->ws_slices + 1;   // two strided passes per slice, one contiguous
+  if (p->mode == DFT3D_FFT && p->fuse12 && !p->knobs.fft_inplace) return 2;   // axis 0, then axes 1 and 2 together
   return pre + count;
 }
 
@@ -1414,6 +1514,8 @@ int dft3d_plan_destroy(dft3d_plan_t p) {
     if (p->fax[a].d_tw2) cudaFree(p->fax[a].d_tw2);
   }
   if (p->workspace) cudaFree(p->workspace);
+  if (p->ring) cudaFree(p->ring);
+  if (p->d_fuse_counters) cudaFree(p->d_fuse_counters);
   if (p->d_status) cudaFree(p->d_status);
   if (p->d_amax) cudaFree(p->d_amax);
   if (p->d_profile) cudaFree(p->d_profile);

@@ -52,6 +52,20 @@ struct FftF16Params {
   float quarter_turn;           // RX == 4: the sign s of the exponent (exp(s*2*pi*i/4) = s*i)
 };
 
+// Two axes in one launch (fft_f16_fused_kernel below): the CTAs of the axis-1 pass write n0-planes of their result
+// into a ring of `ring` planes, the CTAs of the axis-2 pass read them from there, and these counters order the two.
+// All zero for the one-axis kernels.
+struct FftFuse {
+  unsigned int* written;     // [planes] warps that have stored their share of plane p (writer side adds, reader side waits)
+  unsigned int* consumed;    // [planes] warps whose share of plane p has arrived in shared memory (reader side adds)
+  unsigned int written_target, consumed_target;
+  int ring;                  // planes in the ring; plane p lives in slot p % ring
+  long long ring_rows;       // reader: rows (lines) of the whole ring, ring * n1
+  int ctas_writer;           // CTAs 0 .. ctas_writer-1 run the axis-1 pass, the others the axis-2 pass
+  int evict_hints;           // 1: L2 eviction hints (input and output stream: evict first; ring: evict last)
+};
+enum : int { FUSE_NONE = 0, FUSE_WRITER = 1, FUSE_READER = 2 };
+
 struct FftF16Shared {
   uint64_t raw_full[4], raw_empty[4], out_ready[4];
   uint64_t split_done[4];      // STAGE_OUT with tiles that share lines: every tile of the stage has read its input
@@ -98,10 +112,30 @@ __host__ __device__ constexpr size_t fft16_smem_bytes(int R, int RX) {   // RX =
     FFT_PROF_END(code)                                                                    \
   }
 
-template <int MODE, int R, int RX, int COLS, int STAGE_OUT>
-__global__ void __launch_bounds__(kFftThreads, 1)
-fft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_constant__ CUtensorMap map_w,
-                    const __grid_constant__ CUtensorMap map_out, const FftF16Params pp) {
+// Waits until a counter in global memory that other CTAs add to has reached `target` (bounded like every other wait).
+__device__ __forceinline__ bool bounded_wait_counter(const unsigned int* counter, unsigned int target,
+                                                     volatile int* abort_flag, long long limit) {
+  const long long t0 = clock64();
+  for (uint32_t spin = 0;; ++spin) {
+    unsigned int v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(counter) : "memory");
+    if (v >= target) return true;
+    if ((spin & 0xf) == 0xf) {
+      if (*abort_flag) return false;
+      if (clock64() - t0 > limit) return false;
+    }
+    __nanosleep(200);
+  }
+}
+
+// The body of one CTA: CTA number `cta` of `ncta` takes the stages cta, cta + ncta, ...  FUSE: see FftFuse.
+template <int MODE, int R, int RX, int COLS, int STAGE_OUT, int FUSE>
+__device__ __forceinline__ void fft_f16_axis_body(const CUtensorMap* map_data_p, const CUtensorMap* map_w_p,
+                                                  const CUtensorMap* map_out_p, const FftF16Params& pp,
+                                                  const FftFuse& fz, const int cta, const int ncta) {
+  const CUtensorMap& map_data = *map_data_p;
+  const CUtensorMap& map_w = *map_w_p;
+  const CUtensorMap& map_out = *map_out_p;
   const FftParams& p = pp.base;
   extern __shared__ uint8_t smem_raw_[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw_) + 1023) & ~uintptr_t(1023));
@@ -162,7 +196,7 @@ fft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_c
   const uint32_t tmem = sh.tmem_base;
 
   long long my_stages = 0;
-  if ((long long)blockIdx.x < p.num_stages) my_stages = (p.num_stages - 1 - blockIdx.x) / gridDim.x + 1;
+  if ((long long)cta < p.num_stages) my_stages = (p.num_stages - 1 - cta) / ncta + 1;
   const long long my_mtiles = my_stages * p.mtiles_per_stage;
 
   // Registers: the workers keep a line slice in registers and take what the first group can spare.  setmaxnreg is a
@@ -177,19 +211,47 @@ fft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_c
         for (int pc = 0; pc < 2; ++pc)                // [piece][2R rows][64 halves]
           ptx::tma_load_2d(smem_w + pc * kWPiece, &map_w, &sh.w_full, 0, pc * NB);
         long long i = 0;
-        for (long long sidx = blockIdx.x; sidx < p.num_stages; sidx += gridDim.x, ++i) {
+        long long plane_ok = -1;                      // FUSE: the plane the last counter wait was for
+        // FUSE with hints: the stream from HBM leaves L2 first, the ring stays
+        const bool hints = FUSE != FUSE_NONE && fz.evict_hints;
+        const uint64_t pol_load = hints ? (FUSE == FUSE_WRITER ? ptx::l2_policy_evict_first() : ptx::l2_policy_evict_last()) : 0;
+        for (long long sidx = cta; sidx < p.num_stages; sidx += ncta, ++i) {
           const uint32_t s = uint32_t(i % p.raw_stages), ph = uint32_t(i / p.raw_stages) & 1;
           F16_WAIT(&sh.raw_empty[s], ph ^ 1, 0x501);
+          if (FUSE != FUSE_NONE) {
+            // writer: the plane that last lived in this stage's ring slot must have been read completely before
+            // anything of this stage is stored there; the load below gates this CTA's stores (the workers store only
+            // after they have seen it land).  Reader: the plane must have been written completely.
+            const long long plane = sidx / p.fuse_stages_per_plane;
+            const long long need = (FUSE == FUSE_WRITER) ? plane - fz.ring : plane;
+            if (need >= 0 && need != plane_ok) {
+              const unsigned int* counter = (FUSE == FUSE_WRITER ? fz.consumed : fz.written) + need;
+              const unsigned int target = FUSE == FUSE_WRITER ? fz.consumed_target : fz.written_target;
+              if (!bounded_wait_counter(counter, target, &sh.abort_flag, sh.wait_limit)) {
+                sh.abort_flag = 1;
+                atomicCAS(p.status, 0u, 0x502u);
+                goto role_done;
+              }
+              plane_ok = need;
+              // the loads that follow read, through the async proxy, what other CTAs wrote with ordinary stores
+              asm volatile("fence.proxy.async.global;" ::: "memory");
+            }
+          }
           ptx::mbar_arrive_expect_tx(&sh.raw_full[s], uint32_t(p.stage_bytes));
           uint8_t* dst = smem_rawring + size_t(s) * p.stage_bytes;
           if (MODE == FFT_CONTIG) {
-            ptx::tma_load_3d(dst, &map_data, &sh.raw_full[s], 0, 0, int(sidx * Lg));
+            const long long row0 = sidx * Lg;
+            if (hints) ptx::tma_load_3d_hint(dst, &map_data, &sh.raw_full[s], 0, 0, int(row0 % fz.ring_rows), pol_load);
+            else ptx::tma_load_3d(dst, &map_data, &sh.raw_full[s], 0, 0, int(FUSE == FUSE_READER ? row0 % fz.ring_rows : row0));
           } else {
             const long long ct = sidx % p.c_tiles, bt = sidx / p.c_tiles;
             for (int r0 = 0; r0 < p.N; r0 += 256) {
               if (p.in_blocked && p.blk_pair > 1)
                 ptx::tma_load_5d(dst + size_t(r0) * kRowBytes, &map_data, &sh.raw_full[s], 0, 0, int(bt), r0 / p.blk_pair,
                                  int(ct));
+              else if (p.in_blocked && hints)
+                ptx::tma_load_4d_hint(dst + size_t(r0) * kRowBytes, &map_data, &sh.raw_full[s],
+                                      int(ct % p.blk_ratio) * 2 * COLS, int(bt), r0, int(ct / p.blk_ratio), pol_load);
               else if (p.in_blocked)
                 ptx::tma_load_4d(dst + size_t(r0) * kRowBytes, &map_data, &sh.raw_full[s],
                                  int(ct % p.blk_ratio) * 2 * COLS, int(bt), r0, int(ct / p.blk_ratio));
@@ -200,7 +262,7 @@ fft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_c
               else
                 ptx::tma_load_3d(dst + size_t(r0) * kRowBytes, &map_data, &sh.raw_full[s], int(ct * 2 * COLS), r0, int(bt));
             }
-            const long long nidx = sidx + gridDim.x;
+            const long long nidx = sidx + ncta;
             if (p.l2_prefetch && nidx < p.num_stages) {
               const long long nct = nidx % p.c_tiles, nbt = nidx / p.c_tiles;
               for (int r0 = 0; r0 < p.N; r0 += 256)
@@ -272,7 +334,7 @@ fft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_c
     } else if (STAGE_OUT) {
       // ---------------------------------------------------------- warp 3: finished stages leave as TMA stores
       long long istage = 0;
-      for (long long sidx = blockIdx.x; sidx < p.num_stages; sidx += gridDim.x, ++istage) {
+      for (long long sidx = cta; sidx < p.num_stages; sidx += ncta, ++istage) {
         const uint32_t s = uint32_t(istage % p.raw_stages), ph = uint32_t(istage / p.raw_stages) & 1;
         F16_WAIT_WARP(&sh.out_ready[s], ph, 0x902);
         if (lane == 0) {
@@ -333,11 +395,13 @@ fft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_c
       }
     }
     const float om1 = pp.out_mul;
+    const bool st_hints = FUSE != FUSE_NONE && fz.evict_hints;
+    const uint64_t pol_store = st_hints ? (FUSE == FUSE_WRITER ? ptx::l2_policy_evict_last() : ptx::l2_policy_evict_first()) : 0;
 
     for (long long t = g; t < my_mtiles; t += 4) {
       const long long istage = t / p.mtiles_per_stage;
       const int mt = int(t % p.mtiles_per_stage);
-      const long long sidx = (long long)blockIdx.x + istage * gridDim.x;
+      const long long sidx = (long long)cta + istage * ncta;
       const uint32_t s = uint32_t(istage % p.raw_stages), phs = uint32_t(istage / p.raw_stages) & 1;
       const uint32_t pk = uint32_t(t >> 2) & 1;
       uint8_t* stage = smem_rawring + size_t(s) * p.stage_bytes;
@@ -410,7 +474,14 @@ fft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_c
           // the raw stage is refilled by TMA (async proxy): order this thread's reads before that write
           ptx::fence_proxy_async_smem();
           __syncwarp();
-          if (lane == 0) ptx::mbar_arrive(&sh.raw_empty[s]);
+          if (lane == 0) {
+            ptx::mbar_arrive(&sh.raw_empty[s]);
+            if (FUSE == FUSE_READER) {
+              // this warp's share of the plane has left the ring (the load had landed before raw_full completed)
+              __threadfence();
+              atomicAdd(fz.consumed + sidx / p.fuse_stages_per_plane, 1u);
+            }
+          }
         } else if (kPairTiles) {
           // the results return into the raw stage, and the RX tiles of a group of lines all read ALL rows of those
           // lines: none of them may store before the others have read (the tile without twiddles is well ahead)
@@ -508,7 +579,8 @@ fft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_c
             dst = reinterpret_cast<float2*>(p.out) + ((blk * p.N + (RX * k1 + bsel2)) * P + i1 % P) * COLS + (col0 + g2);
             k2_stride = (long long)(RX * R) * COLS * P;
           } else {
-            dst = reinterpret_cast<float2*>(p.out) + (bt * p.N + (RX * k1 + bsel2)) * p.out_pitch + p.out_off + col;
+            const long long slot = (FUSE == FUSE_WRITER) ? bt % fz.ring : bt;
+            dst = reinterpret_cast<float2*>(p.out) + (slot * p.N + (RX * k1 + bsel2)) * p.out_pitch + p.out_off + col;
             k2_stride = (long long)(RX * R) * p.out_pitch;
           }
         }
@@ -548,13 +620,19 @@ fft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_c
           } else if (ok) {
             if (MODE == FFT_CONTIG) {
               float2* pd = dst + ch * 16 * (RX * R);  // compile-time stride: immediate offsets
+              if (st_hints) {
 #pragma unroll
-              for (int j = 0; j < 16; ++j) pd[j * (RX * R)] = make_float2(f[2 * j], f[2 * j + 1]);
+                for (int j = 0; j < 16; ++j) ptx::st_global_v2_hint(pd + j * (RX * R), f[2 * j], f[2 * j + 1], pol_store);
+              } else {
+#pragma unroll
+                for (int j = 0; j < 16; ++j) pd[j * (RX * R)] = make_float2(f[2 * j], f[2 * j + 1]);
+              }
             } else {
               float2* pd = dst + (long long)(ch * 16) * k2_stride;
 #pragma unroll
               for (int j = 0; j < 16; ++j) {
-                *pd = make_float2(f[2 * j], f[2 * j + 1]);
+                if (st_hints) ptx::st_global_v2_hint(pd, f[2 * j], f[2 * j + 1], pol_store);
+                else *pd = make_float2(f[2 * j], f[2 * j + 1]);
                 pd += k2_stride;
                 asm volatile("" : "+l"(pd));          // one running pointer, not sixteen precomputed ones
               }
@@ -562,6 +640,12 @@ fft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_c
           }
         }
         ptx::tc_fence_before();                       // the next tile's split overwrites these columns
+        if (FUSE == FUSE_WRITER) {
+          // this warp's stores of the tile are out: make them visible, then count the warp in for the plane
+          __threadfence();
+          __syncwarp();
+          if (lane == 0) atomicAdd(fz.written + sidx / p.fuse_stages_per_plane, 1u);
+        }
         if (STAGE_OUT) {
           ptx::fence_proxy_async_smem();              // generic writes -> visible to the TMA store
           __syncwarp();
@@ -575,7 +659,7 @@ role_done:
 #ifdef DFT3D_PROFILE_WAITS
   if (p.profile && lane == 0 && (warp <= 3 || (warp & 3) == 0)) {
     // one reporter per role / group: rows 5..9 by wait code, column by code & 7; workers add up over the groups
-    long long* dst = p.profile + size_t(blockIdx.x) * 128;
+    long long* dst = p.profile + size_t(cta) * 128;
     for (int i = 5; i < 10; ++i)
       for (int j = 0; j < 8; ++j)
         if (prof_wait[i][j]) atomicAdd(reinterpret_cast<unsigned long long*>(dst + i * 8 + j), (unsigned long long)prof_wait[i][j]);
@@ -593,5 +677,37 @@ role_done:
 
 #undef F16_WAIT
 #undef F16_WAIT_WARP
+
+// one axis per launch
+template <int MODE, int R, int RX, int COLS, int STAGE_OUT>
+__global__ void __launch_bounds__(kFftThreads, 1)
+fft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_constant__ CUtensorMap map_w,
+                    const __grid_constant__ CUtensorMap map_out, const FftF16Params pp) {
+  const FftFuse none = {};
+  fft_f16_axis_body<MODE, R, RX, COLS, STAGE_OUT, FUSE_NONE>(&map_data, &map_w, &map_out, pp, none, int(blockIdx.x),
+                                                            int(gridDim.x));
+}
+
+// Axes 1 and 2 of a 3D transform in ONE launch (Eq. 17 applied axis after axis, Section IV-D's closing remark): the
+// first `ctas_writer` CTAs run the axis-1 pass (strided, COLS-line stages) plane by plane into a ring of a few
+// n0-planes, the others run the axis-2 pass (contiguous) out of that ring into the output.  The ring is small enough
+// to stay in L2, so the intermediate between the two axes is written and read back there instead of in HBM: 32 bytes
+// of HBM traffic per point and transform instead of 48.  Both kinds of CTA take their stages in plane order, and a
+// stage waits only for stages that come before it in that order (a reader for the writers of its plane, a writer for
+// the readers of the plane that used its ring slot last), so with all CTAs resident (one per SM, grid <= SM count)
+// nobody waits for somebody who waits for them.  Both axes have the same length R*R (same table and twiddles).
+template <int R, int COLS>
+__global__ void __launch_bounds__(kFftThreads, 1)
+fft_f16_fused_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant__ CUtensorMap map_w,
+                     const __grid_constant__ CUtensorMap map_ring, const FftF16Params writer, const FftF16Params reader,
+                     const FftFuse fz) {
+  if (int(blockIdx.x) < fz.ctas_writer)
+    fft_f16_axis_body<FFT_STRIDED, R, 1, COLS, 0, FUSE_WRITER>(&map_in, &map_w, &map_in, writer, fz, int(blockIdx.x),
+                                                               fz.ctas_writer);
+  else
+    fft_f16_axis_body<FFT_CONTIG, R, 1, COLS, 0, FUSE_READER>(&map_ring, &map_w, &map_ring, reader, fz,
+                                                              int(blockIdx.x) - fz.ctas_writer,
+                                                              int(gridDim.x) - fz.ctas_writer);
+}
 
 }  // namespace dft3d

@@ -85,6 +85,7 @@ struct FftParams {
   unsigned int* status;
   long long* profile;    // optional cycle counters (builds with DFT3D_PROFILE_WAITS): [grid][16][8]
   WaitControl wc;
+  long long fuse_stages_per_plane;   // two-axes launch (fp16-piece kernel): stages of this pass per n0-plane
 };
 
 struct FftShared {

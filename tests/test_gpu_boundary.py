@@ -108,7 +108,7 @@ def test_knobs_are_fixed_when_the_plan_is_created(lib, monkeypatch):
 
 
 @pytest.mark.parametrize("mode_name,shape,axes", [("kdft", (64, 64, 64), None), ("kdft_tf32", (64, 64, 64), None),
-                                                 ("fft", (64, 64, 256), (2,)), ("fft", (256, 16, 64), (0,))])
+                                                 ("fft", (64, 64, 256), (2,)), ("fft", (256, 64, 64), (0,))])
 def test_bounded_waits_give_up_and_report(lib, oracle, monkeypatch, mode_name, shape, axes):
     """Every device-side wait has a clock budget.  Here the budget is about a millisecond and the TMA producer of every
     CTA stays silent, so nothing is ever in flight and every role's first wait runs out: the kernels return by

@@ -332,6 +332,54 @@ def test_fft_half_cube_workspace(lib, oracle, shape):
     assert _rel_l2_gpu(a, b) < SANITY
 
 
+@pytest.mark.parametrize("shape", [(256, 256, 256), pytest.param((256, 1024, 1024), marks=pytest.mark.slow),
+                                   (512, 1024, 1024), (1024, 256, 256)])
+def test_fft_two_axes_in_one_launch(lib, oracle, shape, monkeypatch):
+    """With DFT3D_FFT_FUSE=1, plans whose axes 1 and 2 have the same length R*R run those two axes in ONE launch: the
+    CTAs of the axis-1 pass hand n0-planes to the CTAs of the axis-2 pass through a small ring (two launches per
+    transform instead of three).  The arithmetic of every line is that of the one-axis kernels, so the result equals
+    the three-launch schedule bit for bit; the first two shapes also go against the full float64 oracle."""
+    x = _inputs().cube(shape, "normal", 70, device="cuda")
+    plain = lib.Plan(*shape, mode=lib.DFT3D_FFT)
+    assert plain.launches == 3
+    monkeypatch.setenv("DFT3D_FFT_FUSE", "1")
+    fused = lib.Plan(*shape, mode=lib.DFT3D_FFT)
+    assert fused.launches == 2
+    a = fused(x)
+    _finish(fused)
+    b = plain(x)
+    _finish(plain)
+    plain.destroy()
+    assert torch.equal(a, b)
+    del b
+    # again, with the ring and its counters left over from the first run, and with a very short ring
+    a2 = fused(x)
+    _finish(fused)
+    fused.destroy()
+    assert torch.equal(a, a2)
+    monkeypatch.setenv("DFT3D_FFT_FUSE_RING", "2")
+    monkeypatch.setenv("DFT3D_FFT_FUSE_WRITERS", "37")
+    monkeypatch.setenv("DFT3D_FFT_FUSE_HINTS", "1")
+    short = lib.Plan(*shape, mode=lib.DFT3D_FFT)
+    monkeypatch.delenv("DFT3D_FFT_FUSE_RING")
+    monkeypatch.delenv("DFT3D_FFT_FUSE_WRITERS")
+    monkeypatch.delenv("DFT3D_FFT_FUSE_HINTS")
+    a2 = short(x)
+    _finish(short)
+    short.destroy()
+    assert torch.equal(a, a2)
+    del a2
+    if shape[1] * shape[2] * shape[0] <= 256 * 1024 * 1024 and shape[0] == 256:
+        assert oracle.rel_l2(a.cpu().numpy(), oracle.dft3d(x.cpu().numpy())) < SANITY
+    inv = lib.Plan(*shape, mode=lib.DFT3D_FFT, sign=lib.DFT3D_INVERSE)
+    monkeypatch.delenv("DFT3D_FFT_FUSE")
+    assert inv.launches == 2
+    back = inv(a)
+    _finish(inv)
+    inv.destroy()
+    assert _rel_l2_gpu(back, x) < SANITY
+
+
 @pytest.mark.slow
 def test_fft_blocked_order_with_four_rows_per_line(lib):
     """4096-point strided axes have 4-line stages (32-byte pieces): in the blocked order between the axis-0 and the

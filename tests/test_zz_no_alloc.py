@@ -75,6 +75,10 @@ def test_static_entry_point_rejects_what_it_cannot_hold():
     with pytest.raises(dft.Dft3dError) as e:
         dft.kdft_execute_static(x, out, tables)
     assert e.value.status == 2 and "exceed the static scratch" in str(e.value)
+    small = x[:64, :64, :100].contiguous()      # 100 is not a multiple of 64
     with pytest.raises(dft.Dft3dError) as e:
-        dft.kdft_execute_static(x[:64, :64, :100].contiguous(), out, tables)
+        dft.kdft_execute_static(small, torch.empty_like(small),
+                                [torch.zeros((2, 2 * n, 2 * n), device="cuda") for n in small.shape])
     assert e.value.status == 2
+    with pytest.raises(ValueError):             # the binding refuses an output of another shape before any kernel runs
+        dft.kdft_execute_static(small, out, tables)
