@@ -73,7 +73,12 @@ enum {
 typedef struct dft3d_options_s {
   size_t struct_size;     /* sizeof(dft3d_options_t), for forward compatibility */
   unsigned flags;         /* DFT3D_NODES_ON_OUTPUT | DFT3D_UNSCALED_INVERSE | DFT3D_SPLIT_* | DFT3D_DESTROY_INPUT */
-  int fft_split[3][2];    /* FFT mode: {N1, N2} per axis with N1*N2 = n_a; {0,0} = default split */
+  int fft_split[3][2];    /* FFT mode: {N1, N2} per axis with N1*N2 = n_a, first and second matrix product of Eq. 17.
+                             {0,0} = the built-in split, which is also the only one the kernels realise: N2 = 16 for
+                             n_a = 256 and 512, N2 = 32 from 1024 on, N1 = n_a / N2 (256 = 16*16, 512 = 32*16,
+                             1024 = 32*32, 2048 = 64*32, 4096 = 128*32; an N1 above N2 is itself computed as
+                             (N1/N2) * N2 by one more application of Eq. 17).  Any other pair returns
+                             DFT3D_ERR_UNSUPPORTED; dft3d_plan_fft_split reports the pair in use. */
   size_t workspace_limit; /* upper bound in bytes for the plan-owned workspace; 0 = default (16 GiB).  KDFT needs a
                              workspace and shrinks it to groups of n0-planes.  FFT uses one cube of workspace when it
                              fits (fewest launches), else a half, a quarter or an eighth of a cube, whichever fits
@@ -105,8 +110,9 @@ typedef struct dft3d_options_s {
  * reduced phases and rounded once to the stored float32 pieces.  The plan owns its
  * device tables and workspace (allocated on the current device during this call).
  *
- * Supported sizes: KDFT: every n_a even, n_a <= 8192 (tiles that are not full are zero-filled on load
- * and masked on store, the way the paper's compiler pads to its hardware's preferred shapes).  FFT: every
+ * Supported sizes: KDFT: n0 and n1 of any length, n2 even (rows of the data must start on 16-byte boundaries),
+ * transformed n_a <= 8192 (tiles that are not full are zero-filled on load and masked on store, and an odd length pads
+ * the rows of the table, the way the paper's compiler pads to its hardware's preferred shapes).  FFT: every
  * transformed n_a in {256, 512, 1024, 2048, 4096} (N = R*R, 2*R*R or 4*R*R with R = 16 or 32; 4096 with fp16
  * pieces only), the others multiples of 64.
  * Other sizes return DFT3D_ERR_UNSUPPORTED.
@@ -175,6 +181,11 @@ int dft3d_plan_launches(dft3d_plan_t plan);
 
 /* DFT3D_SPLIT_FP16 or DFT3D_SPLIT_TF32: the operand split the plan uses; 0 for NULL. */
 int dft3d_plan_split(dft3d_plan_t plan);
+
+/* The factor pair {N1, N2} of Eq. 17 that the plan uses on `axis` (N1 * N2 = n_axis): DFT3D_OK and the pair for an axis
+ * the plan transforms in the FFT formulation, DFT3D_ERR_INVALID_ARG otherwise (NULL plan or pointers, an axis in the KDFT
+ * formulation or not transformed). */
+int dft3d_plan_fft_split(dft3d_plan_t plan, int axis, int* n1, int* n2);
 
 /* Frees device and host memory of the plan.  NULL is accepted. */
 int dft3d_plan_destroy(dft3d_plan_t plan);

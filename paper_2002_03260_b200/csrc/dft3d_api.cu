@@ -395,10 +395,25 @@ int build_kdft_axis(dft3d_plan_s* p, int a, const double* nodes) {
   }
   if (!solve) dft3d::gen::axis_matrix(n, p->sign, scale, nodes, (p->flags & DFT3D_NODES_ON_OUTPUT) != 0, M.data());
   dft3d::gen::real_table_from_matrix(n, M.data(), W.data(), W.data() + size_t(4) * n * n);
+  // TMA wants every row of the table to start on a 16-byte boundary: rows of 2n floats do when n is even; for odd n the
+  // TABLE gets two columns of padding per row (never read: the tensor map's extent stays 2n), the data is left alone
+  const long long ld = 2 * n + (n % 2 ? 2 : 0);
+  if (ld != 2 * n) {
+    std::vector<float> padded;
+    try {
+      padded.assign(size_t(2) * 2 * n * ld, 0.0f);
+    } catch (const std::bad_alloc&) {
+      return fail(DFT3D_ERR_ALLOC, "host allocation of the axis-%d table failed", a);
+    }
+    for (int pc = 0; pc < 2; ++pc)
+      for (long long r = 0; r < 2 * n; ++r)
+        memcpy(&padded[(size_t(pc) * 2 * n + r) * ld], &W[(size_t(pc) * 2 * n + r) * 2 * n], sizeof(float) * 2 * n);
+    W.swap(padded);
+  }
   DFT3D_CUDA(cudaMalloc(&ax.d_w, W.size() * sizeof(float)));
   DFT3D_CUDA(cudaMemcpy(ax.d_w, W.data(), W.size() * sizeof(float), cudaMemcpyHostToDevice));
   const unsigned long long dims[3] = {(unsigned long long)(2 * n), (unsigned long long)(2 * n), 2ull};
-  const unsigned long long strides[2] = {(unsigned long long)(2 * n * 4), (unsigned long long)(4 * n * n * 4)};
+  const unsigned long long strides[2] = {(unsigned long long)(ld * 4), (unsigned long long)(2 * n * ld * 4)};
   const unsigned box[3] = {unsigned(dft3d::kBlockK), unsigned(ax.bn), 2u};
   return encode_f32(&ax.map_w, ax.d_w, 3, dims, strides, box, 128);
 }
@@ -1069,11 +1084,12 @@ int dft3d_plan_create_ex(dft3d_plan_t* out, long long n0, long long n1, long lon
   for (int a = 0; a < 3; ++a) {
     const bool transformed = (axes >> a) & 1u;
     if (a == 0 && !transformed) continue;   // a pure batch index
-    // KDFT: rows of the table and of the data must start on 16-byte boundaries (TMA), i.e. even lengths;
-    // FFT: the untransformed axes are split into groups of 16 lines
-    const long long quantum = (mode == DFT3D_FFT) ? 64 : 2;
+    // KDFT: rows of the data must start on 16-byte boundaries (TMA): the last axis must be even, the others may have
+    // any length (odd lengths pad the table, not the data).  FFT: the untransformed axes are split into groups of 16 lines
+    const long long quantum = (mode == DFT3D_FFT) ? 64 : (a == 2 ? 2 : 1);
     if (nn[a] % quantum != 0)
-      return fail(DFT3D_ERR_UNSUPPORTED, "n%d = %lld is not a multiple of %lld", a, nn[a], quantum);
+      return fail(DFT3D_ERR_UNSUPPORTED, "n%d = %lld is not a multiple of %lld%s", a, nn[a], quantum,
+                  (mode != DFT3D_FFT && a == 2) ? " (rows of the data, 8*n2 bytes each, must start on 16-byte boundaries)" : "");
     if (transformed && nn[a] > 8192) return fail(DFT3D_ERR_UNSUPPORTED, "n%d = %lld exceeds 8192", a, nn[a]);
     if (transformed && nn[a] % 4 != 0) {
       if (opt.flags & DFT3D_SPLIT_FP16)
@@ -1503,6 +1519,15 @@ int dft3d_plan_launches(dft3d_plan_t p) {
 int dft3d_plan_split(dft3d_plan_t p) {
   if (!p) return 0;
   return p->f16 ? DFT3D_SPLIT_FP16 : DFT3D_SPLIT_TF32;
+}
+
+int dft3d_plan_fft_split(dft3d_plan_t p, int axis, int* n1, int* n2) {
+  if (!p || !n1 || !n2) return fail(DFT3D_ERR_INVALID_ARG, "plan, n1 and n2 must not be NULL");
+  if (axis < 0 || axis > 2 || !((p->axes >> axis) & 1u) || p->amode[axis] != DFT3D_FFT)
+    return fail(DFT3D_ERR_INVALID_ARG, "axis %d is not transformed in the FFT formulation by this plan", axis);
+  *n1 = p->fax[axis].RX * p->fax[axis].R;
+  *n2 = p->fax[axis].R;
+  return DFT3D_OK;
 }
 
 int dft3d_plan_destroy(dft3d_plan_t p) {

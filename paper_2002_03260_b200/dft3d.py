@@ -21,7 +21,8 @@ DFT3D_INVERSE_SOLVE = 32
 EXPORTS = [
     "dft3d_plan_create", "dft3d_plan_create_ex", "dft3d_execute", "dft3d_execute_host", "dft3d_execute_host_batch",
     "dft3d_execute_axis",
-    "dft3d_plan_status", "dft3d_plan_workspace_bytes", "dft3d_plan_launches", "dft3d_plan_split", "dft3d_plan_destroy",
+    "dft3d_plan_status", "dft3d_plan_workspace_bytes", "dft3d_plan_launches", "dft3d_plan_split", "dft3d_plan_fft_split",
+    "dft3d_plan_destroy",
     "dft3d_status_string", "dft3d_last_error", "dft3d_generate_axis_matrix", "dft3d_generate_twiddle", "dft3d_generate_inverse_matrix",
     "dft3d_generate_real_table", "dft3d_kdft_execute_static",
 ]
@@ -61,6 +62,7 @@ def _load():
     lib.dft3d_plan_workspace_bytes.restype = ctypes.c_size_t
     lib.dft3d_plan_launches.argtypes = [vp]
     lib.dft3d_plan_split.argtypes = [vp]
+    lib.dft3d_plan_fft_split.argtypes = [vp, ci, ctypes.POINTER(ci), ctypes.POINTER(ci)]
     lib.dft3d_plan_destroy.argtypes = [vp]
     lib.dft3d_status_string.argtypes = [ci]
     lib.dft3d_status_string.restype = ctypes.c_char_p
@@ -252,6 +254,12 @@ class Plan:
     def split(self):
         """DFT3D_SPLIT_FP16 or DFT3D_SPLIT_TF32: the operand split of the plan's tensor-core products."""
         return int(_lib.dft3d_plan_split(self._h))
+
+    def fft_split(self, axis):
+        """(N1, N2) of Eq. 17 on `axis`: the lengths of the first and the second matrix product."""
+        n1, n2 = ctypes.c_int(0), ctypes.c_int(0)
+        _check(_lib.dft3d_plan_fft_split(self._h, int(axis), ctypes.byref(n1), ctypes.byref(n2)))
+        return n1.value, n2.value
 
     def destroy(self):
         if self._h:

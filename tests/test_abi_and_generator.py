@@ -53,7 +53,7 @@ def test_argument_validation_needs_no_gpu(dft):
         (dict(n=(64, 64, 64), nodes=(np.array([np.nan] * 64), None, None)), 1),
         (dict(n=(64, 64, 64), mode=1, nodes=(np.arange(64) / 64.0, None, None)), 2),
         (dict(n=(64, 64, 64), mode=3), 1),           # 0, 1, 2 (KDFT, FFT, AUTO) are the modes
-        (dict(n=(64, 64, 101), mode=2), 2),          # AUTO falls back to KDFT, which needs even lengths
+        (dict(n=(64, 64, 101), mode=2), 2),          # AUTO falls back to KDFT, which needs an even last axis
         (dict(n=(64, 64, 64), flags=4 | 8), 1),      # both operand splits at once
         (dict(n=(64, 64, 66), flags=4), 2),          # fp16 pieces need lengths that are multiples of 4
     ]
@@ -62,18 +62,20 @@ def test_argument_validation_needs_no_gpu(dft):
         with pytest.raises(dft.Dft3dError) as e:
             dft.Plan(*n, **kw)
         assert e.value.status == status, (n, kw, str(e.value))
-    # axis subsets: an untransformed axis 0 may have any length; the other axes still need multiples of 64
+    # KDFT: axes 0 and 1 may have any length, the last axis must be even (rows of the data start on 16-byte boundaries);
+    # FFT: every axis but an untransformed axis 0 needs a multiple of 64
     with pytest.raises(dft.Dft3dError) as e:
-        dft.Plan(3, 101, 64, axes=(1, 2))
-    assert e.value.status == 2
+        dft.Plan(4, 6, 101, axes=(0, 1))
+    assert e.value.status == 2 and "16-byte" in str(e.value)
     with pytest.raises(dft.Dft3dError) as e:
-        dft.Plan(3, 128, 64, axes=(0, 1, 2))      # axis 0 is transformed here: its length must be even
+        dft.Plan(3, 100, 256, mode=1, axes=(1, 2))
     assert e.value.status == 2
     import torch
     if not torch.cuda.is_available():
-        with pytest.raises(dft.Dft3dError) as e:
-            dft.Plan(3, 128, 64, axes=(1, 2))      # valid sizes: the first failure is the missing device
-        assert e.value.status == 4
+        for n, axes in (((3, 128, 64), (1, 2)), ((3, 101, 64), (0, 1, 2))):
+            with pytest.raises(dft.Dft3dError) as e:
+                dft.Plan(*n, axes=axes)            # valid sizes: the first failure is the missing device
+            assert e.value.status == 4
     from paper_2002_03260_b200 import dft3d as b
     assert b._lib.dft3d_plan_create(None, 64, 64, 64, 0, -1, None, None, None) == 1
     assert b._lib.dft3d_plan_destroy(None) == 0

@@ -136,3 +136,21 @@ def test_bounded_waits_give_up_and_report(lib, oracle, monkeypatch, mode_name, s
     for a in (axes or (0, 1, 2)):
         want = oracle.dft_axis(want, a)
     assert oracle.rel_l2(y.cpu().numpy(), want) < SANITY
+
+
+def test_fft_split_option_and_query(lib):
+    """fft_split names the factor pair {N1, N2} of Eq. 17 per axis.  The kernels realise one pair per length; that pair
+    is accepted (and is what {0, 0} selects), any other is refused, and the plan reports the pair it uses."""
+    shape = (256, 512, 256)
+    plan = lib.Plan(*shape, mode=lib.DFT3D_FFT, fft_split=[(16, 16), (32, 16), None])
+    assert [plan.fft_split(a) for a in range(3)] == [(16, 16), (32, 16), (16, 16)]
+    plan.destroy()
+    for bad in ([(8, 32), None, None], [None, (16, 32), None], [None, None, (16, 8)]):
+        with pytest.raises(lib.Dft3dError) as e:
+            lib.Plan(*shape, mode=lib.DFT3D_FFT, fft_split=bad)
+        assert e.value.status == 2
+    kd = lib.Plan(64, 64, 64)
+    with pytest.raises(lib.Dft3dError) as e:
+        kd.fft_split(0)
+    assert e.value.status == 1
+    kd.destroy()

@@ -738,10 +738,12 @@ def test_batched_1d_fft(lib, oracle):
 # ------------------------------------------------------------------ sizes that are not tile multiples (KDFT)
 
 @pytest.mark.parametrize("shape", [(100, 66, 250), (30, 18, 34), (2, 4, 6), (130, 64, 2), (66, 258, 64),
-                                   (100, 68, 36), (4, 132, 252), (260, 8, 12)])
+                                   (100, 68, 36), (4, 132, 252), (260, 8, 12),
+                                   (3, 5, 6), (129, 33, 64), (1, 7, 2), (5, 64, 130), (255, 1, 8)])
 def test_kdft_general_even_sizes(lib, oracle, shape):
-    """Any even length: ragged K stages are zero-filled by TMA on both operands, ragged tiles masked on store.
-    Shapes whose lengths are all multiples of 4 run the fp16 split, the others fall back to the TF32 split."""
+    """Any length on axes 0 and 1, any even length on the last axis: ragged K stages are zero-filled by TMA on both
+    operands, ragged tiles masked on store, and an odd length pads the rows of the TABLE to a 16-byte multiple (the
+    data is never padded).  Shapes whose lengths are all multiples of 4 run the fp16 split, the others the TF32 split."""
     x = _inputs().cube(shape, "normal", 91, device="cuda")
     guard = torch.full((1 << 14,), 7.0, device="cuda")           # canaries around the output
     out = torch.empty_like(x)
@@ -764,6 +766,15 @@ def test_kdft_general_even_sizes(lib, oracle, shape):
     _finish(plan)
     plan.destroy()
     assert oracle.rel_l2(y.cpu().numpy(), oracle.dft3d(x.cpu().numpy(), nodes=nodes)) < SANITY
+
+
+def test_kdft_refuses_an_odd_last_axis(lib):
+    """Rows of the data are 8*n2 bytes long and TMA needs them to start on 16-byte boundaries: an odd last axis is
+    refused with a message that says so, whether or not that axis is transformed."""
+    for axes in (None, (0, 1)):
+        with pytest.raises(lib.Dft3dError) as e:
+            lib.Plan(8, 6, 7, axes=axes)
+        assert e.value.status == 2 and "16-byte" in str(e.value)
 
 
 # ------------------------------------------------------------------ fp16 split: scaling by powers of two
