@@ -48,6 +48,13 @@ def parse_args():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing leg")
+    ap.add_argument("--config", type=str, default=None,
+                    help="c1..c5 or all: the five configurations the parity tests cover, one JSON line each (time, "
+                         "GFLOP/s in both conventions, issued tensor flops, roofline fraction, oracle seconds)")
+    ap.add_argument("--md", type=str, default=None, help="with --config: also write the lines as a markdown table here")
+    ap.add_argument("--traffic-from-ncu", nargs="+", default=None, metavar="KERNEL:POINTS:CSV",
+                    help="no GPU work: read dram__bytes_read/write.sum per launch of KERNEL from an `ncu --csv` log of a "
+                         "case with POINTS points per launch and write profiles/dram_bytes_per_point.json")
     return ap.parse_args()
 
 
@@ -57,17 +64,49 @@ def conv_flops(n):
     return 5.0 * P * math.log2(P)
 
 
-# DRAM bytes per point per launch (dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture divided by the
-# points of that launch; smaller cases than the bench workload, traffic grows in proportion to the points):
-#   profiles/fft_f16_axis_kernel_1024_dram.md     : the bench workload itself (one-pass capture of the three launches
-#                                                   at 1024^3), 51.68 GB / 3 launches / 1073.7 M points
-#   profiles/kdft_f16_axis_kernel_512.md          : mean of the three launches, (1.081 + 1.031) GB / 134.2 M points
-#   (the TF32-piece kernels, captured before: 15.80 and 15.79)
-NCU_DRAM_BYTES_PER_POINT = {"fft_axis_kernel": 15.80, "fft_f16_axis_kernel": 16.04, "kdft_axis_kernel": 15.79,
-                            "kdft_f16_axis_kernel": 15.73,
-                            # profiles/kdft_f16x2_axis_kernel_2048x128x128.md: (1.241 + 0.261) GB / 33.5 M points; the 64 MiB
-                            # table of a 2048-point axis is fetched again by every wave of tiles
-                            "kdft_f16x2_axis_kernel": 44.8}
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "dram_bytes_per_point.json")
+
+
+def dram_bytes_per_point(kernel):
+    """DRAM bytes per point and launch of `kernel` as ncu measured them (dram__bytes_read.sum + dram__bytes_write.sum
+    of a capture divided by the points of that launch; traffic grows in proportion to the points).  The file is
+    written by `bench.py --traffic-from-ncu` from the ncu logs; None when it has no entry for the kernel."""
+    try:
+        with open(TRAFFIC_FILE) as f:
+            entry = json.load(f).get(kernel)
+    except (OSError, ValueError):
+        return None, None
+    return (entry["bytes_per_point"], entry["case"]) if entry else (None, None)
+
+
+def traffic_from_ncu(specs):
+    """Parses `ncu --csv --metrics dram__bytes_read.sum,dram__bytes_write.sum ...` logs: mean bytes per launch of every
+    launch whose kernel name starts with KERNEL, divided by POINTS."""
+    import csv
+    out = {}
+    if os.path.exists(TRAFFIC_FILE):
+        with open(TRAFFIC_FILE) as f:
+            out = json.load(f)
+    for spec in specs:
+        kernel, points, path = spec.split(":", 2)
+        per_launch = {}
+        with open(path) as f:
+            rows = [r for r in csv.reader(f) if len(r) > 10]
+        hdr = rows[0]
+        ki, mi, vi, ii = hdr.index("Kernel Name"), hdr.index("Metric Name"), hdr.index("Metric Value"), hdr.index("ID")
+        for r in rows[1:]:
+            base = r[ki].replace("void ", "").split("<")[0].split("(")[0]
+            if base == kernel and r[mi] in ("dram__bytes_read.sum", "dram__bytes_write.sum"):
+                per_launch[r[ii]] = per_launch.get(r[ii], 0.0) + float(r[vi].replace(",", ""))
+        if not per_launch:
+            raise SystemExit("no launch of %s in %s" % (kernel, path))
+        mean = sum(per_launch.values()) / len(per_launch)
+        out[kernel] = {"bytes_per_point": mean / float(points), "launches": len(per_launch),
+                       "points_per_launch": int(points), "case": os.path.basename(path)}
+    with open(TRAFFIC_FILE, "w") as f:
+        json.dump(out, f, indent=1, sort_keys=True)
+        f.write("\n")
+    print(json.dumps(out))
 
 
 def measured_peaks():
@@ -194,10 +233,132 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+CONFIGS = {
+    # name: (shape, input recipe, what runs) -- the five configurations the parity tests cover
+    "c1": ((64, 64, 64), "uniform:1001", [("kdft", -1, False)]),
+    "c2": ((512, 512, 512), "normal:1002", [("kdft", -1, False), ("kdft", +1, False)]),
+    "c3": ((1024, 1024, 1024), "uniform:1003", [("fft", -1, False), ("kdft", -1, False)]),
+    "c4": ((256, 256, 256), "normal:1004", [("kdft", -1, True)]),
+    "c5": ((2048, 2048, 2048), "exponentials:2005:1005", [("fft", -1, False), ("kdft", -1, False)]),
+}
+
+
+def run_configs(args):
+    """--config: per configuration and formulation one JSON line: median and minimum time of a transform (CUDA events,
+    3 warm-up + `reps` timed transforms, one event pair each), GFLOP/s in the 5*P*log2(P) convention and by the
+    matrix-product flops the formulation defines (KDFT 8*n_a, FFT 8*(N1+N2) real flops per point and axis), the flops
+    the tensor cores actually issue (three split products; the FFT kernels' R*R core), the roofline fraction, and the
+    oracle's seconds on the host cores (whole transform where that takes under two minutes, else extrapolated from a
+    sample and labelled so)."""
+    import numpy as np
+    import torch
+    import paper_2002_03260_b200 as dft
+    from paper_2002_03260_b200 import inputs
+    from oracle import oracle
+    oracle.build()
+    torch.cuda.set_device(0)
+    peaks, peak_kind = measured_peaks()
+    names = sorted(CONFIGS) if args.config == "all" else [args.config]
+    lines = []
+    for name in names:
+        shape, recipe, runs = CONFIGS[name]
+        P = float(shape[0]) * shape[1] * shape[2]
+        if P * 8 * 2.3 > torch.cuda.mem_get_info()[0]:
+            sys.stderr.write("bench: %s does not fit this device, skipped\n" % name)
+            continue
+        kind = recipe.split(":")
+        if kind[0] == "exponentials":
+            x = inputs.exponentials(shape, 16, int(kind[1]), 1e-3, int(kind[2]), device="cuda")[0]
+        else:
+            x = inputs.cube(shape, kind[0], int(kind[1]), device="cuda")
+        y = torch.empty_like(x)
+        stream = torch.cuda.current_stream()
+        # the oracle beside it: whole transform up to 512^3, a sample beyond
+        n = shape[0]
+        if P <= 512 ** 3:
+            xh = x.cpu().numpy()
+            nodes_o = inputs.sorted_nodes(shape, 2004) if runs[0][2] else None
+            t0 = time.perf_counter()
+            oracle.dft3d(xh, nodes=nodes_o)
+            osec, okind = time.perf_counter() - t0, "whole transform"
+            del xh
+        else:
+            smp = oracle_sample(n, oracle_planes(n), 1003)
+            osec, okind = smp["seconds_per_transform_extrapolated"], "extrapolated from " + smp["sample"].split(";")[0]
+        for mode, sign, with_nodes in runs:
+            nodes = inputs.sorted_nodes(shape, 2004) if with_nodes else None
+            limit = 4 * 2 ** 30 if (mode == "kdft" and P * 8 > 32 * 2 ** 30) else 0
+            plan = dft.Plan(*shape, mode=dft.DFT3D_KDFT if mode == "kdft" else dft.DFT3D_FFT, sign=sign, nodes=nodes,
+                            workspace_limit=limit)
+            reps = 200 if P <= 64 ** 3 else (20 if P <= 1024 ** 3 else 3)
+            for _ in range(3):
+                plan.execute(x, y)
+            torch.cuda.synchronize()
+            sampler = ClockSampler(0)
+            sampler.start()
+            pairs = []
+            for _ in range(reps):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                plan.execute(x, y)
+                e1.record(stream)
+                pairs.append((e0, e1))
+            torch.cuda.synchronize()
+            clk = sampler.stop()
+            plan.status()
+            ms = sorted(a.elapsed_time(b) for a, b in pairs)
+            med, mn = ms[len(ms) // 2], ms[0]
+            f16 = plan.split == dft.DFT3D_SPLIT_FP16
+            if mode == "kdft":
+                gemm = 8.0 * sum(shape) * P
+                issued = 3.0 * gemm
+                peak = peaks["bf16_tflops_sustained"] * (1.0 if f16 else 1.1 / 2.25)
+                roof = {"bound": "tensor", "achieved": issued / (med * 1e-3) * 1e-12, "peak": peak, "unit": "TFLOP/s",
+                        "peak_source": "%s bf16 sustained%s" % (peak_kind, "" if f16 else " x 1.1/2.25 (TF32)")}
+            else:
+                splits = [plan.fft_split(a) for a in range(3)]
+                gemm = 8.0 * sum(a + b for a, b in splits) * P
+                issued = 3.0 * 8.0 * sum(2 * b for a, b in splits) * P
+                roof = {"bound": "hbm", "achieved": 48.0 * P / (med * 1e-3) * 1e-9, "peak": peaks["hbm_gbs"],
+                        "unit": "GB/s", "peak_source": "%s STREAM-style copy" % peak_kind}
+            roof["frac"] = roof["achieved"] / roof["peak"]
+            line = {"config": name, "shape": list(shape), "formulation": mode, "sign": sign, "nonuniform": with_nodes,
+                    "split": "fp16" if f16 else "tf32", "launches": plan.launches, "reps": reps,
+                    "ms_median": med, "ms_min": mn,
+                    "gflops_5PlogP": conv_flops(shape) / (med * 1e-3) * 1e-9,
+                    "gflops_gemm": gemm / (med * 1e-3) * 1e-9, "tflops_issued_tensor": issued / (med * 1e-3) * 1e-12,
+                    "roofline": roof, "clocks": clk,
+                    "oracle_seconds": osec, "oracle_kind": okind, "oracle_cores": oracle.num_threads()}
+            print(json.dumps(line), flush=True)
+            lines.append(line)
+            plan.destroy()
+        del x, y
+        torch.cuda.empty_cache()
+    if args.md:
+        with open(args.md, "w") as f:
+            f.write("| config | shape | formulation | split | launches | median ms | min ms | GFLOP/s (5P log2 P) | GFLOP/s "
+                    "(matrix-product flops) | issued tensor TFLOP/s | roofline | SM MHz | oracle s (cores) |\n")
+            f.write("|---|---|---|---|---|---|---|---|---|---|---|---|---|\n")
+            for d in lines:
+                r = d["roofline"]
+                f.write("| %s | %s | %s%s%s | %s | %d | %.4g | %.4g | %.4g | %.4g | %.4g | %.2f of %s (%.4g of %.4g %s) | %s | %.4g (%d), %s |\n"
+                        % (d["config"], "x".join(str(v) for v in d["shape"]), d["formulation"],
+                           " inverse" if d["sign"] > 0 else "", " nonuniform" if d["nonuniform"] else "", d["split"],
+                           d["launches"], d["ms_median"], d["ms_min"], d["gflops_5PlogP"], d["gflops_gemm"],
+                           d["tflops_issued_tensor"], r["frac"], r["bound"], r["achieved"], r["peak"], r["unit"],
+                           d["clocks"].get("sm_mhz"), d["oracle_seconds"], d["oracle_cores"], d["oracle_kind"]))
+
+
 def main():
     args = parse_args()
+    if args.traffic_from_ncu:
+        traffic_from_ncu(args.traffic_from_ncu)
+        return
     if args.impl == "reference":
         run_reference(args)
+        return
+    if args.config:
+        run_configs(args)
         return
     import torch
     import torch.distributed as dist
@@ -333,9 +494,10 @@ def main():
                 src = "%s bf16 sustained x nominal TF32/bf16 ratio (1.1/2.25)" % peak_kind
                 axis_launches = nlaunch
             return {"bound": "tensor", "kernel": kernel, "achieved": ach, "peak": peak, "unit": "TFLOP/s",
-                    "frac": ach / peak, "traffic": NCU_DRAM_BYTES_PER_POINT[kernel] * P,
-                    "traffic_note": "DRAM bytes per launch, ncu capture at %s scaled by points (algorithmic: 16 B/point)"
-                                    % ("2048x128x128" if kernel == "kdft_f16x2_axis_kernel" else "512^3"),
+                    "frac": ach / peak,
+                    "traffic": (dram_bytes_per_point(kernel)[0] or 0.0) * P or None,
+                    "traffic_note": "DRAM bytes per launch, ncu capture (%s) scaled by points (algorithmic: 16 B/point)"
+                                    % dram_bytes_per_point(kernel)[1],
                     "peak_source": src,
                     "flops": "issued tensor flops = 3 split products x 8*n_a flops per point per axis",
                     "useful_gemm_tflops": algo_flops / (ms * 1e-3) * 1e-12, "avg_launch_ms": ms / axis_launches}
@@ -349,9 +511,10 @@ def main():
             fkernel = "fft_f16_axis_kernel" if psplit == dft.DFT3D_SPLIT_FP16 else "fft_axis_kernel"
             roofline = {"bound": "hbm", "kernel": fkernel, "achieved": achieved, "peak": peaks["hbm_gbs"],
                         "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
-                        "traffic": NCU_DRAM_BYTES_PER_POINT[fkernel] * P,
-                        "traffic_note": "DRAM bytes per launch, one-pass ncu capture at 1024^3 (mean of the three launches)"
-                                        + ("" if shape == (1024, 1024, 1024) else " scaled by points"),
+                        "traffic": (dram_bytes_per_point(fkernel)[0] or 0.0) * P or None,
+                        "traffic_note": "DRAM bytes per launch, ncu capture (%s) scaled by points"
+                                        % dram_bytes_per_point(fkernel)[1],
+                        "bytes_per_point_algorithmic": 16.0 * len(taxes),
                         "peak_source": "%s STREAM-style copy" % peak_kind, "avg_launch_ms": ms_step / launches,
                         "bytes": "8 B read + 8 B written per point per axis pass"}
         if kdft_info is not None:
