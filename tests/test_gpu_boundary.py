@@ -154,3 +154,23 @@ def test_fft_split_option_and_query(lib):
         kd.fft_split(0)
     assert e.value.status == 1
     kd.destroy()
+
+
+@pytest.mark.parametrize("sign", [-1, +1])
+def test_ring_blocks_of_axis0_on_the_gpu_kernels(lib, oracle, sign):
+    """The per-rank block product of the one-shuffle ring (a square nonuniform-node plan per source rank and a phase
+    on the input rows) is a function of (rank, source rank) alone: summing it over the source ranks, rank by rank in
+    this one process with no exchange, must give each rank's slab of the axis-0 transform."""
+    from paper_2002_03260_b200 import sharded
+    n0, n1, n2, world = 256, 64, 64, 4
+    b = n0 // world
+    x = _inputs().cube((n0, n1, n2), "normal", 210, device="cuda")
+    want = oracle.dft_axis(x.cpu().numpy().astype(np.complex128), 0, sign=sign, scale=(1.0 / n0 if sign > 0 else 1.0))
+    for rank in (0, 3):
+        _, block_product = sharded.gpu_transforms(n0, n1, n2, rank, world, "kdft", sign=sign)
+        acc = None
+        for src in range(world):
+            part = block_product(x[src * b:(src + 1) * b].contiguous(), src)
+            acc = part if acc is None else acc + part
+        torch.cuda.synchronize()
+        assert oracle.rel_l2(acc.cpu().numpy(), want[rank * b:(rank + 1) * b]) < SANITY
