@@ -418,7 +418,7 @@ def main():
         plan = None
     kdft_info = None
     if mode == "fft" and not args.no_kdft:
-        ksteps = max(1, min(args.steps, 3))
+        ksteps = max(1, min(args.steps, 10 if n <= 1024 else 3))
         kplan, kms, kclk = time_mode("kdft", ksteps, 3, True)
         kdft_info = {"ms_per_step": kms, "steps": ksteps, "warmup": 3, "launches_per_step": kplan.launches,
                      "split": "fp16" if kplan.split == dft.DFT3D_SPLIT_FP16 else "tf32", "clocks": kclk}
