@@ -11,7 +11,8 @@
  *   FFT  (Section III-B, Eq. 14-18): every axis of length N = N1*N2 becomes a
  *        length-N1 DFT (matrix product), an elementwise phase adjustment
  *        (twiddle), and a length-N2 DFT (matrix product); output in natural
- *        order.  Uniform grids only.
+ *        order.  Uniform grids only.  (Lengths above 1024 apply Eq. 17 once
+ *        more, with a factor 2, 4 or 8 whose small DFT runs on the CUDA cores.)
  *
  * Data layout everywhere: row-major [n0][n1][n2], interleaved complex64
  * (re, im as two float32), 8 bytes per point.
@@ -77,7 +78,8 @@ typedef struct dft3d_options_s {
                              {0,0} = the built-in split, which is also the only one the kernels realise: N2 = 16 for
                              n_a = 256 and 512, N2 = 32 from 1024 on, N1 = n_a / N2 (256 = 16*16, 512 = 32*16,
                              1024 = 32*32, 2048 = 64*32, 4096 = 128*32; an N1 above N2 is itself computed as
-                             (N1/N2) * N2 by one more application of Eq. 17).  Any other pair returns
+                             (N1/N2) * N2 by one more application of Eq. 17; 8192 = 1024*8, the 1024 again 32*32).
+                             Any other pair returns
                              DFT3D_ERR_UNSUPPORTED; dft3d_plan_fft_split reports the pair in use. */
   size_t workspace_limit; /* upper bound in bytes for the plan-owned workspace; 0 = default (16 GiB).  KDFT needs a
                              workspace and shrinks it to groups of n0-planes.  FFT uses one cube of workspace when it
@@ -113,8 +115,10 @@ typedef struct dft3d_options_s {
  * Supported sizes: KDFT: n0 and n1 of any length, n2 even (rows of the data must start on 16-byte boundaries),
  * transformed n_a <= 8192 (tiles that are not full are zero-filled on load and masked on store, and an odd length pads
  * the rows of the table, the way the paper's compiler pads to its hardware's preferred shapes).  FFT: every
- * transformed n_a in {256, 512, 1024, 2048, 4096} (N = R*R, 2*R*R or 4*R*R with R = 16 or 32; 4096 with fp16
- * pieces only), the others multiples of 64.
+ * transformed n_a in {256, 512, 1024, 2048, 4096, 8192} (N = R*R, 2*R*R or 4*R*R with R = 16 or 32, and 8192 = 1024*8;
+ * 4096 and 8192 with fp16 pieces only), the others multiples of 64.  An 8192-point axis takes two launches (the fused
+ * 1024-point kernel over the eight stride-8 sub-sequences, then the phase adjustment and the 8-point DFT), and a plan
+ * that has one owns a cube of workspace and runs its axes one after the other in the natural layout.
  * Other sizes return DFT3D_ERR_UNSUPPORTED.
  */
 int dft3d_plan_create(dft3d_plan_t* out, long long n0, long long n1, long long n2, int mode, int sign,

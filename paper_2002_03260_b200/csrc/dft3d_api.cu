@@ -21,6 +21,7 @@
 #include "fft_f16_kernel.cuh"
 #include "kdft_f16x2_kernel.cuh"
 #include "fft_kernel.cuh"
+#include "radix8_kernel.cuh"
 
 namespace {
 
@@ -177,6 +178,10 @@ struct FftAxis {
   float2* d_tw2 = nullptr; // RX == 2: exp(s*2*pi*i*m/n), m < R*R
   float out_mul = 1.0f;    // fp16 pieces: the factor the store applies (powers of two, 1/n for a scaled inverse)
   CUtensorMap map_w;
+  // 8192-point axis = 1024 x 8 (Eq. 17 once more): the fused kernel transforms the eight stride-8 sub-sequences (n = 1024
+  // above), a second launch applies the phase adjustment and the 8-point DFT (radix8_kernel.cuh)
+  bool r8 = false;
+  float2* d_tw8 = nullptr; // [1024][8] complex64, exp(s*2*pi*i*k1*beta/8192), times 1/8 for a scaled inverse
 };
 
 }  // namespace
@@ -556,7 +561,21 @@ int prepare_scales(dft3d_plan_s* p, const float* in, cudaStream_t stream) {
 // once to complex64.  The 1/n of a scaled inverse is 1/R in each stage's matrix and 1/RX in the twiddles.
 int build_fft_axis(dft3d_plan_s* p, int a, const int split[2]) {
   FftAxis& ax = p->fax[a];
-  const long long n = p->n[a];
+  long long n = p->n[a];
+  const bool scaled = (p->sign > 0) && !(p->flags & DFT3D_UNSCALED_INVERSE);
+  if (n == 8192 && p->f16) {
+    // 8192 = 1024 * 8: tables of the 1024-point kernel, and the phase adjustment between the two steps
+    if ((split[0] || split[1]) && (split[0] != 1024 || split[1] != 8))
+      return fail(DFT3D_ERR_UNSUPPORTED, "FFT split %dx%d for n%d = 8192 is not supported (only 1024x8)", split[0], split[1], a);
+    ax.r8 = true;
+    n = 1024;
+    std::vector<double> T(size_t(2) * 1024 * 8);
+    std::vector<float> t8(T.size());
+    dft3d::gen::twiddle(1024, 8, p->sign, T.data());
+    for (size_t i = 0; i < T.size(); ++i) t8[i] = float(T[i] * (scaled ? 0.125 : 1.0));
+    DFT3D_CUDA(cudaMalloc(&ax.d_tw8, t8.size() * sizeof(float)));
+    DFT3D_CUDA(cudaMemcpy(ax.d_tw8, t8.data(), t8.size() * sizeof(float), cudaMemcpyHostToDevice));
+  }
   int R = 0, RX = 1;
   if (n == 256) { R = 16; }
   if (n == 512) { R = 16; RX = 2; }
@@ -564,9 +583,9 @@ int build_fft_axis(dft3d_plan_s* p, int a, const int split[2]) {
   if (n == 2048) { R = 32; RX = 2; }
   if (n == 4096 && p->f16) { R = 32; RX = 4; }   // three factors: 4 * 32 * 32 (fp16-piece kernel only)
   if (!R)
-    return fail(DFT3D_ERR_UNSUPPORTED, "FFT mode supports axis lengths 256, 512, 1024, 2048 and (fp16 pieces) 4096; "
+    return fail(DFT3D_ERR_UNSUPPORTED, "FFT mode supports axis lengths 256, 512, 1024, 2048 and (fp16 pieces) 4096 and 8192; "
                 "n%d = %lld", a, n);
-  if ((split[0] || split[1]) && (split[0] != RX * R || split[1] != R))
+  if (!ax.r8 && (split[0] || split[1]) && (split[0] != RX * R || split[1] != R))
     return fail(DFT3D_ERR_UNSUPPORTED, "FFT split %dx%d for n%d = %lld is not supported (only %dx%d)", split[0],
                 split[1], a, n, RX * R, R);
   ax.n = n;
@@ -574,7 +593,6 @@ int build_fft_axis(dft3d_plan_s* p, int a, const int split[2]) {
   ax.RX = RX;
   ax.cols = (R == 32 && RX == 4) ? 4 : ((R == 32 && RX == 2) ? 8 : 16);   // a 128 KB stage holds all n rows of `cols` lines
                                                                            // (fft_axis_pass may pick 8 for R = 32, RX = 1)
-  const bool scaled = (p->sign > 0) && !(p->flags & DFT3D_UNSCALED_INVERSE);
   const int K = 2 * R, NB = 2 * R, panels = K / 32;
   if (p->f16) {
     // fp16 pieces: 1024 * F_R (real form), rows of 64 halves (zero-padded for R = 16), [hi piece; lo piece]; the twiddle
@@ -709,13 +727,20 @@ struct FftCapture {
   dft3d::FftF16Params hp;
 };
 
+// A strided pass over an explicit view [batches][N][C] (natural layout) with the tables of `axis`: the first step of an
+// 8192-point axis, whose eight stride-8 sub-sequences are eight times as many columns of 1024-point lines.
+struct FftView {
+  long long batches, C;
+  int cols;              // lines per stage: 16, or 8 when the view has only eight columns
+};
+
 // map_rows != 0 (axis 2 only): the input is a ring of that many lines (the tensor map covers just them).
 int fft_axis_pass(dft3d_plan_s* p, int axis, const float* in, float* out, cudaStream_t stream,
                   int layout = FFT_NATURAL, long long n2_off = 0, long long n2_sub = 0, long long map_rows = 0,
-                  FftCapture* capture = nullptr) {
+                  FftCapture* capture = nullptr, const FftView* view = nullptr) {
   const FftAxis& ax = p->fax[axis];
   const int R = ax.R, RX = ax.RX, N = int(ax.n), Lg = 128 / (R * RX);
-  const int cols = fft_cols_for(p, axis, layout);
+  const int cols = view ? view->cols : fft_cols_for(p, axis, layout);
   dft3d::FftParams fp;
   memset(&fp, 0, sizeof(fp));
   fp.N = N;
@@ -730,8 +755,8 @@ int fft_axis_pass(dft3d_plan_s* p, int axis, const float* in, float* out, cudaSt
   int rc;
   int stage_out = 0;
   const Knobs& kn = p->knobs;
-  const int tag_in = 0x200 + axis * 8 + layout, tag_out = 0x300 + axis * 8 + layout;
-  if (axis == 2) {
+  const int tag_in = 0x200 + axis * 8 + layout + (view ? 0x40 : 0), tag_out = 0x300 + axis * 8 + layout + (view ? 0x40 : 0);
+  if (axis == 2 && !view) {
     const long long rows = p->n[0] * p->n[1];
     fp.rows = rows;
     fp.mtiles_per_stage = 1;
@@ -745,10 +770,10 @@ int fft_axis_pass(dft3d_plan_s* p, int axis, const float* in, float* out, cudaSt
     });
     map_out = map_data;   // unused on this axis
   } else {
-    const long long batches = (axis == 0) ? 1 : p->n[0];
+    const long long batches = view ? view->batches : ((axis == 0) ? 1 : p->n[0]);
     const long long n2v = n2_sub ? n2_sub : p->n[2];                            // columns of the last axis this pass covers
-    const long long C = (axis == 0) ? p->n[1] * n2v : n2v;                      // columns per batch of this pass
-    const long long Cmap = (axis == 0) ? p->n[1] * p->n[2] : p->n[2];           // columns per batch of the full array
+    const long long C = view ? view->C : ((axis == 0) ? p->n[1] * n2v : n2v);   // columns per batch of this pass
+    const long long Cmap = view ? view->C : ((axis == 0) ? p->n[1] * p->n[2] : p->n[2]);   // columns per batch of the full array
     if (n2_sub && (!p->f16 || layout == FFT_NATURAL)) return fail(DFT3D_ERR_UNSUPPORTED, "internal: sliced pass");
     fp.C = C;
     fp.out_pitch = (n2_sub && layout == FFT_IN_BLOCKED) ? Cmap : C;
@@ -860,7 +885,7 @@ int fft_axis_pass(dft3d_plan_s* p, int axis, const float* in, float* out, cudaSt
 #define DFT3D_FFT16_LAUNCH(MODE, R_, RX_, COLS_, SO_)                                         \
   dft3d::fft_f16_axis_kernel<MODE, R_, RX_, COLS_, SO_>                                        \
       <<<grid, dft3d::kFftThreads, smem, stream>>>(map_data, ax.map_w, map_out, hp)
-    if (axis == 2) {
+    if (axis == 2 && !view) {
       if (R == 32 && RX == 1) DFT3D_FFT16_LAUNCH(dft3d::FFT_CONTIG, 32, 1, 16, 0);
       else if (R == 16 && RX == 1) DFT3D_FFT16_LAUNCH(dft3d::FFT_CONTIG, 16, 1, 16, 0);
       else if (R == 32 && RX == 4) DFT3D_FFT16_LAUNCH(dft3d::FFT_CONTIG, 32, 4, 16, 0);
@@ -920,6 +945,39 @@ int fft_axis_pass(dft3d_plan_s* p, int axis, const float* in, float* out, cudaSt
     else DFT3D_FFT_LAUNCH(dft3d::FFT_STRIDED, 16, 2, 16, 2, 1);
   }
 #undef DFT3D_FFT_LAUNCH
+  DFT3D_CUDA(cudaGetLastError());
+  return DFT3D_OK;
+}
+
+// The two launches of an 8192-point axis (see FftAxis::r8), natural layout: src -> mid -> dst (three distinct cubes, or
+// mid == the caller's scratch).  lines = product of the dimensions before the axis, C = columns behind it.
+void r8_geometry(const dft3d_plan_s* p, int axis, long long* lines, long long* C) {
+  *lines = axis == 0 ? 1 : (axis == 1 ? p->n[0] : p->n[0] * p->n[1]);
+  *C = axis == 0 ? p->n[1] * p->n[2] : (axis == 1 ? p->n[2] : 1);
+}
+
+int fft_r8_first(dft3d_plan_s* p, int axis, const float* src, float* mid, cudaStream_t stream) {
+  long long lines, C;
+  r8_geometry(p, axis, &lines, &C);
+  FftView v;
+  v.batches = lines;
+  v.C = 8 * C;                       // sub-sequence beta of column c is column beta*C + c of the 1024-point lines
+  v.cols = (8 * C) % 16 == 0 ? 16 : 8;
+  return fft_axis_pass(p, axis, src, mid, stream, FFT_NATURAL, 0, 0, 0, nullptr, &v);
+}
+
+int fft_r8_second(dft3d_plan_s* p, int axis, const float* mid, float* dst, cudaStream_t stream) {
+  dft3d::Radix8Params rp;
+  rp.in = reinterpret_cast<const float2*>(mid);
+  rp.out = reinterpret_cast<float2*>(dst);
+  rp.tw = p->fax[axis].d_tw8;
+  r8_geometry(p, axis, &rp.lines, &rp.C);
+  rp.sign = float(p->sign);
+  const long long total = rp.lines * 1024 * rp.C;
+  long long blocks = (total + dft3d::kRadix8Threads - 1) / dft3d::kRadix8Threads;
+  const long long cap = (long long)p->sm_count * 32;
+  if (blocks > cap) blocks = cap;
+  dft3d::fft_radix8_kernel<<<int(blocks), dft3d::kRadix8Threads, 0, stream>>>(rp);
   DFT3D_CUDA(cudaGetLastError());
   return DFT3D_OK;
 }
@@ -1109,7 +1167,9 @@ int dft3d_plan_create_ex(dft3d_plan_t* out, long long n0, long long n1, long lon
       if (!((axes >> a) & 1u)) { if (a != 0 && nn[a] % 64 != 0) fft_sizes_ok = false; continue; }
       const long long n = nn[a];
       const bool length_ok = n == 256 || n == 512 || n == 1024 || n == 2048 || (n == 4096 && f16);
-      const bool fft_ok = !nodes[a] && length_ok && inner[a] % 16 == 0;
+      // (8192 points: the first launch sees eight times as many columns, so an even count, or the last axis, will do)
+      const bool fft_ok = !nodes[a] && ((length_ok && inner[a] % 16 == 0) ||
+                                        (n == 8192 && f16 && (a == 2 || inner[a] % 2 == 0)));
       amode[a] = fft_ok ? DFT3D_FFT : DFT3D_KDFT;
       (fft_ok ? all_kdft : all_fft) = false;
       if (nn[a] % 64 != 0) fft_sizes_ok = false;
@@ -1119,6 +1179,11 @@ int dft3d_plan_create_ex(dft3d_plan_t* out, long long n0, long long n1, long lon
     if (mode != DFT3D_AUTO)
       for (int a = 0; a < 3; ++a) amode[a] = mode;
   }
+  // An 8192-point FFT axis takes two launches (FftAxis::r8); plans that have one run the axes one after the other in
+  // the natural layout, like plans that mix the formulations
+  if (mode == DFT3D_FFT)
+    for (int a = 0; a < 3; ++a)
+      if (((axes >> a) & 1u) && nn[a] == 8192) mode = DFT3D_AUTO;
 
   int ndev = 0;
   if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev < 1) return fail(DFT3D_ERR_CUDA, "no CUDA device available");
@@ -1159,11 +1224,11 @@ int dft3d_plan_create_ex(dft3d_plan_t* out, long long n0, long long n1, long lon
     if (e != cudaSuccess) { rc = fail(DFT3D_ERR_ALLOC, "cudaMalloc(amax): %s", cudaGetErrorString(e)); break; }
     if (mode == DFT3D_AUTO) {
       // both formulations in one plan: every pass goes from one cube to another in the natural layout
-      int count = 0;
+      int count = 0;   // passes: one per axis, two for an 8192-point FFT axis
       for (int a = 0; a < 3 && rc == DFT3D_OK; ++a)
         if ((axes >> a) & 1u) {
-          ++count;
           rc = amode[a] == DFT3D_FFT ? build_fft_axis(p, a, opt.fft_split[a]) : build_kdft_axis(p, a, nodes[a]);
+          count += (amode[a] == DFT3D_FFT && p->fax[a].r8) ? 2 : 1;
         }
       if (rc != DFT3D_OK) break;
       p->group_planes = n0;
@@ -1173,7 +1238,7 @@ int dft3d_plan_create_ex(dft3d_plan_t* out, long long n0, long long n1, long lon
         // Three passes go in -> out -> workspace -> out, so the input may serve as the workspace once the first pass
         // has read it.  Two passes go in -> workspace -> out: the first would run in place on the input, which a KDFT
         // pass cannot (every output tile re-reads whole lines), so two-axis plans allocate their workspace.
-        if ((opt.flags & DFT3D_DESTROY_INPUT) && count == 3) {
+        if ((opt.flags & DFT3D_DESTROY_INPUT) && count >= 3 && count % 2 == 1) {
           p->in_is_ws = true;
         } else if (cube_bytes > limit) {
           rc = fail(DFT3D_ERR_UNSUPPORTED, "a plan that mixes the formulations needs a workspace as large as the cube "
@@ -1300,6 +1365,11 @@ int dft3d_execute_axis(dft3d_plan_t p, int axis, const void* in, void* out, void
     if ((rc = prepare_scales(p, static_cast<const float*>(in), stream)) != DFT3D_OK) return rc;
     return kdft_axis_pass(p, axis, static_cast<const float*>(in), static_cast<float*>(out), p->n[0], stream, 0);
   }
+  if (p->fax[axis].r8) {
+    if (!p->workspace) return fail(DFT3D_ERR_UNSUPPORTED, "an 8192-point FFT axis alone needs the plan's workspace, which this plan does not own");
+    if ((rc = fft_r8_first(p, axis, static_cast<const float*>(in), static_cast<float*>(p->workspace), stream)) != DFT3D_OK) return rc;
+    return fft_r8_second(p, axis, static_cast<const float*>(p->workspace), static_cast<float*>(out), stream);
+  }
   return fft_axis_pass(p, axis, static_cast<const float*>(in), static_cast<float*>(out), stream);
 }
 
@@ -1314,7 +1384,10 @@ int dft3d_execute(dft3d_plan_t p, const void* in, void* out, void* cuda_stream) 
     // mixed formulations: axis 0, 1, 2 in turn, natural layout throughout, alternating between the cubes so that the
     // last pass writes `out` (three passes: in -> out -> workspace -> out; two: in -> workspace -> out)
     float* ws = p->in_is_ws ? const_cast<float*>(fin) : static_cast<float*>(p->workspace);
-    int remaining = int((axes & 1u) + ((axes >> 1) & 1u) + ((axes >> 2) & 1u));
+    // the passes: one per axis, two for an 8192-point FFT axis
+    int remaining = 0;
+    for (int a = 0; a < 3; ++a)
+      if ((axes >> a) & 1u) remaining += (p->amode[a] == DFT3D_FFT && p->fax[a].r8) ? 2 : 1;
     if (p->f16) DFT3D_CUDA(cudaMemsetAsync(p->d_amax, 0, 4 * sizeof(unsigned int), stream));
     const float* src = fin;
     int pos = 0;
@@ -1322,6 +1395,16 @@ int dft3d_execute(dft3d_plan_t p, const void* in, void* out, void* cuda_stream) 
     for (int a = 0; a < 3; ++a) {
       if (!((axes >> a) & 1u)) continue;
       float* dst = (remaining % 2 == 1) ? fout : ws;
+      if (p->amode[a] == DFT3D_FFT && p->fax[a].r8) {
+        float* dst2 = (remaining % 2 == 1) ? ws : fout;   // the second launch's target: the other cube
+        if ((rc = fft_r8_first(p, a, src, dst, stream)) != DFT3D_OK) return rc;
+        if ((rc = fft_r8_second(p, a, dst, dst2, stream)) != DFT3D_OK) return rc;
+        src = dst2;
+        remaining -= 2;
+        ++pos;
+        have_amax = false;
+        continue;
+      }
       if (p->amode[a] == DFT3D_FFT) {
         if ((rc = fft_axis_pass(p, a, src, dst, stream)) != DFT3D_OK) return rc;
         have_amax = false;
@@ -1502,7 +1585,7 @@ int dft3d_plan_launches(dft3d_plan_t p) {
     bool have_amax = false;
     for (int a = 0; a < 3; ++a) {
       if (!((p->axes >> a) & 1u)) continue;
-      if (p->amode[a] == DFT3D_FFT) { ++launches; have_amax = false; }
+      if (p->amode[a] == DFT3D_FFT) { launches += p->fax[a].r8 ? 2 : 1; have_amax = false; }
       else { launches += (p->f16 && !have_amax) ? 2 : 1; have_amax = true; }
     }
     return launches;
@@ -1525,8 +1608,8 @@ int dft3d_plan_fft_split(dft3d_plan_t p, int axis, int* n1, int* n2) {
   if (!p || !n1 || !n2) return fail(DFT3D_ERR_INVALID_ARG, "plan, n1 and n2 must not be NULL");
   if (axis < 0 || axis > 2 || !((p->axes >> axis) & 1u) || p->amode[axis] != DFT3D_FFT)
     return fail(DFT3D_ERR_INVALID_ARG, "axis %d is not transformed in the FFT formulation by this plan", axis);
-  *n1 = p->fax[axis].RX * p->fax[axis].R;
-  *n2 = p->fax[axis].R;
+  *n1 = p->fax[axis].r8 ? 1024 : p->fax[axis].RX * p->fax[axis].R;
+  *n2 = p->fax[axis].r8 ? 8 : p->fax[axis].R;
   return DFT3D_OK;
 }
 
@@ -1537,6 +1620,7 @@ int dft3d_plan_destroy(dft3d_plan_t p) {
     if (p->fax[a].d_w) cudaFree(p->fax[a].d_w);
     if (p->fax[a].d_tw) cudaFree(p->fax[a].d_tw);
     if (p->fax[a].d_tw2) cudaFree(p->fax[a].d_tw2);
+    if (p->fax[a].d_tw8) cudaFree(p->fax[a].d_tw8);
   }
   if (p->workspace) cudaFree(p->workspace);
   if (p->ring) cudaFree(p->ring);

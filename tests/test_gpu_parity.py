@@ -948,6 +948,74 @@ def test_2d_kdft_8192_squared_separable_input(lib, oracle):
     assert err < SANITY, err
 
 
+@pytest.mark.parametrize("shape,axis", [((4, 64, 8192), 2), ((2, 8192, 64), 1), pytest.param((8192, 64, 64), 0, marks=pytest.mark.slow)])
+def test_fft_8192_point_axis(lib, oracle, shape, axis):
+    """8192 = 1024 * 8 (Eq. 17 once more): the fused 1024-point kernel over the eight stride-8 sub-sequences, then the
+    phase adjustment and the 8-point DFT in a second launch.  Each axis alone against the oracle, forward and scaled
+    inverse; the plan reports the factor pair."""
+    x = _inputs().cube(shape, "normal", 110 + axis, device="cuda")
+    xh = x.cpu().numpy().astype(np.complex128)
+    for sign in (lib.DFT3D_FORWARD, lib.DFT3D_INVERSE):
+        plan = lib.Plan(*shape, mode=lib.DFT3D_FFT, sign=sign, axes=(axis,))
+        assert plan.launches == 2 and plan.fft_split(axis) == (1024, 8)
+        y = plan(x)
+        _finish(plan)
+        ya = plan.execute_axis(axis, x)
+        _finish(plan)
+        plan.destroy()
+        assert torch.equal(y, ya)
+        want = oracle.dft_axis(xh, axis, sign=sign, scale=(1.0 / 8192 if sign > 0 else 1.0))
+        assert oracle.rel_l2(y.cpu().numpy(), want) < SANITY_AXIS, (axis, sign)
+
+
+@pytest.mark.slow
+def test_2d_fft_8192_squared_matches_kdft_and_separable_input(lib, oracle):
+    """The paper's 2D workload (Section V-A, 8192 x 8192) in the FFT formulation: four launches.  Against the sum of
+    outer products of 1D oracle transforms (as the KDFT test above), against the KDFT plan, and AUTO picks it."""
+    n = 8192
+    rng = np.random.default_rng(112)
+    a = (rng.standard_normal((3, n)) + 1j * rng.standard_normal((3, n)))
+    b = (rng.standard_normal((3, n)) + 1j * rng.standard_normal((3, n)))
+    x = torch.from_numpy(np.einsum("ij,ik->jk", a, b).astype(np.complex64)).reshape(1, n, n).cuda()
+    fa = np.stack([oracle.dft_axis(a[i].reshape(1, 1, n), 2).reshape(n) for i in range(3)])
+    fb = np.stack([oracle.dft_axis(b[i].reshape(1, 1, n), 2).reshape(n) for i in range(3)])
+    ref = np.einsum("ij,ik->jk", fa, fb)
+    plan = lib.Plan(1, n, n, mode=lib.DFT3D_FFT, axes=(1, 2))
+    assert plan.launches == 4 and plan.workspace_bytes == x.numel() * 8
+    y = plan(x)
+    _finish(plan)
+    plan.destroy()
+    got = y.cpu().numpy().reshape(n, n).astype(np.complex128)
+    assert np.linalg.norm(got - ref) / np.linalg.norm(ref) < SANITY
+    kd = lib.Plan(1, n, n, axes=(1, 2))
+    z = kd(x)
+    _finish(kd)
+    kd.destroy()
+    assert _rel_l2_gpu(y, z) < SANITY
+    auto = lib.Plan(1, n, n, mode=lib.DFT3D_AUTO, axes=(1, 2))
+    assert auto.launches == 4
+    w = auto(x)
+    _finish(auto)
+    auto.destroy()
+    assert torch.equal(w, y)
+
+
+def test_fft_8192_with_other_axes_and_destroy_input(lib, oracle):
+    """An 8192-point axis beside a 256-point axis: three launches through the plan's own cube, against the oracle."""
+    shape = (2, 256, 8192)
+    x = _inputs().cube(shape, "uniform", 113, device="cuda")
+    plan = lib.Plan(*shape, mode=lib.DFT3D_FFT, axes=(1, 2))
+    assert plan.launches == 3
+    y = plan(x)
+    _finish(plan)
+    plan.destroy()
+    want = _oracle_axes(oracle, x.cpu().numpy(), (1, 2))
+    assert oracle.rel_l2(y.cpu().numpy(), want) < SANITY
+    with pytest.raises(lib.Dft3dError) as e:
+        lib.Plan(*shape, mode=lib.DFT3D_FFT, axes=(1, 2), flags=lib.DFT3D_SPLIT_TF32)
+    assert e.value.status == 2
+
+
 # ------------------------------------------------------------------ inverse nonuniform transform
 
 @pytest.mark.parametrize("split", SPLITS)
