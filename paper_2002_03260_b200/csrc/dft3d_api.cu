@@ -463,7 +463,8 @@ int launch_kdft_strided(dft3d_plan_s* p, int a, const float* in, float* out, lon
   int rc = cached_map(p, &map_data, 0x100 + a, in, batches, C, [&](CUtensorMap* m) {
     const unsigned long long dims[3] = {(unsigned long long)(2 * C), (unsigned long long)J, (unsigned long long)batches};
     const unsigned long long strides[2] = {(unsigned long long)(C * 8), (unsigned long long)(J * C * 8)};
-    const unsigned box[3] = {unsigned(2 * kp.lpb), unsigned((f16 ? dft3d::kF16BlockK : dft3d::kBlockK) / 2), unsigned(kp.bpt)};
+    // rows j per box: a whole stage for the paired-CTA kernel (32), half a stage for the one-CTA fp16 kernel, a TF32 stage (16)
+    const unsigned box[3] = {unsigned(2 * kp.lpb), unsigned((f16 && ax.pair) ? dft3d::kF16BlockK / 2 : 16), unsigned(kp.bpt)};
     return encode_f32(m, in, 3, dims, strides, box, 0, -1, p->knobs.promo_narrow);
   });
   if (rc != DFT3D_OK) return rc;

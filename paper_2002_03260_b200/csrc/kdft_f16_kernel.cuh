@@ -20,9 +20,13 @@
 namespace dft3d {
 
 constexpr int kF16BlockK = 64;          // reals of the contraction per pipeline stage
-constexpr int kF16StagesA = 1;          // raw fp32 data stages (32 KB each)
-constexpr int kF16BytesStageA = kTileM * kF16BlockK * 4;
-constexpr size_t kKdftF16SmemBytes = size_t(kStagesB) * kBytesStageB + size_t(kF16StagesA) * kF16BytesStageA + 1024 + 512;
+constexpr int kF16BytesStageA = kTileM * kF16BlockK * 4;   // raw fp32 data of one stage: 32 KB
+// The raw data of a stage arrives as two halves of 32 reals (16 KB each) with a barrier pair of their own, so that the
+// second half (and the next stage's first) is on its way while the split warps convert the first: a double buffer in
+// the room of one stage.
+constexpr int kF16HalvesA = 2;
+constexpr int kF16BytesHalfA = kF16BytesStageA / 2;
+constexpr size_t kKdftF16SmemBytes = size_t(kStagesB) * kBytesStageB + size_t(kF16BytesStageA) + 1024 + 512;
 
 struct KdftF16Params {
   int k2, bn, n_tiles, chunk_kb;        // as KdftParams; chunk_kb counts 64-real stages
@@ -40,7 +44,7 @@ struct KdftF16Params {
 
 struct KdftF16Shared {
   uint64_t b_full[kStagesB], b_empty[kStagesB];
-  uint64_t a_full[kF16StagesA], a_empty[kF16StagesA];
+  uint64_t a_full[kF16HalvesA], a_empty[kF16HalvesA];
   uint64_t t_full[kStagesT], t_empty[kStagesT];
   uint64_t acc_full, acc_empty;
   uint32_t tmem_base;
@@ -84,7 +88,7 @@ kdft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* smem_b = smem;
   uint8_t* smem_a = smem + size_t(kStagesB) * kBytesStageB;
-  KdftF16Shared& sh = *reinterpret_cast<KdftF16Shared*>(smem_a + size_t(kF16StagesA) * kF16BytesStageA);
+  KdftF16Shared& sh = *reinterpret_cast<KdftF16Shared*>(smem_a + size_t(kF16BytesStageA));
 
   const int tid = threadIdx.x;
   const int warp = tid >> 5;
@@ -92,7 +96,7 @@ kdft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_
 
   if (tid == 0) {
     for (int i = 0; i < kStagesB; ++i) { ptx::mbar_init(&sh.b_full[i], 1); ptx::mbar_init(&sh.b_empty[i], 1); }
-    for (int i = 0; i < kF16StagesA; ++i) { ptx::mbar_init(&sh.a_full[i], 1); ptx::mbar_init(&sh.a_empty[i], 4); }
+    for (int i = 0; i < kF16HalvesA; ++i) { ptx::mbar_init(&sh.a_full[i], 1); ptx::mbar_init(&sh.a_empty[i], 4); }
     for (int i = 0; i < kStagesT; ++i) { ptx::mbar_init(&sh.t_full[i], 4); ptx::mbar_init(&sh.t_empty[i], 1); }
     ptx::mbar_init(&sh.acc_full, 1);
     ptx::mbar_init(&sh.acc_empty, kEpilogueWarps);
@@ -158,16 +162,16 @@ kdft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_
               ptx::tma_load_3d(smem_b + size_t(s) * kBytesStageB, &map_w, &sh.b_full[s], kb * kF16BlockK, nt * p.bn, 0);
               ++ib;
             }
-            {
-              const uint32_t s = ia % kF16StagesA, ph = (ia / kF16StagesA) & 1;
+#pragma unroll
+            for (int h = 0; h < kF16HalvesA; ++h) {
+              const uint32_t s = ia % kF16HalvesA, ph = (ia / kF16HalvesA) & 1;
               DFT3D_WAIT(&sh.a_empty[s], ph ^ 1, 0x102);
-              ptx::mbar_arrive_expect_tx(&sh.a_full[s], kF16BytesStageA);
-              if (MODE == KDFT_CONTIG) {   // two 128-byte-wide halves (the 128B swizzle spans 32 floats)
-                ptx::tma_load_2d(smem_a + size_t(s) * kF16BytesStageA, &map_data, &sh.a_full[s], kb * kF16BlockK, ay);
-                ptx::tma_load_2d(smem_a + size_t(s) * kF16BytesStageA + kF16BytesStageA / 2, &map_data, &sh.a_full[s],
-                                 kb * kF16BlockK + 32, ay);
-              } else
-                ptx::tma_load_3d(smem_a + size_t(s) * kF16BytesStageA, &map_data, &sh.a_full[s], ax, kb * (kF16BlockK / 2), az);
+              ptx::mbar_arrive_expect_tx(&sh.a_full[s], kF16BytesHalfA);
+              if (MODE == KDFT_CONTIG)     // a 128-byte-wide half (the 128B swizzle spans 32 floats)
+                ptx::tma_load_2d(smem_a + size_t(s) * kF16BytesHalfA, &map_data, &sh.a_full[s], kb * kF16BlockK + 32 * h, ay);
+              else                         // 16 rows j of the stage's 32
+                ptx::tma_load_3d(smem_a + size_t(s) * kF16BytesHalfA, &map_data, &sh.a_full[s], ax,
+                                 kb * (kF16BlockK / 2) + 16 * h, az);
               ++ia;
             }
           }
@@ -244,21 +248,21 @@ kdft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_
     const int m = q * 32 + lane;            // lane of the tile
     const uint32_t lane_addr = tmem + (uint32_t(q * 32) << 16);
     int strided_off = 0;                    // float2 index of (j = 0) for this lane in a STRIDED stage
-    if (MODE == KDFT_STRIDED) strided_off = (m / p.lpb) * (kF16BlockK / 2) * p.lpb + (m % p.lpb);
+    if (MODE == KDFT_STRIDED) strided_off = (m / p.lpb) * (kF16BlockK / 4) * p.lpb + (m % p.lpb);   // 16 rows per half
     const uint64_t scale2 = pack2(in_scale, in_scale);
     uint32_t ia = 0, it = 0;
     for (long long t = blockIdx.x; t < total_tiles; t += gridDim.x) {
       for (int kb = 0; kb < num_kb; ++kb) {
-        const uint32_t sa = ia % kF16StagesA, pha = (ia / kF16StagesA) & 1;
         const uint32_t st = it % kStagesT, pht = (it / kStagesT) & 1;
-        DFT3D_WAIT_WARP(&sh.a_full[sa], pha, 0x301);
         uint32_t ph[32], pl[32];                 // 64 scaled values as fp16 pairs: hi pieces, lo pieces
-        const uint8_t* stage = smem_a + size_t(sa) * kF16BytesStageA;
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
+          const uint32_t sa = ia % kF16HalvesA, pha = (ia / kF16HalvesA) & 1;
+          DFT3D_WAIT_WARP(&sh.a_full[sa], pha, 0x301);
+          const uint8_t* stage = smem_a + size_t(sa) * kF16BytesHalfA;
           uint32_t x[32];
           if (MODE == KDFT_CONTIG) {
-            const uint4* rowp = reinterpret_cast<const uint4*>(stage + h * (kF16BytesStageA / 2) + m * 128);
+            const uint4* rowp = reinterpret_cast<const uint4*>(stage + m * 128);
 #pragma unroll
             for (int c = 0; c < 8; ++c) {
               const uint4 v = rowp[c ^ (m & 7)];
@@ -268,16 +272,15 @@ kdft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_
             const uint2* colp = reinterpret_cast<const uint2*>(stage) + strided_off;
 #pragma unroll
             for (int j = 0; j < 16; ++j) {
-              const uint2 v = colp[(h * 16 + j) * p.lpb];
+              const uint2 v = colp[j * p.lpb];
               x[2 * j] = v.x; x[2 * j + 1] = v.y;
             }
           }
-          if (h == 1) {
-            // the stage is refilled by TMA (async proxy): order this thread's reads before that write
-            ptx::fence_proxy_async_smem();
-            __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(&sh.a_empty[sa]);
-          }
+          // the half is refilled by TMA (async proxy): order this thread's reads before that write
+          ptx::fence_proxy_async_smem();
+          __syncwarp();
+          if (lane == 0) ptx::mbar_arrive(&sh.a_empty[sa]);
+          ++ia;
 #pragma unroll
           for (int i = 0; i < 16; ++i)   // element 2i in the low half of each fp16 pair; packed fp32 instructions
             split_half2(mul2(pack2_bits(x[2 * i], x[2 * i + 1]), scale2), ph[h * 16 + i], pl[h * 16 + i]);
@@ -290,7 +293,6 @@ kdft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_
         ptx::tc_fence_before();
         __syncwarp();
         if (lane == 0) ptx::mbar_arrive(&sh.t_full[st]);
-        ++ia;
         ++it;
       }
     }
