@@ -1024,6 +1024,44 @@ def test_fft_8192_with_other_axes_and_destroy_input(lib, oracle):
     assert e.value.status == 2
 
 
+@pytest.mark.slow
+def test_fft_3d_with_an_8192_point_axis_and_the_input_as_workspace(lib):
+    """A 3D plan with one 8192-point axis: four launches through the plan's cube, against the KDFT kernels (whose axes
+    are checked against the oracle one by one).  With DFT3D_AUTO over an 8192-point axis 0 (two passes) and a 100-point
+    axis 1 (KDFT) there are three passes, an odd number, so DFT3D_DESTROY_INPUT may use the input cube as the workspace."""
+    shape = (256, 256, 8192)
+    x = _inputs().cube(shape, "normal", 114, device="cuda")
+    fft = lib.Plan(*shape, mode=lib.DFT3D_FFT)
+    assert fft.launches == 4 and fft.workspace_bytes == x.numel() * 8
+    a = fft(x)
+    _finish(fft)
+    fft.destroy()
+    kd = lib.Plan(*shape, mode=lib.DFT3D_KDFT)
+    b = kd(x)
+    _finish(kd)
+    kd.destroy()
+    assert _rel_l2_gpu(a, b) < SANITY
+    del a, b, x
+    shape = (8192, 100, 128)
+    x = _inputs().cube(shape, "normal", 115, device="cuda")
+    auto = lib.Plan(*shape, mode=lib.DFT3D_AUTO, flags=lib.DFT3D_DESTROY_INPUT, axes=(0, 1))
+    assert auto.workspace_bytes == 0 and auto.launches == 2 + 2     # two for the 8192-point axis, a reduction and a KDFT pass
+    keep = lib.Plan(*shape, mode=lib.DFT3D_AUTO, axes=(0, 1))
+    assert keep.workspace_bytes == x.numel() * 8
+    want = keep(x)
+    _finish(keep)
+    keep.destroy()
+    got = auto(x.clone())
+    _finish(auto)
+    auto.destroy()
+    assert torch.equal(got, want)
+    kd = lib.Plan(*shape, mode=lib.DFT3D_KDFT, axes=(0, 1))
+    b = kd(x)
+    _finish(kd)
+    kd.destroy()
+    assert _rel_l2_gpu(got, b) < SANITY
+
+
 # ------------------------------------------------------------------ inverse nonuniform transform
 
 @pytest.mark.parametrize("split", SPLITS)
