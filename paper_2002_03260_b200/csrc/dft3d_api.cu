@@ -75,7 +75,7 @@ struct Knobs {
   int fft_inplace = 0, fft_no_half = 0, fft_slices = 0;
   int fft_fuse = -1;                                            // axes 1 and 2 in one launch through an L2-resident ring
   int fft_fuse_ring = -1, fft_fuse_writers = -1, fft_fuse_hints = -1;   // its ring length (planes), writer CTAs, L2 hints
-  int kdft_pair = -1, chunk_kb = -1;
+  int kdft_pair = -1, chunk_kb = -1, kdft_ngroup = -1;
   long long wait_limit = 0;                                     // clock budget of the kernels' bounded waits (0 = default)
   int test_silent_producer = 0;                                 // test of the give-up path: TMA producers issue nothing
 };
@@ -108,6 +108,7 @@ Knobs read_knobs() {
   k.fft_fuse_hints = env_int("DFT3D_FFT_FUSE_HINTS", -1);
   k.kdft_pair = env_int("DFT3D_KDFT_PAIR", -1);
   k.chunk_kb = env_int("DFT3D_CHUNK_KB", -1);
+  k.kdft_ngroup = env_int("DFT3D_KDFT_NGROUP", -1);
   if (const char* v = getenv("DFT3D_WAIT_LIMIT_CLOCKS")) k.wait_limit = atoll(v);
   k.test_silent_producer = env_int("DFT3D_TEST_SILENT_PRODUCER", 0);
   return k;
@@ -434,6 +435,9 @@ void fill_f16_params(Params& fp, const dft3d::KdftParams& kp, const KdftAxis& ax
   fp.amax_in = p->d_amax + chain_pos;
   fp.amax_out = p->d_amax + chain_pos + 1;
   fp.wc = kp.wc;
+  // paired-CTA kernel: eight table panels live at a time once there are sixteen or more (measured: 8192 x 8192 26.9 -> 24.5 ms,
+  // 64 x 4096 x 4096 214 -> 202 ms, 2048^3 unchanged; groups of 1, 2, 4, 16, 32 panels are slower)
+  fp.n_group = p->knobs.kdft_ngroup >= 0 ? p->knobs.kdft_ngroup : (kp.n_tiles >= 16 ? 8 : 0);
 }
 
 // chain_pos: position of this pass in the sequence of passes of one execute (fp16 pieces: which amax word to read)

@@ -37,6 +37,8 @@ struct KdftF16Params {
   unsigned int* status;
   long long* profile;
   float out_mul;                        // 2^-10, times 1/n for a scaled inverse
+  int n_group;                          // paired-CTA kernel: table panels (n-tiles) that are live at a time; the tiles go
+                                        // panel group by panel group, all lines within a group (0 or n_tiles: one group)
   const unsigned int* amax_in;          // float bits: largest |input| (an upper bound is enough)
   unsigned int* amax_out;               // float bits: receives the largest |output| (atomic max)
   WaitControl wc;

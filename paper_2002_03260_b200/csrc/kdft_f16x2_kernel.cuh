@@ -148,6 +148,11 @@ kdft_f16x2_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __gri
   // pair tiles: 256 lanes (two M-tiles, one per CTA) x one N-tile; an odd M-tile count leaves the last peer a phantom
   // tile (its loads are out of bounds and zero-filled, its stores masked)
   const long long total_pairs = ((p.m_tiles + 1) / 2) * p.n_tiles;
+  // Order of the tile pairs: within a group of n_group table panels all line tiles, panel fastest; then the next group.
+  // The pairs that run at the same time then share n_group panels (n_group * 4 MiB at 2048 points) instead of all of
+  // them, which keeps the table in L2 at the price of reading the data once per group.
+  const long long ng = (p.n_group > 0 && p.n_group < p.n_tiles && p.n_tiles % p.n_group == 0) ? p.n_group : p.n_tiles;
+  const long long pairs_per_group = ((p.m_tiles + 1) / 2) * ng;
   const long long pair0 = blockIdx.x >> 1, pair_step = gridDim.x >> 1;
   const int num_kb = (p.k2 + kF16BlockK - 1) / kF16BlockK;   // a ragged last stage is zero-filled by TMA on both operands
 
@@ -176,8 +181,8 @@ kdft_f16x2_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __gri
 #pragma unroll
         for (int i = 0; i < kX2StagesB; ++i) leader_b_full[i] = ptx::map_to_cta(&sh.b_full[i], 0);
         for (long long tp = pair0; tp < total_pairs; tp += pair_step) {
-          const long long mt = 2 * (tp / p.n_tiles) + rank;
-          const int nt = int(tp % p.n_tiles);
+          const long long mt = 2 * ((tp % pairs_per_group) / ng) + rank;
+          const int nt = int((tp / pairs_per_group) * ng + tp % ng);
           int ax = 0, ay = 0, az = 0;
           if (MODE == KDFT_CONTIG) {
             ay = int(mt * kTileM);
@@ -349,8 +354,8 @@ kdft_f16x2_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __gri
     const int chunks_per_tile = (num_kb + p.chunk_kb - 1) / p.chunk_kb;
     uint32_t chunk_count = 0;
     for (long long tp = pair0; tp < total_pairs; tp += pair_step) {
-      const long long mt = 2 * (tp / p.n_tiles) + rank;
-      const int nt = int(tp % p.n_tiles);
+      const long long mt = 2 * ((tp % pairs_per_group) / ng) + rank;
+      const int nt = int((tp / pairs_per_group) * ng + tp % ng);
       float acc[128];
 #pragma unroll
       for (int i = 0; i < 128; ++i) acc[i] = 0.0f;
