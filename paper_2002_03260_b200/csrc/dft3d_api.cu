@@ -437,7 +437,7 @@ void fill_f16_params(Params& fp, const dft3d::KdftParams& kp, const KdftAxis& ax
   fp.wc = kp.wc;
   // paired-CTA kernel: eight table panels live at a time once there are sixteen or more (measured: 8192 x 8192 26.9 -> 24.5 ms,
   // 64 x 4096 x 4096 214 -> 202 ms, 2048^3 unchanged; groups of 1, 2, 4, 16, 32 panels are slower)
-  fp.n_group = p->knobs.kdft_ngroup >= 0 ? p->knobs.kdft_ngroup : (kp.n_tiles >= 16 ? 8 : 0);
+  fp.n_group = p->knobs.kdft_ngroup >= 0 ? p->knobs.kdft_ngroup : ((kp.n_tiles >= 16 && ax.pair) ? 8 : 0);
 }
 
 // chain_pos: position of this pass in the sequence of passes of one execute (fp16 pieces: which amax word to read)

@@ -37,7 +37,7 @@ struct KdftF16Params {
   unsigned int* status;
   long long* profile;
   float out_mul;                        // 2^-10, times 1/n for a scaled inverse
-  int n_group;                          // paired-CTA kernel: table panels (n-tiles) that are live at a time; the tiles go
+  int n_group;                          // table panels (n-tiles) that are live at a time; the tiles go
                                         // panel group by panel group, all lines within a group (0 or n_tiles: one group)
   const unsigned int* amax_in;          // float bits: largest |input| (an upper bound is enough)
   unsigned int* amax_out;               // float bits: receives the largest |output| (atomic max)
@@ -120,6 +120,9 @@ kdft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_
   const uint32_t tmem = sh.tmem_base;
 
   const long long total_tiles = p.m_tiles * p.n_tiles;
+  // tile order: panel group by panel group (see KdftF16Params::n_group); one group = panel fastest over all line tiles
+  const long long ng = (p.n_group > 0 && p.n_group < p.n_tiles && p.n_tiles % p.n_group == 0) ? p.n_group : p.n_tiles;
+  const long long tiles_per_group = p.m_tiles * ng;
   const int num_kb = (p.k2 + kF16BlockK - 1) / kF16BlockK;   // a ragged last stage is zero-filled by TMA on both operands
   const uint32_t bytes_b = 2u * uint32_t(p.bn) * 128u;            // two pieces, bn rows of 64 halves
 
@@ -145,8 +148,8 @@ kdft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_
       if (lane == 0 && !p.wc.silent_producer) {
         uint32_t ib = 0, ia = 0;   // running stage counters
         for (long long t = blockIdx.x; t < total_tiles; t += gridDim.x) {
-          const long long mt = t / p.n_tiles;
-          const int nt = int(t % p.n_tiles);
+          const long long mt = (t % tiles_per_group) / ng;
+          const int nt = int((t / tiles_per_group) * ng + t % ng);
           int ax = 0, ay = 0, az = 0;
           if (MODE == KDFT_CONTIG) {
             ay = int(mt * kTileM);
@@ -313,8 +316,8 @@ kdft_f16_axis_kernel(const __grid_constant__ CUtensorMap map_data, const __grid_
     const int chunks_per_tile = (num_kb + p.chunk_kb - 1) / p.chunk_kb;
     uint32_t chunk_count = 0;
     for (long long t = blockIdx.x; t < total_tiles; t += gridDim.x) {
-      const long long mt = t / p.n_tiles;
-      const int nt = int(t % p.n_tiles);
+      const long long mt = (t % tiles_per_group) / ng;
+      const int nt = int((t / tiles_per_group) * ng + t % ng);
       float acc[128];
 #pragma unroll
       for (int i = 0; i < 128; ++i) acc[i] = 0.0f;
